@@ -1,0 +1,165 @@
+/* elitekv.h -- C ABI of the EliteKV decode-attention library for NVIDIA B200 (sm_100a).
+ *
+ * EliteKV (arXiv 2503.01586) shrinks the KV cache of a RoPE multi-head-attention layer in two
+ * steps.  RoPElite (Section 3.1) keeps the rotary embedding only on r "elite" 2-D chunks per
+ * head (each head has its own index set I_r^e); J-LRD (Section 3.2) replaces the remaining key
+ * dims of all heads and the values of all heads by ONE latent vector c = x A^kv per token, from
+ * which they are up-projected by B^kv = [B^k_J, B^v_J].  Per token and layer the cache therefore
+ * holds 2 r n_h rotated key elements plus d_c latent elements (end of Section 3.2).
+ *
+ * Notation used below (the paper's):
+ *   n_h heads, d_h head dim, r elite chunks per head, d_c latent width,
+ *   W_uk = B^k_J  [d_c][n_h (d_h - 2r)]   head h owns columns [h (d_h-2r), (h+1)(d_h-2r))
+ *   W_uv = B^v_J  [d_c][n_h d_h]          head h owns columns [h d_h, (h+1) d_h)
+ *   theta_i = rope_base^(-2 i / d_h), chunk i = dims (2i, 2i+1)            (Section 2.2)
+ *
+ * One decode step of a layer is   elitekv_append -> elitekv_absorb_query -> elitekv_decode.
+ *
+ * General rules
+ *   - Pointers are DEVICE pointers unless a comment says "host".  All floating-point tensors
+ *     are bf16, row-major, densely packed, with the shapes given; index tensors are int32.
+ *   - The caller owns every buffer.  The library allocates device memory only inside
+ *     elitekv_layer_create (tables and repacked weights, released by elitekv_layer_destroy).
+ *   - Every call only enqueues work on `stream` and returns; lengths, positions and page
+ *     tables are read on the device, so a step can be replayed from a CUDA graph.
+ *   - Every function returns 0 on success or a negative elitekv_status.  Nothing throws, exits
+ *     or asserts on the device.  Invalid arguments are rejected before anything is launched.
+ *     Faults that only the device can see (a position beyond max_pos, a page id outside the
+ *     pool, a wait that ran out) are recorded in a status word and the offending access is
+ *     skipped; elitekv_check_status reads that word.
+ */
+#ifndef ELITEKV_H_
+#define ELITEKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* elitekv_stream_t;   /* a cudaStream_t */
+typedef struct elitekv_layer elitekv_layer;     /* opaque */
+
+typedef enum {
+  ELITEKV_OK = 0,
+  ELITEKV_ERR_INVALID_ARG = -1,
+  ELITEKV_ERR_UNSUPPORTED_SHAPE = -2,
+  ELITEKV_ERR_WORKSPACE_TOO_SMALL = -3,
+  ELITEKV_ERR_CUDA = -4,
+  ELITEKV_ERR_TIMEOUT = -5,       /* a bounded device-side wait ran out            */
+  ELITEKV_ERR_BAD_PAGE = -6,      /* page id outside [0, num_pages)                */
+  ELITEKV_ERR_BAD_POSITION = -7   /* position outside [0, max_pos) or the cache    */
+} elitekv_status;
+
+/* Layer description (Sections 3.1 and 3.2).  Host struct; elite_idx is a HOST pointer, the
+ * weights are DEVICE pointers that must stay valid until elitekv_layer_create returns. */
+typedef struct {
+  int32_t n_h, d_h, r, d_c;
+  const int32_t* elite_idx;   /* host [n_h][r]: chunk ids of I_r^e per head, distinct, each in
+                                 [0, d_h/2).  Their order is the order of the chunks inside a
+                                 cached rope row and inside k_e / q_rope.                     */
+  float rope_base;            /* 10000 for LLaMA2                                              */
+  float softmax_scale;        /* 0 selects 1/sqrt(d_h) (Section 2.1)                           */
+  int32_t pair_mode;          /* how chunk i maps to query dims: 0 = (2i, 2i+1) as in Section
+                                 2.2; 1 = (i, i + d_h/2).  Keys arrive already paired.         */
+  const void* W_uk;           /* bf16 [d_c][n_h*(d_h-2r)]  (B^k_J)                             */
+  const void* W_uv;           /* bf16 [d_c][n_h*d_h]       (B^v_J)                             */
+  int32_t max_pos;            /* positions are in [0, max_pos)                                 */
+  const float* cos_sin;       /* optional DEVICE fp32 [max_pos][d_h/2][2] = (cos, sin) of
+                                 pos*theta_i.  NULL: the library tabulates them itself in double
+                                 precision at create time.  With a caller table the rotated
+                                 values are a pure function of the table (each product and sum
+                                 rounded separately in fp32, then bf16 nearest-even).          */
+  int32_t decode_kernel;      /* 0 = choose by shape; 1 = generic CUDA-core kernel;
+                                 2 = tensor-core (tcgen05) kernel, error if the shape is not
+                                 covered.                                                      */
+} elitekv_params;
+
+/* The two cache planes.  Contiguous (page_table == NULL): sequence s, position p live in row
+ * s*max_ctx + p.  Paged: row page_table[s][p / page_size]*page_size + p % page_size.  A rope
+ * row is [n_h][r][2] (head-major, chunk order of elite_idx, (even, odd)); a latent row is
+ * [d_c].  This struct lives on the HOST; its pointer members are DEVICE pointers. */
+typedef struct {
+  void* rope;                  /* bf16 [rows][n_h*2r]                                          */
+  void* latent;                /* bf16 [rows][d_c]                                             */
+  const int32_t* page_table;   /* int32 [n_seqs][max_pages_per_seq] or NULL                    */
+  int32_t page_size;           /* tokens per page (64 in the benchmarks), power of two         */
+  int32_t max_pages_per_seq;
+  int64_t num_pages;           /* paged: pages in the pool (rows = num_pages*page_size)        */
+  int64_t max_ctx;             /* contiguous: rows per sequence                                */
+  int32_t n_seqs;              /* sequences the cache (and page table) is laid out for         */
+} elitekv_cache;
+
+/* Validates the description (r <= d_h/2, distinct in-range indices, d_c % 8 == 0, ...), copies
+ * the index sets, tabulates (cos, sin) and repacks W_uk for the absorption kernel.  Must be
+ * called with the target device current.  `*out` is written only on success. */
+int elitekv_layer_create(const elitekv_params* params, elitekv_layer** out);
+int elitekv_layer_destroy(elitekv_layer* layer);
+
+/* Cache append (Section 3.1, "incorporated into the KV cache"; Section 3.2, shared latent).
+ * For each of the T new tokens: rotate chunk j of head h by R(pos * theta_{idx[h][j]})
+ * (Eq. 1a; (x0,x1) -> (x0 cos - x1 sin, x0 sin + x1 cos)) and write the rope row and the
+ * latent row to the token's cache row.  The rotation happens here once; decode never rotates
+ * keys again.
+ *   k_e    bf16  [T][n_h][r][2]  un-rotated elite key chunks (x W^k_{e,h})
+ *   c      bf16  [T][d_c]        latent (x A^kv), copied bit for bit
+ *   seq_id int32 [T], pos int32 [T] (0-based position inside the sequence)
+ * Tokens must target distinct rows.  T == 0 is a no-op. */
+int elitekv_append(const elitekv_layer* layer, const elitekv_cache* cache, const void* k_e,
+                   const void* c, const int32_t* seq_id, const int32_t* pos, int64_t T,
+                   elitekv_stream_t stream);
+
+/* Query preparation (score equation of Section 3.1; absorption of B^k, Section 5).
+ *   q      bf16  [B][n_h][d_h]  un-rotated queries,  q_pos int32 [B]
+ *   q_rope bf16  [B][n_h][2r]   elite chunks of q rotated at q_pos
+ *   q_abs  bf16  [B][n_h][d_c]  q_nope[b,h,:] . W_uk,h^T, q_nope = the other d_h-2r dims of
+ *                               q[b,h] in ascending order; fp32 accumulation. */
+int elitekv_absorb_query(const elitekv_layer* layer, const void* q, const int32_t* q_pos,
+                         int32_t B, void* q_rope, void* q_abs, elitekv_stream_t stream);
+
+/* Scratch needed by elitekv_decode for a batch of B sequences (split-K partial results and
+ * the work plan).  It depends on the layer shape, on B and on the device, not on the lengths. */
+int elitekv_decode_workspace_size(const elitekv_layer* layer, int32_t B, size_t* bytes);
+
+/* Decode attention over the compressed cache (Sections 2.1, 3.1, 3.2, 5):
+ *   s[b,h,t] = q_rope[b,h] . k_rope[t,h] + q_abs[b,h] . c[t]        t < seq_lens[b]
+ *   p = softmax(scale * s),   o[b,h] = (sum_t p[b,h,t] c[t]) . W_uv,h
+ * seq_lens[b] counts the cached tokens INCLUDING the one just appended (the query attends to
+ * its own token).  seq_lens[b] == 0 gives a zero row.
+ *   out bf16 [B][n_h][d_h];  workspace: 256-byte aligned, at least
+ *   elitekv_decode_workspace_size bytes, private to this call until the stream reaches its end.
+ * Launches: plan, split-K attention, combine + up-projection. */
+int elitekv_decode(const elitekv_layer* layer, const elitekv_cache* cache, const void* q_rope,
+                   const void* q_abs, const int32_t* seq_lens, int32_t B, void* workspace,
+                   size_t workspace_bytes, void* out, elitekv_stream_t stream);
+
+/* Work plan of the split-K kernel, exported for inspection (the paper has no counterpart: it
+ * is this library's load balancer for ragged batches).  Cuts the batch's token tiles into at
+ * most `max_items` pieces of near-equal size, never across a sequence.
+ *   items int32 [max_items][4] = (sequence, first token, token count, 0);  unused entries have
+ *   sequence = -1.   seq_first_item int32 [B+1]: items of sequence b are
+ *   [seq_first_item[b], seq_first_item[b+1]). */
+int elitekv_plan(const int32_t* seq_lens, int32_t B, int32_t tile_tokens, int32_t max_items,
+                 int32_t* items, int32_t* seq_first_item, elitekv_stream_t stream);
+
+/* Synchronises `stream`, returns the layer's device status word (0 or a negative
+ * elitekv_status recorded by a kernel) and clears it. */
+int elitekv_check_status(const elitekv_layer* layer, elitekv_stream_t stream);
+
+/* Comparator: uncompressed RoPE multi-head attention decode (Sections 2.1 and 2.2) over a
+ * contiguous cache of rotated keys and values.
+ *   q_hat bf16 [B][n_h][d_h] rotated query;  K_hat, V bf16 [B][max_ctx][n_h][d_h];
+ *   out bf16 [B][n_h][d_h];  scale 0 selects 1/sqrt(d_h). */
+int elitekv_mha_workspace_size(int32_t B, int32_t n_h, int32_t d_h, size_t* bytes);
+int elitekv_mha_decode(const void* q_hat, const void* K_hat, const void* V,
+                       const int32_t* seq_lens, int32_t B, int32_t n_h, int32_t d_h,
+                       int64_t max_ctx, float scale, void* workspace, size_t workspace_bytes,
+                       void* out, elitekv_stream_t stream);
+
+const char* elitekv_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ELITEKV_H_ */

@@ -1,0 +1,130 @@
+// Shared declarations of the EliteKV CUDA library (sm_100a).  Host-side layer object, status
+// word helpers and small device utilities.  Nothing here is used by the CPU oracle.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/elitekv.h"
+
+typedef __nv_bfloat16 bf16;
+typedef __nv_bfloat162 bf162;
+
+// The work plan cuts sequences in units of this many tokens (also the page size the
+// tensor-core kernel expects).
+#define ELITEKV_TILE_TOKENS 64
+
+struct elitekv_layer {
+  int n_h, d_h, r, d_c, dn;        // dn = d_h - 2r (un-rotated key dims per head)
+  float rope_base;
+  float scale;                     // softmax scale actually used
+  int pair_mode;
+  int max_pos;
+  int decode_kernel;
+  int device;
+  int sm_count;
+  int smem_optin;                  // max dynamic shared memory per block
+  int32_t* d_idx;                  // [n_h][r] elite chunk ids
+  int32_t* d_qdims;                // [n_h][d_h]: 2r dims of the elite chunks in cache order,
+                                   // then the dn remaining dims ascending
+  const float2* d_cs;              // [max_pos][d_h/2] (cos, sin)
+  float2* d_cs_owned;              // same pointer when the library built the table
+  bf16* d_WukT;                    // [n_h][dn][d_c]: W_uk regrouped per head, d_c contiguous
+  bf16* d_Wuv;                     // [d_c][n_h*d_h] private copy
+  int32_t* d_status;               // [4] device status word: code, detail0, detail1, count
+};
+
+#define EKV_CUDA_OK(expr)                                   \
+  do {                                                      \
+    cudaError_t _e = (expr);                                \
+    if (_e != cudaSuccess) return ELITEKV_ERR_CUDA;         \
+  } while (0)
+
+// Records the first device-side fault; later ones only bump the counter.
+__device__ __forceinline__ void ekv_record(int32_t* status, int code, int d0, int d1) {
+  if (atomicCAS(&status[0], 0, code) == 0) {
+    status[1] = d0;
+    status[2] = d1;
+  }
+  atomicAdd(&status[3], 1);
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem_src));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
+}
+
+// Where a (sequence, position) lives in the cache planes.
+struct CacheView {
+  const int32_t* page_table;
+  int page_shift, page_mask, max_pages_per_seq;
+  long long num_pages, max_ctx;
+  int n_seqs;
+};
+
+// Row index (in tokens) of (seq, pos), or -1 with (code, detail) left for the caller to record.
+__device__ __forceinline__ long long ekv_token_row(const CacheView& cv, int seq, int pos,
+                                                   int* code, int* detail) {
+  *code = ELITEKV_ERR_BAD_POSITION;
+  *detail = pos;
+  if (seq < 0 || seq >= cv.n_seqs || pos < 0) return -1;
+  if (cv.page_table == nullptr) {
+    if (pos >= cv.max_ctx) return -1;
+    return (long long)seq * cv.max_ctx + pos;
+  }
+  int pi = pos >> cv.page_shift;
+  if (pi >= cv.max_pages_per_seq) return -1;
+  int page = cv.page_table[(long long)seq * cv.max_pages_per_seq + pi];
+  if (page < 0 || page >= cv.num_pages) {
+    *code = ELITEKV_ERR_BAD_PAGE;
+    *detail = page;
+    return -1;
+  }
+  return ((long long)page << cv.page_shift) + (pos & cv.page_mask);
+}
+
+// Host-side helpers shared by the entry points.
+int ekv_make_view(const elitekv_cache* cache, CacheView* out);
+
+// Kernel launchers (one per .cu file).
+int ekv_launch_append(const elitekv_layer* L, const elitekv_cache* cache, const CacheView& cv,
+                      const void* k_e, const void* c, const int32_t* seq_id, const int32_t* pos,
+                      long long T, cudaStream_t st);
+int ekv_launch_absorb(const elitekv_layer* L, const void* q, const int32_t* q_pos, int B,
+                      void* q_rope, void* q_abs, cudaStream_t st);
+int ekv_launch_plan(const int32_t* seq_lens, int B, int tile_tokens, int max_items, int32_t* items,
+                    int32_t* seq_first_item, cudaStream_t st);
+
+struct DecodeScratch {
+  int max_items;          // capacity of the plan
+  int32_t* items;         // [max_items][4]
+  int32_t* seq_first;     // [B+1]
+  float* part_acc;        // [max_items][n_h][d_c]
+  float* part_ml;         // [max_items][n_h][2]  (running max in log2 units, running sum)
+};
+
+int ekv_generic_supported(const elitekv_layer* L);
+int ekv_generic_max_items(const elitekv_layer* L, int B);
+int ekv_launch_decode_generic(const elitekv_layer* L, const elitekv_cache* cache,
+                              const CacheView& cv, const void* q_rope, const void* q_abs, int B,
+                              const DecodeScratch& ws, cudaStream_t st);
+int ekv_launch_combine(const elitekv_layer* L, int B, const DecodeScratch& ws, void* out,
+                       cudaStream_t st);

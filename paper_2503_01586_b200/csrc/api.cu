@@ -1,0 +1,94 @@
+// C entry points: argument checks, workspace carving, kernel selection.
+#include "common.cuh"
+
+namespace {
+
+inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+// Which split-K kernel a layer uses: 1 = generic CUDA-core kernel.
+int select_kernel(const elitekv_layer* L) {
+  if (L->decode_kernel == 2) return -1;          // tensor-core kernel: not built for this shape
+  return ekv_generic_supported(L) ? 1 : -1;
+}
+
+int max_items_for(const elitekv_layer* L, int B, int kernel) {
+  (void)kernel;
+  return ekv_generic_max_items(L, B);
+}
+
+struct Carve {
+  size_t off_items, off_first, off_ml, off_acc, total;
+};
+
+Carve carve(const elitekv_layer* L, int B, int max_items) {
+  Carve c;
+  size_t o = 0;
+  c.off_items = o; o = align256(o + sizeof(int32_t) * 4 * (size_t)max_items);
+  c.off_first = o; o = align256(o + sizeof(int32_t) * ((size_t)B + 1));
+  c.off_ml = o;    o = align256(o + sizeof(float) * 2 * (size_t)max_items * L->n_h);
+  c.off_acc = o;   o = align256(o + sizeof(float) * (size_t)max_items * L->n_h * L->d_c);
+  c.total = o;
+  return c;
+}
+
+}  // namespace
+
+extern "C" int elitekv_append(const elitekv_layer* L, const elitekv_cache* cache, const void* k_e,
+                              const void* c, const int32_t* seq_id, const int32_t* pos, int64_t T,
+                              elitekv_stream_t stream) {
+  if (!L || !cache || T < 0) return ELITEKV_ERR_INVALID_ARG;
+  if (T == 0) return ELITEKV_OK;
+  if (!c || !seq_id || !pos || (L->r > 0 && !k_e)) return ELITEKV_ERR_INVALID_ARG;
+  if (((uintptr_t)k_e & 15) || ((uintptr_t)c & 15)) return ELITEKV_ERR_INVALID_ARG;
+  CacheView cv;
+  int rc = ekv_make_view(cache, &cv);
+  if (rc != ELITEKV_OK) return rc;
+  return ekv_launch_append(L, cache, cv, k_e, c, seq_id, pos, T, (cudaStream_t)stream);
+}
+
+extern "C" int elitekv_absorb_query(const elitekv_layer* L, const void* q, const int32_t* q_pos,
+                                    int32_t B, void* q_rope, void* q_abs, elitekv_stream_t stream) {
+  if (!L || !q || !q_pos || !q_abs || B < 0 || (L->r > 0 && !q_rope)) return ELITEKV_ERR_INVALID_ARG;
+  if (((uintptr_t)q & 15) || ((uintptr_t)q_abs & 15) || ((uintptr_t)q_rope & 3))
+    return ELITEKV_ERR_INVALID_ARG;
+  return ekv_launch_absorb(L, q, q_pos, B, q_rope, q_abs, (cudaStream_t)stream);
+}
+
+extern "C" int elitekv_decode_workspace_size(const elitekv_layer* L, int32_t B, size_t* bytes) {
+  if (!L || !bytes || B <= 0) return ELITEKV_ERR_INVALID_ARG;
+  const int kernel = select_kernel(L);
+  if (kernel < 0) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
+  *bytes = carve(L, B, max_items_for(L, B, kernel)).total;
+  return ELITEKV_OK;
+}
+
+extern "C" int elitekv_decode(const elitekv_layer* L, const elitekv_cache* cache,
+                              const void* q_rope, const void* q_abs, const int32_t* seq_lens,
+                              int32_t B, void* workspace, size_t workspace_bytes, void* out,
+                              elitekv_stream_t stream) {
+  if (!L || !cache || !q_abs || !seq_lens || !workspace || !out || B <= 0 || (L->r > 0 && !q_rope))
+    return ELITEKV_ERR_INVALID_ARG;
+  if (((uintptr_t)q_abs & 15) || ((uintptr_t)out & 3)) return ELITEKV_ERR_INVALID_ARG;
+  if (B > cache->n_seqs) return ELITEKV_ERR_INVALID_ARG;
+  const int kernel = select_kernel(L);
+  if (kernel < 0) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
+  CacheView cv;
+  int rc = ekv_make_view(cache, &cv);
+  if (rc != ELITEKV_OK) return rc;
+  const int max_items = max_items_for(L, B, kernel);
+  const Carve cw = carve(L, B, max_items);
+  if (((uintptr_t)workspace & 255) || workspace_bytes < cw.total) return ELITEKV_ERR_WORKSPACE_TOO_SMALL;
+  unsigned char* base = (unsigned char*)workspace;
+  DecodeScratch ws;
+  ws.max_items = max_items;
+  ws.items = (int32_t*)(base + cw.off_items);
+  ws.seq_first = (int32_t*)(base + cw.off_first);
+  ws.part_ml = (float*)(base + cw.off_ml);
+  ws.part_acc = (float*)(base + cw.off_acc);
+  cudaStream_t st = (cudaStream_t)stream;
+  rc = ekv_launch_plan(seq_lens, B, ELITEKV_TILE_TOKENS, max_items, ws.items, ws.seq_first, st);
+  if (rc != ELITEKV_OK) return rc;
+  rc = ekv_launch_decode_generic(L, cache, cv, q_rope, q_abs, B, ws, st);
+  if (rc != ELITEKV_OK) return rc;
+  return ekv_launch_combine(L, B, ws, out, st);
+}

@@ -1,0 +1,107 @@
+// Work plan for the split-K decode kernels: cuts every sequence's token range into pieces of
+// near-equal size so that ragged batches keep all SMs busy.  Integer arithmetic only, on
+// device-resident lengths, so a decode step never synchronises with the host.  (The paper
+// leaves scheduling open; this is the library's load balancer.)
+//
+// With tiles_b = ceil(len_b / tile), total = sum tiles_b and budget = max_items - B:
+//   target   = max(1, ceil(total / budget))            tiles per item
+//   pieces_b = ceil(tiles_b / target)                  (sum <= budget + B = max_items)
+//   piece j of sequence b covers tiles [tiles_b*j/pieces_b, tiles_b*(j+1)/pieces_b)
+#include "common.cuh"
+
+namespace {
+
+constexpr int kPlanThreads = 1024;
+
+__device__ __forceinline__ int block_exclusive_scan(int v, int* smem, int* total) {
+  // Hillis-Steele over blockDim.x entries
+  const int t = threadIdx.x;
+  smem[t] = v;
+  __syncthreads();
+  for (int o = 1; o < blockDim.x; o <<= 1) {
+    int x = t >= o ? smem[t - o] : 0;
+    __syncthreads();
+    smem[t] += x;
+    __syncthreads();
+  }
+  int incl = smem[t];
+  *total = smem[blockDim.x - 1];
+  __syncthreads();
+  return incl - v;
+}
+
+__global__ void __launch_bounds__(kPlanThreads)
+plan_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int max_items,
+            int32_t* __restrict__ items, int32_t* __restrict__ seq_first) {
+  __shared__ int scan[kPlanThreads];
+  __shared__ long long s_total;
+  const int t = threadIdx.x;
+  if (t == 0) s_total = 0;
+  __syncthreads();
+  long long local = 0;
+  for (int b = t; b < B; b += blockDim.x) {
+    int n = seq_lens[b];
+    local += n > 0 ? (n + tile - 1) / tile : 0;
+  }
+  atomicAdd((unsigned long long*)&s_total, (unsigned long long)local);
+  __syncthreads();
+  const long long total = s_total;
+  const long long budget = max_items - B > 0 ? max_items - B : 1;
+  long long target = (total + budget - 1) / budget;
+  if (target < 1) target = 1;
+
+  int carry = 0;
+  for (int b0 = 0; b0 < B; b0 += blockDim.x) {
+    const int b = b0 + t;
+    int n = 0, tiles = 0, pieces = 0;
+    if (b < B) {
+      n = seq_lens[b];
+      tiles = n > 0 ? (n + tile - 1) / tile : 0;
+      pieces = (int)((tiles + target - 1) / target);
+    }
+    int chunk_total;
+    const int first = carry + block_exclusive_scan(pieces, scan, &chunk_total);
+    if (b < B) {
+      seq_first[b] = first;
+      for (int j = 0; j < pieces; ++j) {
+        const int ta = (int)((long long)tiles * j / pieces);
+        const int tb = (int)((long long)tiles * (j + 1) / pieces);
+        const int tok0 = ta * tile;
+        const int tok1 = min(tb * tile, n);
+        const int it = first + j;
+        if (it < max_items) {
+          items[4 * it + 0] = b;
+          items[4 * it + 1] = tok0;
+          items[4 * it + 2] = tok1 - tok0;
+          items[4 * it + 3] = 0;
+        }
+      }
+    }
+    carry += chunk_total;
+  }
+  if (t == 0) seq_first[B] = carry;
+  for (int it = carry + t; it < max_items; it += blockDim.x) {
+    items[4 * it + 0] = -1;
+    items[4 * it + 1] = 0;
+    items[4 * it + 2] = 0;
+    items[4 * it + 3] = 0;
+  }
+}
+
+}  // namespace
+
+int ekv_launch_plan(const int32_t* seq_lens, int B, int tile_tokens, int max_items, int32_t* items,
+                    int32_t* seq_first_item, cudaStream_t st) {
+  plan_kernel<<<1, kPlanThreads, 0, st>>>(seq_lens, B, tile_tokens, max_items, items, seq_first_item);
+  EKV_CUDA_OK(cudaGetLastError());
+  return ELITEKV_OK;
+}
+
+extern "C" int elitekv_plan(const int32_t* seq_lens, int32_t B, int32_t tile_tokens,
+                            int32_t max_items, int32_t* items, int32_t* seq_first_item,
+                            elitekv_stream_t stream) {
+  if (!seq_lens || !items || !seq_first_item || B <= 0 || tile_tokens <= 0 || max_items <= B)
+    return ELITEKV_ERR_INVALID_ARG;
+  return ekv_launch_plan(seq_lens, B, tile_tokens, max_items, items, seq_first_item,
+                         (cudaStream_t)stream);
+}

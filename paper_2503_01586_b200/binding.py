@@ -1,0 +1,224 @@
+"""ctypes binding of libelitekv.so: same names as the C ABI, argument marshalling only.
+
+torch supplies device memory (`tensor.data_ptr()`) and the current stream; every step of the
+path runs in the library's CUDA kernels.  There is no CPU or PyTorch fallback: if the shared
+library is missing or fails to load, importing this module's functions raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libelitekv.so")
+
+OK = 0
+ERR_INVALID_ARG = -1
+ERR_UNSUPPORTED_SHAPE = -2
+ERR_WORKSPACE_TOO_SMALL = -3
+ERR_CUDA = -4
+ERR_TIMEOUT = -5
+ERR_BAD_PAGE = -6
+ERR_BAD_POSITION = -7
+
+
+class ElitekvError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+class Params(C.Structure):
+    _fields_ = [("n_h", C.c_int32), ("d_h", C.c_int32), ("r", C.c_int32), ("d_c", C.c_int32),
+                ("elite_idx", C.c_void_p), ("rope_base", C.c_float), ("softmax_scale", C.c_float),
+                ("pair_mode", C.c_int32), ("W_uk", C.c_void_p), ("W_uv", C.c_void_p),
+                ("max_pos", C.c_int32), ("cos_sin", C.c_void_p), ("decode_kernel", C.c_int32)]
+
+
+class CacheDesc(C.Structure):
+    _fields_ = [("rope", C.c_void_p), ("latent", C.c_void_p), ("page_table", C.c_void_p),
+                ("page_size", C.c_int32), ("max_pages_per_seq", C.c_int32),
+                ("num_pages", C.c_int64), ("max_ctx", C.c_int64), ("n_seqs", C.c_int32)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads the shared library (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with "
+                              "`python -m paper_2503_01586_b200.build` (needs nvcc, sm_100a)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+        L.elitekv_layer_create.argtypes = [C.POINTER(Params), C.POINTER(vp)]
+        L.elitekv_layer_destroy.argtypes = [vp]
+        L.elitekv_append.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, vp, i64, vp]
+        L.elitekv_absorb_query.argtypes = [vp, vp, vp, i32, vp, vp, vp]
+        L.elitekv_decode_workspace_size.argtypes = [vp, i32, C.POINTER(sz)]
+        L.elitekv_decode.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, i32, vp, sz, vp, vp]
+        L.elitekv_plan.argtypes = [vp, i32, i32, i32, vp, vp, vp]
+        L.elitekv_check_status.argtypes = [vp, vp]
+        L.elitekv_mha_workspace_size.argtypes = [i32, i32, i32, C.POINTER(sz)]
+        L.elitekv_mha_decode.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, C.c_float, vp, sz, vp, vp]
+        L.elitekv_strerror.argtypes = [C.c_int]
+        L.elitekv_strerror.restype = C.c_char_p
+        for name in ("elitekv_layer_create", "elitekv_layer_destroy", "elitekv_append",
+                     "elitekv_absorb_query", "elitekv_decode_workspace_size", "elitekv_decode",
+                     "elitekv_plan", "elitekv_check_status", "elitekv_mha_workspace_size",
+                     "elitekv_mha_decode"):
+            getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().elitekv_strerror(int(code)).decode()
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise ElitekvError(code, where)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_contiguous()
+    return t.data_ptr()
+
+
+def _dev(t: torch.Tensor, dtype) -> torch.Tensor:
+    assert t.is_cuda and t.dtype == dtype and t.is_contiguous(), (t.device, t.dtype)
+    return t
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+class Layer:
+    """Owns an `elitekv_layer*`.  elite_idx is an int32 CPU tensor [n_h][r]; W_uk, W_uv are
+    bf16 CUDA tensors; cos_sin an optional fp32 CUDA tensor [max_pos][d_h/2][2]."""
+
+    def __init__(self, n_h, d_h, r, d_c, elite_idx, W_uk, W_uv, max_pos, rope_base=10000.0,
+                 softmax_scale=0.0, pair_mode=0, cos_sin=None, decode_kernel=0):
+        idx = elite_idx.to(torch.int32).contiguous().cpu()
+        assert tuple(idx.shape) == (n_h, r)
+        self.n_h, self.d_h, self.r, self.d_c = n_h, d_h, r, d_c
+        self._keep = (idx, cos_sin)
+        p = Params(n_h, d_h, r, d_c, idx.data_ptr() if r > 0 else None, rope_base, softmax_scale,
+                   pair_mode, _ptr(W_uk) if W_uk is not None and W_uk.numel() else None,
+                   _ptr(_dev(W_uv, torch.bfloat16)), max_pos,
+                   _ptr(_dev(cos_sin, torch.float32)) if cos_sin is not None else None,
+                   decode_kernel)
+        h = C.c_void_p()
+        _check(lib().elitekv_layer_create(C.byref(p), C.byref(h)), "elitekv_layer_create")
+        self.handle = h
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib().elitekv_layer_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def make_cache(rope: torch.Tensor, latent: torch.Tensor, *, n_seqs: int, max_ctx: int = 0,
+               page_table: Optional[torch.Tensor] = None, page_size: int = 64) -> CacheDesc:
+    """Describes caller-owned cache planes.  Keep the tensors alive while the descriptor is used."""
+    _dev(rope, torch.bfloat16)
+    _dev(latent, torch.bfloat16)
+    d = CacheDesc()
+    d.rope, d.latent = rope.data_ptr(), latent.data_ptr()
+    d.n_seqs = n_seqs
+    if page_table is not None:
+        _dev(page_table, torch.int32)
+        d.page_table = page_table.data_ptr()
+        d.page_size = page_size
+        d.max_pages_per_seq = page_table.shape[1]
+        d.num_pages = latent.shape[0] // page_size if latent.dim() == 2 else latent.shape[0]
+        d.max_ctx = 0
+    else:
+        d.page_table = None
+        d.page_size = page_size
+        d.max_ctx = max_ctx
+    return d
+
+
+def elitekv_append(layer: Layer, cache: CacheDesc, k_e, c, seq_id, pos) -> None:
+    T = c.shape[0]
+    _check(lib().elitekv_append(layer.handle, C.byref(cache), _ptr(k_e), _ptr(_dev(c, torch.bfloat16)),
+                                _ptr(_dev(seq_id, torch.int32)), _ptr(_dev(pos, torch.int32)), T,
+                                _stream()), "elitekv_append")
+
+
+def elitekv_absorb_query(layer: Layer, q, q_pos, q_rope=None, q_abs=None):
+    B = q.shape[0]
+    _dev(q, torch.bfloat16)
+    if q_rope is None:
+        q_rope = torch.empty((B, layer.n_h, 2 * layer.r), dtype=torch.bfloat16, device=q.device)
+    if q_abs is None:
+        q_abs = torch.empty((B, layer.n_h, layer.d_c), dtype=torch.bfloat16, device=q.device)
+    _check(lib().elitekv_absorb_query(layer.handle, _ptr(q), _ptr(_dev(q_pos, torch.int32)), B,
+                                      _ptr(q_rope), _ptr(q_abs), _stream()), "elitekv_absorb_query")
+    return q_rope, q_abs
+
+
+def elitekv_decode_workspace_size(layer: Layer, B: int) -> int:
+    n = C.c_size_t()
+    _check(lib().elitekv_decode_workspace_size(layer.handle, B, C.byref(n)),
+           "elitekv_decode_workspace_size")
+    return n.value
+
+
+def elitekv_decode(layer: Layer, cache: CacheDesc, q_rope, q_abs, seq_lens, workspace, out=None):
+    B = q_abs.shape[0]
+    if out is None:
+        out = torch.empty((B, layer.n_h, layer.d_h), dtype=torch.bfloat16, device=q_abs.device)
+    _check(lib().elitekv_decode(layer.handle, C.byref(cache), _ptr(q_rope), _ptr(_dev(q_abs, torch.bfloat16)),
+                                _ptr(_dev(seq_lens, torch.int32)), B, workspace.data_ptr(),
+                                workspace.numel() * workspace.element_size(), _ptr(out), _stream()),
+           "elitekv_decode")
+    return out
+
+
+def elitekv_plan(seq_lens, tile_tokens: int, max_items: int):
+    B = seq_lens.shape[0]
+    items = torch.empty((max_items, 4), dtype=torch.int32, device=seq_lens.device)
+    first = torch.empty((B + 1,), dtype=torch.int32, device=seq_lens.device)
+    _check(lib().elitekv_plan(_ptr(_dev(seq_lens, torch.int32)), B, tile_tokens, max_items,
+                              _ptr(items), _ptr(first), _stream()), "elitekv_plan")
+    return items, first
+
+
+def elitekv_check_status(layer: Layer) -> int:
+    return lib().elitekv_check_status(layer.handle, _stream())
+
+
+def elitekv_mha_workspace_size(B: int, n_h: int, d_h: int) -> int:
+    n = C.c_size_t()
+    _check(lib().elitekv_mha_workspace_size(B, n_h, d_h, C.byref(n)), "elitekv_mha_workspace_size")
+    return n.value
+
+
+def elitekv_mha_decode(q_hat, K_hat, V, seq_lens, workspace, out=None, scale: float = 0.0):
+    B, n_h, d_h = q_hat.shape
+    max_ctx = K_hat.shape[1]
+    if out is None:
+        out = torch.empty_like(q_hat)
+    _check(lib().elitekv_mha_decode(_ptr(_dev(q_hat, torch.bfloat16)), _ptr(_dev(K_hat, torch.bfloat16)),
+                                    _ptr(_dev(V, torch.bfloat16)), _ptr(_dev(seq_lens, torch.int32)),
+                                    B, n_h, d_h, max_ctx, scale, workspace.data_ptr(),
+                                    workspace.numel() * workspace.element_size(), _ptr(out),
+                                    _stream()), "elitekv_mha_decode")
+    return out

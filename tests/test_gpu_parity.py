@@ -1,0 +1,286 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the float64 oracle on the
+same seeded bytes.  Integer/layout work must match bit for bit; floating-point outputs within
+relative L2 error 1e-2 and max abs error 3e-2 (bf16 inputs, fp32 accumulation)."""
+import ctypes as C
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import elitekv_oracle as O
+from paper_2503_01586_b200 import inputs as gen
+
+from . import harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ek():
+    from paper_2503_01586_b200 import binding
+    binding.lib()
+    return binding
+
+
+SMALL = gen.Workload("small", n_h=6, d_h=32, r=3, d_c=72, d=192, B=3, ctx=150, seed=41)
+
+
+# ------------------------------------------------------------------ append
+@pytest.mark.parametrize("paged", [False, True])
+def test_append_layout_and_bits(ek, paged):
+    w = replace(SMALL, paged=paged, page_size=16, seed=42 + paged)
+    lens = [37, 1, 100]
+    table32 = torch.from_numpy(O.rope_table_f32(128, w.d_h, w.rope_base)).cuda()
+    st = H.setup(w, lens=lens, cos_sin=table32, fill=False)
+    # canary pattern in both planes; append must touch only the addressed rows
+    g = torch.Generator(device="cpu").manual_seed(5)
+    rope0 = torch.randint(0, 2 ** 15, tuple(st.rope_plane.shape), generator=g, dtype=torch.int16)
+    lat0 = torch.randint(0, 2 ** 15, tuple(st.latent_plane.shape), generator=g, dtype=torch.int16)
+    st.rope_plane.copy_(rope0.view(torch.bfloat16))
+    st.latent_plane.copy_(lat0.view(torch.bfloat16))
+    # append in two calls with a shuffled token order
+    N = st.c.shape[0]
+    perm = torch.randperm(N, generator=g).cuda()
+    half = N // 2
+    for sel in (perm[:half], perm[half:]):
+        ek.elitekv_append(st.layer, st.cache, st.k_e[sel].contiguous(), st.c[sel].contiguous(),
+                          st.seq_id[sel].contiguous(), st.pos[sel].contiguous())
+    torch.cuda.synchronize()
+    assert ek.elitekv_check_status(st.layer) == 0
+    pt = st.page_table.cpu().numpy() if paged else None
+    max_ctx = st.cache.max_ctx if not paged else None
+    rope_exp, lat_exp = O.append_expected(
+        rope0.numpy().view(np.uint16), lat0.numpy().view(np.uint16), H.bits(st.k_e), H.bits(st.c),
+        st.seq_id.cpu().numpy(), st.pos.cpu().numpy(), st.idx.numpy(), w.d_h, base=w.rope_base,
+        max_ctx=max_ctx, page_table=pt, page_size=w.page_size, table32=table32.cpu().numpy())
+    assert np.array_equal(H.bits(st.latent_plane), lat_exp)
+    assert np.array_equal(H.bits(st.rope_plane), rope_exp)
+
+
+def test_append_own_table_within_one_ulp(ek):
+    w = replace(SMALL, seed=44)
+    st = H.setup(w, lens=[64, 65, 129])
+    torch.cuda.synchronize()
+    rope0 = np.zeros(tuple(st.rope_plane.shape), dtype=np.uint16)
+    lat0 = np.zeros(tuple(st.latent_plane.shape), dtype=np.uint16)
+    rope_exp, lat_exp = O.append_expected(rope0, lat0, H.bits(st.k_e), H.bits(st.c),
+                                          st.seq_id.cpu().numpy(), st.pos.cpu().numpy(),
+                                          st.idx.numpy(), w.d_h, base=w.rope_base,
+                                          max_ctx=st.cache.max_ctx)
+    assert np.array_equal(H.bits(st.latent_plane), lat_exp)
+    got = H.bits(st.rope_plane).astype(np.int32)
+    # same sign/exponent neighbourhood: compare as ordered integers of the magnitude
+    assert np.max(np.abs(got - rope_exp.astype(np.int32))) <= 1
+    # rows never written stay zero
+    written = O.token_slot(st.seq_id.cpu().numpy(), st.pos.cpu().numpy(), max_ctx=st.cache.max_ctx)
+    mask = np.ones(got.shape[0], dtype=bool)
+    mask[written] = False
+    assert not got[mask].any()
+
+
+def test_append_bad_position_is_reported_not_written(ek):
+    w = replace(SMALL, seed=45)
+    st = H.setup(w, lens=[4, 4, 4], fill=False)
+    k_e, c = gen.tokens(w, 2, "cuda")
+    seq = torch.tensor([0, 1], dtype=torch.int32, device="cuda")
+    pos = torch.tensor([2, 10_000], dtype=torch.int32, device="cuda")
+    ek.elitekv_append(st.layer, st.cache, k_e, c, seq, pos)
+    assert ek.elitekv_check_status(st.layer) == ek.ERR_BAD_POSITION
+    assert ek.elitekv_check_status(st.layer) == 0          # cleared by the read
+    lat = H.bits(st.latent_plane)
+    assert np.array_equal(lat[2], H.bits(c)[0])
+    assert np.count_nonzero(lat.any(axis=1)) == 1
+
+
+# ------------------------------------------------------------------ query preparation
+@pytest.mark.parametrize("pair_mode", [0, 1])
+def test_absorb_query(ek, pair_mode):
+    w = replace(SMALL, B=19, seed=46)
+    idx = gen.elite_index_sets(w)
+    W_uk, W_uv = gen.up_projections(w, "cuda")
+    layer = ek.Layer(w.n_h, w.d_h, w.r, w.d_c, idx, W_uk, W_uv, 4096, pair_mode=pair_mode)
+    q = gen.queries(w, "cuda")
+    q_pos = torch.randint(0, 4096, (w.B,), dtype=torch.int32).cuda()
+    q_rope, q_abs = ek.elitekv_absorb_query(layer, q, q_pos)
+    torch.cuda.synchronize()
+    assert ek.elitekv_check_status(layer) == 0
+    for b in range(w.B):
+        r_ref, a_ref = O.absorb_query(H.f64(q[b]), int(q_pos[b]), idx.numpy(), H.f64(W_uk), w.d_h,
+                                      w.rope_base, pair_mode)
+        # bf16 output of an fp32 computation: half an ulp plus accumulation noise
+        assert np.all(np.abs(H.f64(q_rope[b]) - r_ref) <= np.abs(r_ref) * 2.0 ** -8 + 1e-6)
+        assert np.all(np.abs(H.f64(q_abs[b]) - a_ref) <= np.abs(a_ref) * 2.0 ** -8 + 1e-4)
+
+
+# ------------------------------------------------------------------ decode
+def test_decode_tiny_config_all_units(ek):
+    """Configuration 1: the whole chain from hidden states, every (sequence, head) unit."""
+    w = gen.TINY
+    st = H.setup(w, fill=False)
+    idx = st.idx
+    q_all, k_e, c = gen.projected_chain(w, idx, w.ctx)
+    st.k_e, st.c = k_e.cuda(), c.cuda()
+    st.q = q_all[-1:].contiguous().cuda()
+    ek.elitekv_append(st.layer, st.cache, st.k_e, st.c, st.seq_id, st.pos)
+    out = H.run_decode(st)
+    rel, mx = H.check_parity(st, out, H.all_units(st))
+    assert rel < 5e-3
+
+
+CASES = [
+    # name, workload, lens
+    ("ragged", replace(SMALL, seed=51), [150, 1, 77]),
+    ("tile-edges", replace(SMALL, seed=52), [64, 65, 63]),
+    ("paged", replace(SMALL, paged=True, page_size=64, seed=53), [130, 64, 1]),
+    ("paged-small-pages", replace(SMALL, paged=True, page_size=16, seed=54), [100, 17, 48]),
+    ("one-head-odd", gen.Workload("odd", n_h=1, d_h=8, r=1, d_c=8, d=8, B=2, ctx=20, seed=55), [20, 3]),
+    ("nine-heads", gen.Workload("nine", n_h=9, d_h=64, r=4, d_c=264, d=576, B=2, ctx=90, seed=56), [90, 33]),
+    ("no-rope", gen.Workload("r0", n_h=4, d_h=16, r=0, d_c=40, d=64, B=2, ctx=50, seed=57), [50, 9]),
+    ("all-rope", gen.Workload("rfull", n_h=4, d_h=16, r=8, d_c=64, d=64, B=2, ctx=50, seed=58), [50, 9]),
+    ("wide-latent", gen.Workload("wide", n_h=2, d_h=32, r=2, d_c=3072, d=64, B=1, ctx=70, seed=59), [70]),
+]
+
+
+@pytest.mark.parametrize("name,w,lens", CASES, ids=[c[0] for c in CASES])
+def test_decode_small_cases(ek, name, w, lens):
+    st = H.setup(w, lens=lens)
+    out = H.run_decode(st)
+    H.check_parity(st, out, H.all_units(st))
+
+
+def test_decode_empty_sequence_gives_zero_row(ek):
+    w = replace(SMALL, seed=60)
+    st = H.setup(w, lens=[40, 0, 5])
+    out = H.run_decode(st)
+    assert not H.bits(out[1]).any()
+    H.check_parity(st, out, [(b, h) for b in (0, 2) for h in range(w.n_h)])
+
+
+def test_decode_single_token_equals_up_projected_latent(ek):
+    w = replace(SMALL, seed=61)
+    st = H.setup(w, lens=[1, 1, 1])
+    out = H.f64(H.run_decode(st))
+    c, W_uv = H.f64(st.c), H.f64(st.W_uv)
+    for b in range(3):
+        want = (c[b] @ W_uv).reshape(w.n_h, w.d_h)
+        assert np.max(np.abs(out[b] - want)) <= 2.0 ** -8 * np.max(np.abs(want)) + 1e-3
+
+
+def test_decode_shift_invariance_on_gpu(ek):
+    w = replace(SMALL, seed=62)
+    a = H.f64(H.run_decode(H.setup(w, lens=[90, 20, 64])))
+    b = H.f64(H.run_decode(H.setup(w, lens=[90, 20, 64], pos_offset=777)))
+    rel, mx = H.errors(b, a)
+    assert rel <= H.REL_L2_TOL and mx <= H.MAX_ABS_TOL
+
+
+def test_decode_page_permutation_is_bit_identical(ek):
+    """Where pages sit physically must not matter: same logical cache, other permutation."""
+    w1 = replace(SMALL, paged=True, seed=63)
+    st1 = H.setup(w1, lens=[130, 70, 64])
+    o1 = H.bits(H.run_decode(st1))
+    # rebuild with the page table reversed, same tokens
+    st2 = H.setup(w1, lens=[130, 70, 64], fill=False)
+    num_pages = st2.cache.num_pages
+    flipped = torch.where(st2.page_table >= 0, num_pages - 1 - st2.page_table, st2.page_table)
+    st2.page_table.copy_(flipped)
+    ek.elitekv_append(st2.layer, st2.cache, st2.k_e, st2.c, st2.seq_id, st2.pos)
+    o2 = H.bits(H.run_decode(st2))
+    assert np.array_equal(o1, o2)
+
+
+def test_decode_7b_shape_small_context(ek):
+    """Layer shape of configuration 2 at a context the oracle finishes quickly: spans several
+    64-token tiles with ragged tails; all heads of every sequence."""
+    w = gen.shrink(gen.LLAMA7B_75, B=3, ctx=700)
+    st = H.setup(w, lens=[700, 333, 65])
+    out = H.run_decode(st)
+    H.check_parity(st, out, H.all_units(st))
+
+
+def test_decode_13b_shape_small_context(ek):
+    w = gen.shrink(gen.LLAMA13B_75, B=2, ctx=300)
+    st = H.setup(w, lens=[300, 129])
+    out = H.run_decode(st)
+    H.check_parity(st, out, H.all_units(st))
+
+
+@pytest.mark.parametrize("w", [gen.SWEEP_50, gen.SWEEP_875], ids=["50pct", "87.5pct"])
+def test_decode_sweep_shapes_small_context(ek, w):
+    ws = gen.shrink(w, B=2, ctx=200)
+    st = H.setup(ws, lens=[200, 70])
+    out = H.run_decode(st)
+    H.check_parity(st, out, H.all_units(st))
+
+
+# ------------------------------------------------------------------ plan
+@pytest.mark.parametrize("lens,max_items", [([1], 5), ([64, 65, 0, 1000], 9), ([4096] * 16, 164),
+                                             (list(range(1, 300, 7)), 80), ([100000, 3], 40)])
+def test_plan_partitions_every_sequence(ek, lens, max_items):
+    t = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    max_items = max(max_items, len(lens) + 1)
+    items, first = ek.elitekv_plan(t, 64, max_items)
+    torch.cuda.synchronize()
+    items, first = items.cpu().numpy(), first.cpu().numpy()
+    assert first[0] == 0 and first[-1] <= max_items
+    sizes = []
+    for b, n in enumerate(lens):
+        rows = items[first[b]:first[b + 1]]
+        at = 0
+        for s, t0, cnt, _ in rows:
+            assert s == b and t0 == at and cnt > 0 and t0 % 64 == 0
+            at += cnt
+            sizes.append(cnt)
+        assert at == n
+    assert np.all(items[first[-1]:, 0] == -1)
+    if sizes:   # near-equal pieces: no piece more than one tile above the ideal share
+        total_tiles = sum((n + 63) // 64 for n in lens)
+        budget = max_items - len(lens)
+        target = max(1, -(-total_tiles // budget))
+        assert max(sizes) <= target * 64
+
+
+# ------------------------------------------------------------------ comparator
+@pytest.mark.parametrize("n_h,d_h,lens", [(3, 64, [100, 1, 64]), (32, 128, [300, 77]), (9, 16, [50, 0])])
+def test_mha_comparator(ek, n_h, d_h, lens):
+    B, max_ctx = len(lens), max(lens) + 3
+    g = torch.Generator(device="cuda").manual_seed(7)
+    q = torch.randn(B, n_h, d_h, generator=g, device="cuda").to(torch.bfloat16)
+    K = torch.randn(B, max_ctx, n_h, d_h, generator=g, device="cuda").to(torch.bfloat16)
+    V = torch.randn(B, max_ctx, n_h, d_h, generator=g, device="cuda").to(torch.bfloat16)
+    ws = torch.empty(ek.elitekv_mha_workspace_size(B, n_h, d_h), dtype=torch.uint8, device="cuda")
+    out = ek.elitekv_mha_decode(q, K, V, torch.tensor(lens, dtype=torch.int32, device="cuda"), ws)
+    torch.cuda.synchronize()
+    for b, n in enumerate(lens):
+        want = O.mha_decode(H.f64(q[b]), H.f64(K[b, :n]), H.f64(V[b, :n]))
+        rel, mx = H.errors(H.f64(out[b]), want)
+        assert rel <= H.REL_L2_TOL and mx <= H.MAX_ABS_TOL
+
+
+# ------------------------------------------------------------------ argument checking
+def test_invalid_arguments_are_rejected_before_launch(ek):
+    w = SMALL
+    idx = gen.elite_index_sets(w)
+    W_uk, W_uv = gen.up_projections(w, "cuda")
+    bad = idx.clone()
+    bad[0, 1] = bad[0, 0]                      # duplicate chunk in one head
+    with pytest.raises(ek.ElitekvError) as e:
+        ek.Layer(w.n_h, w.d_h, w.r, w.d_c, bad, W_uk, W_uv, 64)
+    assert e.value.code == ek.ERR_INVALID_ARG
+    bad = idx.clone()
+    bad[1, 0] = w.d_h // 2                     # out of range
+    with pytest.raises(ek.ElitekvError):
+        ek.Layer(w.n_h, w.d_h, w.r, w.d_c, bad, W_uk, W_uv, 64)
+    with pytest.raises(ek.ElitekvError) as e:   # latent width not a multiple of 8
+        ek.Layer(w.n_h, w.d_h, w.r, 76, idx, W_uk, W_uv, 64)
+    assert e.value.code == ek.ERR_UNSUPPORTED_SHAPE
+    st = H.setup(w, lens=[5, 5, 5])
+    q_rope, q_abs = ek.elitekv_absorb_query(st.layer, st.q, st.q_pos)
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(ek.ElitekvError) as e:
+        ek.elitekv_decode(st.layer, st.cache, q_rope, q_abs, st.lens_dev, small)
+    assert e.value.code == ek.ERR_WORKSPACE_TOO_SMALL
+    lib = ek.lib()
+    assert lib.elitekv_decode(None, None, None, None, None, 1, None, 0, None, None) == ek.ERR_INVALID_ARG
+    assert lib.elitekv_append(None, None, None, None, None, None, 1, None) == ek.ERR_INVALID_ARG

@@ -1,0 +1,415 @@
+#!/usr/bin/env python
+"""Benchmark of EliteKV decode attention on B200.
+
+One step = one pass of the whole decode hot path for one layer over a batch of sequences:
+    elitekv_append (1 new token per sequence) -> elitekv_absorb_query -> elitekv_decode.
+Metric: decode-attention tokens/s (= sequences advanced per second for one layer), plus the
+achieved cache-read bandwidth.  Workload at one GPU: LLaMA2-7B-shaped layer, 75 % KV reduction
+(r = 8 elite chunks/head, d_c = 1536), batch 16, context 4096, contiguous cache, bf16,
+synthetic seeded inputs.  With N GPUs every rank runs its own batch (sequences are
+independent; no data-path collective) and the values add up.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
+
+`--impl reference` times the float64 CPU oracle on a bounded sample of the same workload.
+Prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2503_01586_b200 import inputs as gen  # noqa: E402
+
+METRIC = "decode_attention_tokens_per_s"
+UNIT = "tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.tmp.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.tmp.close()
+        try:
+            os.unlink(self.tmp.name)
+        except OSError:
+            pass
+        if sm:
+            out["sm_mhz"] = statistics.median(sm)
+            out["sm_max_mhz"] = max(mx)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ---------------------------------------------------------------------------------------------
+# CPU oracle leg
+# ---------------------------------------------------------------------------------------------
+def oracle_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return len(os.sched_getaffinity(0))
+
+
+def oracle_sample(w: gen.Workload, n_units: int, seed_shift: int = 0):
+    """Times the oracle, as it stands, on `n_units` (sequence, head) units of the workload at
+    full context: returns (seconds, units, description)."""
+    from oracle import elitekv_oracle as O
+    idx = gen.elite_index_sets(w).numpy().astype(np.int64)
+    W_uk, W_uv = gen.up_projections(w, "cpu")
+    W_uk, W_uv = W_uk.double().numpy(), W_uv.double().numpy()
+    lens = gen.sequence_lengths(w).tolist()
+    b = seed_shift % w.B
+    n = int(lens[b])
+    k_e, c = gen.tokens(w, n, "cpu", stream=1 + seed_shift)
+    q = gen.queries(w, "cpu")[b].double().numpy()
+    k_e, c = k_e.double().numpy(), c.double().numpy()
+    heads = list(range(min(n_units, w.n_h)))
+    t0 = time.perf_counter()
+    O.decode_from_raw(q, n - 1, k_e, np.arange(n), c, W_uk, W_uv, idx, w.d_h, base=w.rope_base,
+                      heads=heads)
+    dt = time.perf_counter() - t0
+    return dt, len(heads), f"{len(heads)} heads of sequence {b} at full context {n} (of {w.B}x{w.n_h} units)"
+
+
+def cpu_baseline(w: gen.Workload, budget_s: float = 15.0):
+    dt1, u1, _ = oracle_sample(w, 2)
+    units = int(max(2, min(w.n_h, budget_s / max(dt1 / u1, 1e-6))))
+    dt, u, what = oracle_sample(w, units)
+    # tokens/s for the whole step: B sequences need B*n_h units
+    value = (u / w.n_h) / dt
+    return {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+            "sample": what + f"; {dt:.2f} s, scaled by units"}
+
+
+def run_reference(args, w: gen.Workload):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    times = []
+    n_units = 4
+    for i in range(args.warmup + args.steps):
+        dt, u, what = oracle_sample(w, n_units, seed_shift=i)
+        if i >= args.warmup:
+            times.append(dt / u)
+    per_unit = sum(times) / len(times)
+    value = 1.0 / (per_unit * w.n_h)     # sequences (tokens) per second for one layer
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_unit * w.n_h * w.B * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": w.name, "n_h": w.n_h, "d_h": w.d_h, "r": w.r, "d_c": w.d_c,
+                   "batch": w.B, "context": w.ctx},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+                         "sample": f"each step {n_units} (sequence, head) units at full context, "
+                                   "time scaled to the whole batch"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------
+# GPU leg
+# ---------------------------------------------------------------------------------------------
+def build_workload(w: gen.Workload, ek, device):
+    """Cache prefilled with len-1 tokens per sequence; the step appends the last one."""
+    idx = gen.elite_index_sets(w)
+    W_uk, W_uv = gen.up_projections(w, device)
+    lens = gen.sequence_lengths(w)                       # tokens INCLUDING the decoded one
+    B = w.B
+    max_pos = int(lens.max()) + 1
+    layer = ek.Layer(w.n_h, w.d_h, w.r, w.d_c, idx, W_uk, W_uv, max_pos, rope_base=w.rope_base)
+    rope_w = w.n_h * 2 * w.r
+    page_table = None
+    if w.paged:
+        table, num_pages = gen.page_table(w, lens, headroom_tokens=0)
+        rows, max_ctx = num_pages * w.page_size, 0
+        page_table = table.to(device)
+    else:
+        max_ctx = int(lens.max())
+        rows = B * max_ctx
+    rope_plane = torch.zeros((rows, rope_w), dtype=torch.bfloat16, device=device)
+    latent_plane = torch.zeros((rows, w.d_c), dtype=torch.bfloat16, device=device)
+    cache = ek.make_cache(rope_plane, latent_plane, n_seqs=B, max_ctx=max_ctx,
+                          page_table=page_table, page_size=w.page_size)
+    # prefill through the library, sequence by sequence (bounded staging memory)
+    for b in range(B):
+        n = int(lens[b]) - 1
+        if n <= 0:
+            continue
+        k_e, c = gen.tokens(w, n, device, stream=10 + b)
+        seq = torch.full((n,), b, dtype=torch.int32, device=device)
+        pos = torch.arange(n, dtype=torch.int32, device=device)
+        ek.elitekv_append(layer, cache, k_e, c, seq, pos)
+    torch.cuda.synchronize()
+    # the step's inputs: one new token per sequence + the queries (host copies for the e2e leg)
+    k_new, c_new = gen.tokens(w, B, "cpu", stream=5)
+    q = gen.queries(w, "cpu")
+    host = {
+        "k_e": k_new.pin_memory(), "c": c_new.pin_memory(), "q": q.pin_memory(),
+        "seq_id": torch.arange(B, dtype=torch.int32).pin_memory(),
+        "pos": (lens - 1).to(torch.int32).pin_memory(),
+        "lens": lens.to(torch.int32).pin_memory(),
+    }
+    dev = {k: v.to(device) for k, v in host.items()}
+    ws = torch.empty(ek.elitekv_decode_workspace_size(layer, B), dtype=torch.uint8, device=device)
+    bufs = {
+        "q_rope": torch.empty((B, w.n_h, 2 * w.r), dtype=torch.bfloat16, device=device),
+        "q_abs": torch.empty((B, w.n_h, w.d_c), dtype=torch.bfloat16, device=device),
+        "out": torch.empty((B, w.n_h, w.d_h), dtype=torch.bfloat16, device=device),
+        "out_host": torch.empty((B, w.n_h, w.d_h), dtype=torch.bfloat16).pin_memory(),
+    }
+    keep = (W_uk, W_uv, rope_plane, latent_plane, page_table)
+    return layer, cache, lens, host, dev, ws, bufs, keep
+
+
+def step(ek, layer, cache, d, ws, bufs):
+    ek.elitekv_append(layer, cache, d["k_e"], d["c"], d["seq_id"], d["pos"])
+    ek.elitekv_absorb_query(layer, d["q"], d["pos"], bufs["q_rope"], bufs["q_abs"])
+    ek.elitekv_decode(layer, cache, bufs["q_rope"], bufs["q_abs"], d["lens"], ws, bufs["out"])
+
+
+KERNELS_PER_STEP = 5   # append, absorb, plan, split-K attention, combine + up-projection
+
+
+def run_gpu(args, w: gen.Workload):
+    from paper_2503_01586_b200 import binding as ek
+    ek.lib()   # fail loudly if the CUDA library is missing
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=device)
+        dist = dist_mod
+
+    w_rank = gen.replace(w, seed=w.seed + 100 * rank) if rank else w
+    layer, cache, lens, host, dev, ws, bufs, keep = build_workload(w_rank, ek, device)
+    total_tokens = int(lens.sum())
+    bytes_per_token = 2 * w.cache_elems_per_token
+    cache_bytes = total_tokens * bytes_per_token
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=device)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step(ek, layer, cache, dev, ws, bufs)
+    torch.cuda.synchronize()
+    assert ek.elitekv_check_status(layer) == 0
+
+    # ---- device-resident timing: K steps, L2 flushed before each, events around each step
+    ek.elitekv_profile_enable(layer, True)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+          for _ in range(args.steps)]
+    sampler = ClockSampler(local) if rank == 0 else None
+    barrier()
+    for a, b in ev:
+        flush.fill_(1)
+        a.record()
+        step(ek, layer, cache, dev, ws, bufs)
+        b.record()
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    total_ms = sum(step_ms)
+    kern_ms, kern_n = ek.elitekv_profile_collect(layer)
+    ek.elitekv_profile_enable(layer, False)
+
+    # ---- end to end: host buffers in, host result out, every step
+    h2d = sum(host[k].numel() * host[k].element_size() for k in host)
+    d2h = bufs["out_host"].numel() * bufs["out_host"].element_size()
+    staged = {k: torch.empty_like(v, device=device) for k, v in host.items()}
+
+    def e2e_step():
+        for k in host:
+            staged[k].copy_(host[k], non_blocking=True)
+        step(ek, layer, cache, staged, ws, bufs)
+        bufs["out_host"].copy_(bufs["out"], non_blocking=True)
+        torch.cuda.synchronize()
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        e2e_step()           # no flush here: the 268 MB+ cache does not fit the 126 MB L2
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    assert ek.elitekv_check_status(layer) == 0
+
+    # ---- comparator: uncompressed RoPE-MHA decode at the same shape (rank 0, one GPU)
+    comparator = None
+    if rank == 0 and not w.paged and not args.no_comparator:
+        try:
+            max_ctx = int(lens.max())
+            K, V = gen.mha_cache(w, w.B * max_ctx, device)
+            K = K.view(w.B, max_ctx, w.n_h, w.d_h)
+            V = V.view(w.B, max_ctx, w.n_h, w.d_h)
+            qh = dev["q"]
+            mws = torch.empty(ek.elitekv_mha_workspace_size(w.B, w.n_h, w.d_h), dtype=torch.uint8,
+                              device=device)
+            mo = torch.empty_like(qh)
+            for _ in range(3):
+                ek.elitekv_mha_decode(qh, K, V, dev["lens"], mws, mo)
+            evs = []
+            for _ in range(min(args.steps, 20)):
+                flush.fill_(1)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                ek.elitekv_mha_decode(qh, K, V, dev["lens"], mws, mo)
+                b.record()
+                evs.append((a, b))
+            torch.cuda.synchronize()
+            ms = sum(a.elapsed_time(b) for a, b in evs) / len(evs)
+            mha_bytes = total_tokens * 4 * w.n_h * w.d_h
+            comparator = {"kind": "uncompressed RoPE-MHA decode, same shape", "ms": ms,
+                          "tokens_per_s": w.B / (ms * 1e-3), "cache_bytes": mha_bytes,
+                          "gbs": mha_bytes / (ms * 1e-3) / 1e9}
+            del K, V
+        except torch.cuda.OutOfMemoryError:
+            comparator = None
+
+    # ---- reduce over ranks
+    t = torch.tensor([total_ms, e2e_s, kern_ms], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, e2e_s, kern_ms = (float(x) for x in t.tolist())
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peaks()
+    ms_per_step = total_ms / args.steps
+    value = world * w.B / (ms_per_step * 1e-3)
+    kern_avg_s = (kern_ms / max(kern_n, 1)) * 1e-3
+    achieved = cache_bytes / kern_avg_s / 1e9 if kern_n else None
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "n_h": w.n_h, "d_h": w.d_h, "r": w.r, "d_c": w.d_c,
+                   "batch_per_gpu": w.B, "context": w.ctx, "paged": w.paged,
+                   "cache_bytes_per_step": cache_bytes,
+                   "l2": "256 MiB flush write before every timed step; cache larger than L2",
+                   "parallelism": f"replicas x{world} (independent sequences, no collective)"},
+        "hbm_gbs_whole_step": cache_bytes / (ms_per_step * 1e-3) / 1e9,
+        "pct_of_nominal_8tbs_whole_step": 100.0 * cache_bytes / (ms_per_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+        "roofline": {"bound": "hbm", "kernel": "split-K decode attention", "achieved": achieved,
+                     "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                     "frac": (achieved / peak) if achieved else None,
+                     "frac_of_nominal_8tbs": (achieved / NOMINAL_HBM_GBS) if achieved else None,
+                     "kernel_us": kern_avg_s * 1e6, "launches_timed": kern_n,
+                     "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(w.name)},
+        "e2e": {"value": world * w.B * args.steps / e2e_s, "unit": UNIT,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": KERNELS_PER_STEP * args.steps,
+        "clocks": clocks,
+        "comparator": comparator,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = cpu_baseline(w)
+    else:
+        line["cpu_baseline"] = None
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one split-K launch from the ncu capture
+# summarised under profiles/ (None until a capture of the current kernel exists).
+TRAFFIC_BYTES_PER_LAUNCH = {}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=gen.LLAMA7B_75.name, choices=sorted(gen.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-comparator", action="store_true")
+    args = ap.parse_args()
+    w = gen.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_gpu(args, w)
+
+
+if __name__ == "__main__":
+    main()

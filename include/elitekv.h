@@ -157,6 +157,13 @@ int elitekv_mha_decode(const void* q_hat, const void* K_hat, const void* V,
                        int64_t max_ctx, float scale, void* workspace, size_t workspace_bytes,
                        void* out, elitekv_stream_t stream);
 
+/* Timing aid (the paper has no counterpart).  While enabled, elitekv_decode brackets its
+ * split-K attention kernel with a pair of CUDA events on the caller's stream (up to 512 calls
+ * between collections).  elitekv_profile_collect waits for the recorded events, returns the
+ * summed kernel time in milliseconds and the number of launches it covers, and starts over. */
+int elitekv_profile_enable(elitekv_layer* layer, int32_t on);
+int elitekv_profile_collect(elitekv_layer* layer, float* total_ms, int32_t* launches);
+
 const char* elitekv_strerror(int status);
 
 #ifdef __cplusplus

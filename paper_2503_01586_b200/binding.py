@@ -66,11 +66,14 @@ def lib() -> C.CDLL:
         L.elitekv_check_status.argtypes = [vp, vp]
         L.elitekv_mha_workspace_size.argtypes = [i32, i32, i32, C.POINTER(sz)]
         L.elitekv_mha_decode.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, C.c_float, vp, sz, vp, vp]
+        L.elitekv_profile_enable.argtypes = [vp, i32]
+        L.elitekv_profile_collect.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(i32)]
         L.elitekv_strerror.argtypes = [C.c_int]
         L.elitekv_strerror.restype = C.c_char_p
         for name in ("elitekv_layer_create", "elitekv_layer_destroy", "elitekv_append",
                      "elitekv_absorb_query", "elitekv_decode_workspace_size", "elitekv_decode",
                      "elitekv_plan", "elitekv_check_status", "elitekv_mha_workspace_size",
+                     "elitekv_profile_enable", "elitekv_profile_collect",
                      "elitekv_mha_decode"):
             getattr(L, name).restype = C.c_int
         _lib = L
@@ -203,6 +206,18 @@ def elitekv_plan(seq_lens, tile_tokens: int, max_items: int):
 
 def elitekv_check_status(layer: Layer) -> int:
     return lib().elitekv_check_status(layer.handle, _stream())
+
+
+def elitekv_profile_enable(layer: Layer, on: bool) -> None:
+    _check(lib().elitekv_profile_enable(layer.handle, 1 if on else 0), "elitekv_profile_enable")
+
+
+def elitekv_profile_collect(layer: Layer):
+    """(summed split-K kernel milliseconds, launches) since the last collection."""
+    ms, n = C.c_float(), C.c_int32()
+    _check(lib().elitekv_profile_collect(layer.handle, C.byref(ms), C.byref(n)),
+           "elitekv_profile_collect")
+    return ms.value, n.value
 
 
 def elitekv_mha_workspace_size(B: int, n_h: int, d_h: int) -> int:

@@ -88,7 +88,13 @@ extern "C" int elitekv_decode(const elitekv_layer* L, const elitekv_cache* cache
   cudaStream_t st = (cudaStream_t)stream;
   rc = ekv_launch_plan(seq_lens, B, ELITEKV_TILE_TOKENS, max_items, ws.items, ws.seq_first, st);
   if (rc != ELITEKV_OK) return rc;
+  EkvProfile* prof = (L->prof && L->prof->enabled && L->prof->count < kProfileSlots) ? L->prof : nullptr;
+  if (prof) EKV_CUDA_OK(cudaEventRecord(prof->ev[2 * prof->count], st));
   rc = ekv_launch_decode_generic(L, cache, cv, q_rope, q_abs, B, ws, st);
   if (rc != ELITEKV_OK) return rc;
+  if (prof) {
+    EKV_CUDA_OK(cudaEventRecord(prof->ev[2 * prof->count + 1], st));
+    prof->count++;
+  }
   return ekv_launch_combine(L, B, ws, out, st);
 }

@@ -33,6 +33,14 @@ struct elitekv_layer {
   bf16* d_WukT;                    // [n_h][dn][d_c]: W_uk regrouped per head, d_c contiguous
   bf16* d_Wuv;                     // [d_c][n_h*d_h] private copy
   int32_t* d_status;               // [4] device status word: code, detail0, detail1, count
+  struct EkvProfile* prof;         // optional event pairs around the split-K kernel
+};
+
+constexpr int kProfileSlots = 512;
+struct EkvProfile {
+  int enabled;
+  int count;
+  cudaEvent_t ev[2 * kProfileSlots];
 };
 
 #define EKV_CUDA_OK(expr)                                   \

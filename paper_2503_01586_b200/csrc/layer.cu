@@ -127,6 +127,11 @@ extern "C" int elitekv_layer_destroy(elitekv_layer* L) {
   cudaFree(L->d_cs_owned);
   cudaFree(L->d_WukT);
   cudaFree(L->d_Wuv);
+  if (L->prof) {
+    for (int i = 0; i < 2 * kProfileSlots; ++i)
+      if (L->prof->ev[i]) cudaEventDestroy(L->prof->ev[i]);
+    free(L->prof);
+  }
   free(L);
   return ELITEKV_OK;
 }
@@ -153,6 +158,43 @@ extern "C" const char* elitekv_strerror(int status) {
     case ELITEKV_ERR_BAD_POSITION: return "position or sequence outside the cache";
     default: return "unknown status";
   }
+}
+
+extern "C" int elitekv_profile_enable(elitekv_layer* L, int32_t on) {
+  if (!L) return ELITEKV_ERR_INVALID_ARG;
+  if (on && !L->prof) {
+    EkvProfile* p = (EkvProfile*)calloc(1, sizeof(EkvProfile));
+    if (!p) return ELITEKV_ERR_CUDA;
+    for (int i = 0; i < 2 * kProfileSlots; ++i)
+      if (cudaEventCreate(&p->ev[i]) != cudaSuccess) {
+        for (int j = 0; j < i; ++j) cudaEventDestroy(p->ev[j]);
+        free(p);
+        return ELITEKV_ERR_CUDA;
+      }
+    L->prof = p;
+  }
+  if (L->prof) {
+    L->prof->enabled = on ? 1 : 0;
+    L->prof->count = 0;
+  }
+  return ELITEKV_OK;
+}
+
+extern "C" int elitekv_profile_collect(elitekv_layer* L, float* total_ms, int32_t* launches) {
+  if (!L || !total_ms || !launches) return ELITEKV_ERR_INVALID_ARG;
+  *total_ms = 0.f;
+  *launches = 0;
+  if (!L->prof) return ELITEKV_OK;
+  EkvProfile* p = L->prof;
+  for (int i = 0; i < p->count; ++i) {
+    float ms = 0.f;
+    EKV_CUDA_OK(cudaEventSynchronize(p->ev[2 * i + 1]));
+    EKV_CUDA_OK(cudaEventElapsedTime(&ms, p->ev[2 * i], p->ev[2 * i + 1]));
+    *total_ms += ms;
+  }
+  *launches = p->count;
+  p->count = 0;
+  return ELITEKV_OK;
 }
 
 int ekv_make_view(const elitekv_cache* c, CacheView* v) {

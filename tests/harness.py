@@ -63,22 +63,25 @@ def setup(w: gen.Workload, *, lens: Optional[Sequence[int]] = None, decode_kerne
     seq_id = torch.repeat_interleave(torch.arange(B, dtype=torch.int32), lens_t.to(torch.int64))
     pos = torch.cat([torch.arange(int(n), dtype=torch.int32) for n in lens_t.tolist()]) if N else \
         torch.zeros(0, dtype=torch.int32)
-    pos = pos + pos_offset
     q = gen.queries(w, device)
-    q_pos = (lens_t - 1).clamp(min=0) + pos_offset
-    max_pos = int(lens_t.max().item()) + pos_offset + 2 if B else 2
+    q_pos = (lens_t - 1).clamp(min=0)
+    max_pos = int(lens_t.max().item()) + 2 if B else 2
+    if pos_offset:
+        # RoPE positions shifted by a constant while cache slots stay put: hand the layer a
+        # (cos, sin) table that starts at pos_offset
+        tab = O.rope_table_f32(max_pos + pos_offset, w.d_h, w.rope_base)[pos_offset:]
+        cos_sin = torch.from_numpy(np.ascontiguousarray(tab)).to(device)
     layer = ek.Layer(w.n_h, w.d_h, w.r, w.d_c, idx, W_uk, W_uv, max_pos, rope_base=w.rope_base,
                      cos_sin=cos_sin, decode_kernel=decode_kernel)
     rope_w = w.n_h * 2 * w.r
     if w.paged:
-        # positions are shifted by pos_offset inside the cache too, so pages cover them
-        table, num_pages = gen.page_table(w, lens_t + pos_offset, headroom_tokens=1)
+        table, num_pages = gen.page_table(w, lens_t, headroom_tokens=1)
         rows = num_pages * w.page_size
         page_table = table.to(device)
         max_ctx = 0
     else:
         page_table = None
-        max_ctx = int(lens_t.max().item()) + pos_offset + 1
+        max_ctx = int(lens_t.max().item()) + 1
         rows = B * max_ctx
     rope_plane = (torch.zeros((rows, rope_w), dtype=torch.bfloat16, device=device) if rope_w > 0
                   else torch.zeros((8,), dtype=torch.bfloat16, device=device))   # r = 0: never read

@@ -138,7 +138,7 @@ CASES = [
     ("nine-heads", gen.Workload("nine", n_h=9, d_h=64, r=4, d_c=264, d=576, B=2, ctx=90, seed=56), [90, 33]),
     ("no-rope", gen.Workload("r0", n_h=4, d_h=16, r=0, d_c=40, d=64, B=2, ctx=50, seed=57), [50, 9]),
     ("all-rope", gen.Workload("rfull", n_h=4, d_h=16, r=8, d_c=64, d=64, B=2, ctx=50, seed=58), [50, 9]),
-    ("wide-latent", gen.Workload("wide", n_h=2, d_h=32, r=2, d_c=3072, d=64, B=1, ctx=70, seed=59), [70]),
+    ("wide-latent", gen.Workload("wide", n_h=2, d_h=32, r=2, d_c=3072, d=3072, B=1, ctx=70, seed=59), [70]),
 ]
 
 

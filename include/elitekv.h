@@ -49,7 +49,9 @@ typedef enum {
   ELITEKV_ERR_CUDA = -4,
   ELITEKV_ERR_TIMEOUT = -5,       /* a bounded device-side wait ran out            */
   ELITEKV_ERR_BAD_PAGE = -6,      /* page id outside [0, num_pages)                */
-  ELITEKV_ERR_BAD_POSITION = -7   /* position outside [0, max_pos) or the cache    */
+  ELITEKV_ERR_BAD_POSITION = -7,  /* position outside [0, max_pos) or the cache    */
+  ELITEKV_ERR_STATIC_SCRATCH_EXCEEDED = -8  /* elitekv_decode_static: batch/shape needs more
+                                               scratch than ELITEKV_STATIC_SCRATCH_BYTES     */
 } elitekv_status;
 
 /* Layer description (Sections 3.1 and 3.2).  Host struct; elite_idx is a HOST pointer, the
@@ -133,6 +135,27 @@ int elitekv_decode_workspace_size(const elitekv_layer* layer, int32_t B, size_t*
 int elitekv_decode(const elitekv_layer* layer, const elitekv_cache* cache, const void* q_rope,
                    const void* q_abs, const int32_t* seq_lens, int32_t B, void* workspace,
                    size_t workspace_bytes, void* out, elitekv_stream_t stream);
+
+/* Decode attention without any allocation (the paper has no counterpart; this is a packaging
+ * variant of elitekv_decode).  For callers that must not, or cannot, call cudaMalloc: engines
+ * that give all device memory to one arena up front, plugins running inside another
+ * framework's step, latency-critical loops.  Same arguments and result as elitekv_decode, minus
+ * the workspace: the scratch lives in a device array of ELITEKV_STATIC_SCRATCH_BYTES inside the
+ * library, which every GPU that loads the library holds until the process exits.
+ *   - Returns ELITEKV_ERR_STATIC_SCRATCH_EXCEEDED, launching nothing, when
+ *     elitekv_decode_workspace_size(layer, B) exceeds ELITEKV_STATIC_SCRATCH_BYTES
+ *     (a 7B-shaped layer at 75 % reduction with B = 16 needs about 31 MiB).
+ *   - Calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - The first call on a device looks up the array's device address
+ *     (cudaGetSymbolAddress, with the layer's device current); make that first call before
+ *     any stream capture begins.  The layer's device must be the current device.
+ *   - All calls share the one array, which keeps the previous call's contents (nothing in it
+ *     needs clearing between calls).  Two calls whose kernels can overlap on the GPU -- other
+ *     streams, other host threads, other layers -- race on it: order them on one stream. */
+#define ELITEKV_STATIC_SCRATCH_BYTES (48u << 20)
+int elitekv_decode_static(const elitekv_layer* layer, const elitekv_cache* cache,
+                          const void* q_rope, const void* q_abs, const int32_t* seq_lens,
+                          int32_t B, void* out, elitekv_stream_t stream);
 
 /* Work plan of the split-K kernel, exported for inspection (the paper has no counterpart: it
  * is this library's load balancer for ragged batches).  Cuts the batch's token tiles into at

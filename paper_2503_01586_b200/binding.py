@@ -23,6 +23,8 @@ ERR_CUDA = -4
 ERR_TIMEOUT = -5
 ERR_BAD_PAGE = -6
 ERR_BAD_POSITION = -7
+ERR_STATIC_SCRATCH_EXCEEDED = -8
+STATIC_SCRATCH_BYTES = 48 << 20
 
 
 class ElitekvError(RuntimeError):
@@ -62,6 +64,7 @@ def lib() -> C.CDLL:
         L.elitekv_absorb_query.argtypes = [vp, vp, vp, i32, vp, vp, vp]
         L.elitekv_decode_workspace_size.argtypes = [vp, i32, C.POINTER(sz)]
         L.elitekv_decode.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, i32, vp, sz, vp, vp]
+        L.elitekv_decode_static.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, i32, vp, vp]
         L.elitekv_plan.argtypes = [vp, i32, i32, i32, vp, vp, vp]
         L.elitekv_check_status.argtypes = [vp, vp]
         L.elitekv_mha_workspace_size.argtypes = [i32, i32, i32, C.POINTER(sz)]
@@ -73,7 +76,7 @@ def lib() -> C.CDLL:
         for name in ("elitekv_layer_create", "elitekv_layer_destroy", "elitekv_append",
                      "elitekv_absorb_query", "elitekv_decode_workspace_size", "elitekv_decode",
                      "elitekv_plan", "elitekv_check_status", "elitekv_mha_workspace_size",
-                     "elitekv_profile_enable", "elitekv_profile_collect",
+                     "elitekv_profile_enable", "elitekv_profile_collect", "elitekv_decode_static",
                      "elitekv_mha_decode"):
             getattr(L, name).restype = C.c_int
         _lib = L
@@ -192,6 +195,18 @@ def elitekv_decode(layer: Layer, cache: CacheDesc, q_rope, q_abs, seq_lens, work
                                 _ptr(_dev(seq_lens, torch.int32)), B, workspace.data_ptr(),
                                 workspace.numel() * workspace.element_size(), _ptr(out), _stream()),
            "elitekv_decode")
+    return out
+
+
+def elitekv_decode_static(layer: Layer, cache: CacheDesc, q_rope, q_abs, seq_lens, out):
+    """elitekv_decode with the library's built-in scratch: no workspace argument and no
+    allocation, so `out` must be passed in (this wrapper allocates nothing either)."""
+    B = q_abs.shape[0]
+    _check(lib().elitekv_decode_static(layer.handle, C.byref(cache), _ptr(q_rope),
+                                       _ptr(_dev(q_abs, torch.bfloat16)),
+                                       _ptr(_dev(seq_lens, torch.int32)), B,
+                                       _ptr(_dev(out, torch.bfloat16)), _stream()),
+           "elitekv_decode_static")
     return out
 
 

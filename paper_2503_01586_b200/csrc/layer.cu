@@ -156,6 +156,8 @@ extern "C" const char* elitekv_strerror(int status) {
     case ELITEKV_ERR_TIMEOUT: return "a bounded device-side wait ran out";
     case ELITEKV_ERR_BAD_PAGE: return "page id outside the pool";
     case ELITEKV_ERR_BAD_POSITION: return "position or sequence outside the cache";
+    case ELITEKV_ERR_STATIC_SCRATCH_EXCEEDED:
+      return "scratch need exceeds the built-in array of elitekv_decode_static";
     default: return "unknown status";
   }
 }

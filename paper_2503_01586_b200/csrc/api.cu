@@ -5,15 +5,29 @@ namespace {
 
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
-// Which split-K kernel a layer uses: 1 = generic CUDA-core kernel.
-int select_kernel(const elitekv_layer* L) {
-  if (L->decode_kernel == 2) return -1;          // tensor-core kernel: not built for this shape
+// Which split-K kernel serves a layer (and cache): 1 = generic CUDA-core kernel, 2 = tcgen05
+// tensor-core kernel, -1 = none.  `cache` may be null (shape-only question).
+int select_kernel(const elitekv_layer* L, const elitekv_cache* cache) {
+  const bool tc = ekv_tc_supported(L, cache) != 0;
+  if (L->decode_kernel == 2) return tc ? 2 : -1;
+  if (L->decode_kernel == 1) return ekv_generic_supported(L) ? 1 : -1;
+  if (tc) return 2;
   return ekv_generic_supported(L) ? 1 : -1;
 }
 
 int max_items_for(const elitekv_layer* L, int B, int kernel) {
-  (void)kernel;
-  return ekv_generic_max_items(L, B);
+  return kernel == 2 ? ekv_tc_max_items(L, B) : ekv_generic_max_items(L, B);
+}
+
+// The workspace is sized for whichever kernel may be picked once the cache layout is known.
+int max_items_any(const elitekv_layer* L, int B) {
+  int m = 0;
+  if (ekv_generic_supported(L) && L->decode_kernel != 2) m = ekv_generic_max_items(L, B);
+  if (ekv_tc_supported(L, nullptr) && L->decode_kernel != 1) {
+    const int t = ekv_tc_max_items(L, B);
+    if (t > m) m = t;
+  }
+  return m;
 }
 
 struct Carve {
@@ -56,9 +70,9 @@ extern "C" int elitekv_absorb_query(const elitekv_layer* L, const void* q, const
 
 extern "C" int elitekv_decode_workspace_size(const elitekv_layer* L, int32_t B, size_t* bytes) {
   if (!L || !bytes || B <= 0) return ELITEKV_ERR_INVALID_ARG;
-  const int kernel = select_kernel(L);
-  if (kernel < 0) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
-  *bytes = carve(L, B, max_items_for(L, B, kernel)).total;
+  const int items = max_items_any(L, B);
+  if (items <= 0) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
+  *bytes = carve(L, B, items).total;
   return ELITEKV_OK;
 }
 
@@ -70,7 +84,7 @@ extern "C" int elitekv_decode(const elitekv_layer* L, const elitekv_cache* cache
     return ELITEKV_ERR_INVALID_ARG;
   if (((uintptr_t)q_abs & 15) || ((uintptr_t)out & 3)) return ELITEKV_ERR_INVALID_ARG;
   if (B > cache->n_seqs) return ELITEKV_ERR_INVALID_ARG;
-  const int kernel = select_kernel(L);
+  const int kernel = select_kernel(L, cache);
   if (kernel < 0) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
   CacheView cv;
   int rc = ekv_make_view(cache, &cv);
@@ -86,11 +100,13 @@ extern "C" int elitekv_decode(const elitekv_layer* L, const elitekv_cache* cache
   ws.part_ml = (float*)(base + cw.off_ml);
   ws.part_acc = (float*)(base + cw.off_acc);
   cudaStream_t st = (cudaStream_t)stream;
-  rc = ekv_launch_plan(seq_lens, B, ELITEKV_TILE_TOKENS, max_items, ws.items, ws.seq_first, st);
+  rc = ekv_launch_plan(seq_lens, B, kernel == 2 ? 128 : ELITEKV_TILE_TOKENS, max_items, ws.items,
+                       ws.seq_first, st);
   if (rc != ELITEKV_OK) return rc;
   EkvProfile* prof = (L->prof && L->prof->enabled && L->prof->count < kProfileSlots) ? L->prof : nullptr;
   if (prof) EKV_CUDA_OK(cudaEventRecord(prof->ev[2 * prof->count], st));
-  rc = ekv_launch_decode_generic(L, cache, cv, q_rope, q_abs, B, ws, st);
+  rc = kernel == 2 ? ekv_launch_decode_tc(L, cache, cv, q_rope, q_abs, B, ws, st)
+                   : ekv_launch_decode_generic(L, cache, cv, q_rope, q_abs, B, ws, st);
   if (rc != ELITEKV_OK) return rc;
   if (prof) {
     EKV_CUDA_OK(cudaEventRecord(prof->ev[2 * prof->count + 1], st));

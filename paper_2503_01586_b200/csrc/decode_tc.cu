@@ -1,0 +1,633 @@
+// Tensor-core split-K decode kernel for sm_100a (tcgen05 + TMEM + TMA).
+//
+// All heads of a layer read the SAME latent row (J-LRD, Section 3.2), so for one sequence the
+// two latent contractions are dense GEMMs against a tile of T = 128 cached tokens:
+//     S   [T x n_h]    = C[T x d_c] . Q_abs^T[d_c x n_h]          (score equation of Section
+//                                                                   3.1 with B^k absorbed)
+//     acc [d_c x n_h] += C^T[d_c x T] . P[T x n_h]                 (sum_t p_t c_t, Section 2.1;
+//                                                                   B^v applied later)
+// Both run as tcgen05.mma (M = 128, N = n_h, K = 16, bf16 in, fp32 accumulate in TMEM) straight
+// from the 128-byte-swizzled shared-memory tiles that TMA writes; the narrow per-head rope dot
+// product stays on FP32 FMA in the softmax threads.
+//
+// The absorbed queries of a sequence (n_h x d_c bf16, 96 KB at d_c = 1536) must stay resident
+// beside the token tile, which leaves no room to keep a whole 128 x d_c tile in shared memory.
+// The tile is therefore streamed twice through a small ring of [128 tokens x 64 coords] chunks:
+// pass A accumulates S over the latent axis, the softmax threads turn S (+ rope part) into P,
+// pass B streams the same chunks again (they were just read, so they come from L2, not HBM)
+// and accumulates P-weighted latents into the TMEM-resident output.  HBM sees every cache byte
+// once per step.
+//
+// One thread block (192 threads) per plan item:
+//   warp 0    TMA producer (one lane): absorbed queries once, then per tile the latent chunks
+//             of pass A interleaved with the rope boxes, then the latent chunks of pass B
+//   warp 1    TMEM allocation; one lane issues every tcgen05.mma and the commits that free
+//             ring slots; the warp zero-fills token rows past the end of the sequence
+//   warps 2-5 one thread per token row: rope dot products, S from TMEM, masking, running
+//             max / sum in base 2 with a lazily moved reference max, P to shared memory in the
+//             layout the second GEMM wants, TMEM rescale when the reference moves, epilogue
+// Every wait is bounded: when a limit is hit the block records ELITEKV_ERR_TIMEOUT in the
+// layer's status word, stops issuing work, frees its TMEM and leaves.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace {
+
+constexpr int kTile = 128;            // tokens per tile
+constexpr int kChunkBytes = 16384;    // [128 tokens][64 bf16] with 128-byte rows
+constexpr int kLatSlots = 4;
+constexpr int kRopeSlots = 3;
+constexpr int kThreads = 192;
+constexpr int kSoftmaxThreads = 128;
+constexpr unsigned kWaitLimit = 1u << 20;   // polls of mbarrier.try_wait before giving up
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait; returns false (and raises the block's abort flag) when the limit is hit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (unsigned i = 0; i < kWaitLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 1023) == 1023 && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"((uint64_t)map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
+  uint32_t* r = (uint32_t*)v;
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const float* v) {
+  const uint32_t* r = (const uint32_t*)v;
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
+      ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]),
+        "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void named_bar_sync(int id, int n) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory");
+}
+
+// Shared-memory matrix descriptor of tcgen05.mma: start address, leading / stride byte offsets
+// (each >> 4), descriptor version 1, swizzle mode in the top bits (2 = 128-byte, 0 = none).
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)layout << 61;
+  return d;
+}
+// Instruction descriptor for kind::f16 with bf16 inputs and fp32 accumulation.
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N, int a_mn_major, int b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
+         ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// order-preserving float <-> int map so that redux.sync.max.s32 gives a float max
+__device__ __forceinline__ int f2ord(float f) {
+  int i = __float_as_int(f);
+  return i ^ ((i >> 31) & 0x7fffffff);
+}
+__device__ __forceinline__ float ord2f(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
+
+struct TcArgs {
+  const int32_t* items;
+  const int32_t* page_table;
+  float* part_acc;
+  float* part_ml;
+  const bf16* q_rope;       // [B][n_h][2r]
+  int32_t* status;
+  long long max_ctx;
+  long long num_pages;
+  int page_shift, page_mask, max_pages_per_seq;
+  int n_h, d_c;
+  float scale_log2e;
+};
+
+struct __align__(8) TcBarriers {
+  uint64_t lat_full[kLatSlots], lat_empty[kLatSlots];
+  uint64_t rope_full[kRopeSlots], rope_empty[kRopeSlots];
+  uint64_t q_full, s_full, p_ready, pv_done;
+};
+
+// shared-memory carve-up (offsets from a 1024-byte aligned base)
+template <int N>
+struct Smem {
+  __host__ __device__ static constexpr int q_bytes(int d_c) { return (d_c / 64) * N * 128; }
+  __host__ __device__ static constexpr int lat_off(int d_c) { return q_bytes(d_c); }
+  __host__ __device__ static constexpr int rope_off(int d_c) { return lat_off(d_c) + kLatSlots * kChunkBytes; }
+  __host__ __device__ static constexpr int p_off(int d_c) { return rope_off(d_c) + kRopeSlots * kChunkBytes; }
+  static constexpr int p_bytes = kTile * N * 2;
+  __host__ __device__ static constexpr int misc_off(int d_c) { return p_off(d_c) + p_bytes; }
+  // misc: q_rope fp32 [N][R2max=32] 4 KB | wmax [4][N] | corr [N] | barriers | tmem base | abort
+  static constexpr int misc_bytes = N * 32 * 4 + 4 * N * 4 + N * 4 + (int)sizeof(TcBarriers) + 64;
+  __host__ __device__ static constexpr int total(int d_c) { return misc_off(d_c) + misc_bytes + 1024; }
+};
+
+template <int N, int R2>
+__global__ void __launch_bounds__(kThreads, 1)
+decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_constant__ CUtensorMap map_rope,
+                 const __grid_constant__ CUtensorMap map_q, const TcArgs a) {
+  extern __shared__ unsigned char smem_raw[];
+  const int item = blockIdx.x;
+  const int seq = a.items[4 * item + 0];
+  if (seq < 0) return;
+  const int tok0 = a.items[4 * item + 1];
+  const int ntok = a.items[4 * item + 2];
+  const int n_tiles = (ntok + kTile - 1) / kTile;
+  const int d_c = a.d_c;
+  const int NKC = d_c >> 6;      // 64-wide latent chunks
+  const int NB = d_c >> 7;       // 128-row output blocks
+  constexpr int NRB = N * R2 / 64;   // rope boxes per tile
+  constexpr int HPB = 64 / R2;       // heads per rope box
+
+  unsigned char* base = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  unsigned char* s_q = base;
+  unsigned char* s_lat = base + Smem<N>::lat_off(d_c);
+  unsigned char* s_rope = base + Smem<N>::rope_off(d_c);
+  unsigned char* s_p = base + Smem<N>::p_off(d_c);
+  unsigned char* s_misc = base + Smem<N>::misc_off(d_c);
+  float* s_qrope = (float*)s_misc;                         // [N][R2]
+  float* s_wmax = (float*)(s_misc + N * 32 * 4);           // [4][N]
+  float* s_corr = s_wmax + 4 * N;                          // [N]
+  TcBarriers* bars = (TcBarriers*)(s_corr + N);
+  uint32_t* s_tmem = (uint32_t*)(bars + 1);
+  volatile int* s_abort = (volatile int*)(s_tmem + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kLatSlots; ++i) {
+      mbar_init(smem_u32(&bars->lat_full[i]), 1);
+      mbar_init(smem_u32(&bars->lat_empty[i]), 1);
+    }
+    for (int i = 0; i < kRopeSlots; ++i) {
+      mbar_init(smem_u32(&bars->rope_full[i]), 1);
+      mbar_init(smem_u32(&bars->rope_empty[i]), kSoftmaxThreads / 32);
+    }
+    mbar_init(smem_u32(&bars->q_full), 1);
+    mbar_init(smem_u32(&bars->s_full), 1);
+    mbar_init(smem_u32(&bars->p_ready), kSoftmaxThreads);
+    mbar_init(smem_u32(&bars->pv_done), 1);
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+  }
+  // rotated query chunks of this sequence as fp32 (broadcast operand of the rope dot products)
+  for (int e = threadIdx.x; e < N * R2; e += kThreads) {
+    const int h = e / R2;
+    s_qrope[e] = h < a.n_h ? __bfloat162float(a.q_rope[((size_t)seq * a.n_h + h) * R2 + (e % R2)]) : 0.f;
+  }
+  const int tmem_cols_needed = NB * N + N;
+  uint32_t tmem_cols = 32;
+  while ((int)tmem_cols < tmem_cols_needed) tmem_cols <<= 1;
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+  const uint32_t tmem_s = tmem_base + NB * N;     // S columns after the NB output blocks
+
+  // ============================================================== warp 0: TMA producer
+  if (warp == 0) {
+    if (lane == 0) {
+      const uint32_t qbar = smem_u32(&bars->q_full);
+      mbar_expect_tx(qbar, (uint32_t)(NKC * N * 128));
+      for (int kc = 0; kc < NKC; ++kc)
+        tma_load_2d(smem_u32(s_q + kc * N * 128), &map_q, kc * 64, seq * a.n_h, qbar);
+
+      unsigned lat_n = 0, rope_n = 0;      // chunks issued so far
+      bool ok = true;
+      for (int tile = 0; tile < n_tiles && ok; ++tile) {
+        const int t_abs = tok0 + tile * kTile;
+        const int nvalid = min(kTile, ntok - tile * kTile);
+        const int halves = nvalid > 64 ? 2 : 1;
+        long long row[2];
+        for (int hf = 0; hf < 2; ++hf) {
+          const int t = t_abs + 64 * hf;
+          if (a.page_table == nullptr) {
+            row[hf] = (long long)seq * a.max_ctx + t;
+          } else {
+            const int pi = t >> a.page_shift;
+            int page = (hf < halves && pi < a.max_pages_per_seq)
+                           ? a.page_table[(long long)seq * a.max_pages_per_seq + pi] : 0;
+            if (page < 0 || page >= a.num_pages) {
+              if (hf < halves) ekv_record(a.status, ELITEKV_ERR_BAD_PAGE, seq, page);
+              page = 0;
+            }
+            row[hf] = ((long long)page << a.page_shift) + (t & a.page_mask);
+          }
+        }
+        auto load_lat = [&](int kc) -> bool {
+          const unsigned slot = lat_n % kLatSlots;
+          if (!mbar_wait(smem_u32(&bars->lat_empty[slot]), ((lat_n / kLatSlots) & 1) ^ 1, s_abort)) return false;
+          const uint32_t fb = smem_u32(&bars->lat_full[slot]);
+          mbar_expect_tx(fb, (uint32_t)(halves * 8192));
+          for (int hf = 0; hf < halves; ++hf)
+            tma_load_2d(smem_u32(s_lat + slot * kChunkBytes + hf * 8192), &map_lat, kc * 64, (int)row[hf], fb);
+          ++lat_n;
+          return true;
+        };
+        auto load_rope = [&](int cb) -> bool {
+          const unsigned slot = rope_n % kRopeSlots;
+          if (!mbar_wait(smem_u32(&bars->rope_empty[slot]), ((rope_n / kRopeSlots) & 1) ^ 1, s_abort)) return false;
+          const uint32_t fb = smem_u32(&bars->rope_full[slot]);
+          mbar_expect_tx(fb, (uint32_t)(halves * 8192));
+          for (int hf = 0; hf < halves; ++hf)
+            tma_load_2d(smem_u32(s_rope + slot * kChunkBytes + hf * 8192), &map_rope, cb * 64, (int)row[hf], fb);
+          ++rope_n;
+          return true;
+        };
+        // pass A: latent chunks with the rope boxes spread between them
+        int cb = 0;
+        for (int kc = 0; kc < NKC && ok; ++kc) {
+          if (cb < NRB && (long long)kc * NRB >= (long long)cb * NKC) ok = load_rope(cb++);
+          if (ok) ok = load_lat(kc);
+        }
+        while (cb < NRB && ok) ok = load_rope(cb++);
+        // pass B: the same latent chunks again (served by L2)
+        for (int kc = 0; kc < NKC && ok; ++kc) ok = load_lat(kc);
+      }
+    }
+  }
+  // ============================================================== warp 1: MMA issuer
+  else if (warp == 1) {
+    constexpr uint32_t idesc_s = make_idesc(128, N, 0, 0);    // S = C . Q^T   (both K-major)
+    constexpr uint32_t idesc_pv = make_idesc(128, N, 1, 1);   // acc = C^T . P (both MN-major)
+    bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->q_full), 0, s_abort));
+    unsigned lat_n = 0;
+    for (int tile = 0; tile < n_tiles && ok; ++tile) {
+      const int nvalid = min(kTile, ntok - tile * kTile);
+      // ---- pass A
+      for (int kc = 0; kc < NKC && ok; ++kc) {
+        const unsigned slot = lat_n % kLatSlots;
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->lat_full[slot]), (lat_n / kLatSlots) & 1, s_abort));
+        if (!ok) break;
+        tc_fence_after();
+        if (lane == 0) {
+          const uint32_t a_addr = smem_u32(s_lat + slot * kChunkBytes);
+          const uint32_t b_addr = smem_u32(s_q + kc * N * 128);
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            tc_mma(tmem_s, make_desc(a_addr + k * 32, 16, 1024, 2), make_desc(b_addr + k * 32, 16, 1024, 2),
+                   idesc_s, (kc | k) != 0);
+          tc_commit(smem_u32(&bars->lat_empty[slot]));
+        }
+        __syncwarp();
+        ++lat_n;
+      }
+      if (!ok) break;
+      if (lane == 0) tc_commit(smem_u32(&bars->s_full));
+      __syncwarp();
+      // ---- wait for P (and the rescaled output) of this tile
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_ready), tile & 1, s_abort));
+      if (!ok) break;
+      tc_fence_after();
+      // ---- pass B
+      const int ksteps = (nvalid + 15) >> 4;
+      const int zero_from = nvalid, zero_to = ksteps * 16;
+      for (int blk = 0; blk < NB && ok; ++blk) {
+        const unsigned s0 = lat_n % kLatSlots, s1 = (lat_n + 1) % kLatSlots;
+        ok = mbar_wait(smem_u32(&bars->lat_full[s0]), (lat_n / kLatSlots) & 1, s_abort) &&
+             mbar_wait(smem_u32(&bars->lat_full[s1]), ((lat_n + 1) / kLatSlots) & 1, s_abort);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        if (zero_to > zero_from) {
+          // token rows past the end of the sequence inside the last 16-token step: make them
+          // exact zeros so that 0-probability rows cannot inject NaN/Inf bit patterns
+          for (int e = lane; e < (zero_to - zero_from) * 16; e += 32) {
+            const int rrow = zero_from + (e >> 4), c16 = e & 15;
+            unsigned char* p = s_lat + (c16 < 8 ? s0 : s1) * kChunkBytes + rrow * 128 + (c16 & 7) * 16;
+            *(uint4*)p = make_uint4(0, 0, 0, 0);
+          }
+          fence_proxy_async();
+          __syncwarp();
+        }
+        tc_fence_after();
+        if (lane == 0) {
+          const uint32_t a_addr = smem_u32(s_lat + s0 * kChunkBytes);
+          const uint32_t b_addr = smem_u32(s_p);
+          for (int k = 0; k < ksteps; ++k)
+            tc_mma(tmem_base + blk * N, make_desc(a_addr + k * 2048, kChunkBytes, 1024, 2),
+                   make_desc(b_addr + k * 256, 128, 2048, 0), idesc_pv, (tile | k) != 0);
+          tc_commit(smem_u32(&bars->lat_empty[s0]));
+          tc_commit(smem_u32(&bars->lat_empty[s1]));
+        }
+        __syncwarp();
+        lat_n += 2;
+      }
+      if (!ok) break;
+      if (lane == 0) tc_commit(smem_u32(&bars->pv_done));
+      __syncwarp();
+    }
+  }
+  // ============================================================== warps 2-5: softmax
+  else {
+    const int quarter = warp & 3;                 // TMEM lane quarter this warp may access
+    const int trow = quarter * 32 + lane;         // token row inside the tile / output row inside a block
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    float l_part[N];                              // per-thread partial softmax denominators
+#pragma unroll
+    for (int h = 0; h < N; ++h) l_part[h] = 0.f;
+    float m_ref = -INFINITY;                      // lane h holds head h's reference max (N <= 32 per group)
+    unsigned rope_n = 0;
+    bool ok = true;
+    static_assert(N == 32, "softmax threads keep one head per lane");
+
+    for (int tile = 0; tile < n_tiles && ok; ++tile) {
+      const int nvalid = min(kTile, ntok - tile * kTile);
+      float s[N];
+#pragma unroll
+      for (int h = 0; h < N; ++h) s[h] = 0.f;
+      // ---- rope part of the score (FP32 FMA)
+#pragma unroll
+      for (int cb = 0; cb < NRB; ++cb) {
+        if (!ok) break;
+        const unsigned slot = rope_n % kRopeSlots;
+        ok = mbar_wait(smem_u32(&bars->rope_full[slot]), (rope_n / kRopeSlots) & 1, s_abort);
+        if (!ok) break;
+        const unsigned char* rowp = s_rope + slot * kChunkBytes + trow * 128;
+        float part[HPB];
+#pragma unroll
+        for (int hh = 0; hh < HPB; ++hh) part[hh] = 0.f;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const uint4 v = *(const uint4*)(rowp + ((c ^ (trow & 7)) << 4));
+          const bf162* k2 = (const bf162*)&v;
+          const int hh = (c * 8) / R2;                       // head inside the box
+          const float* qq = s_qrope + (cb * HPB + hh) * R2 + (c * 8) % R2;
+          const float4 q0 = *(const float4*)qq, q1 = *(const float4*)(qq + 4);
+          const float2 k0 = __bfloat1622float2(k2[0]), k1 = __bfloat1622float2(k2[1]);
+          const float2 k2f = __bfloat1622float2(k2[2]), k3 = __bfloat1622float2(k2[3]);
+          float acc = part[hh];
+          acc = fmaf(q0.x, k0.x, acc); acc = fmaf(q0.y, k0.y, acc);
+          acc = fmaf(q0.z, k1.x, acc); acc = fmaf(q0.w, k1.y, acc);
+          acc = fmaf(q1.x, k2f.x, acc); acc = fmaf(q1.y, k2f.y, acc);
+          acc = fmaf(q1.z, k3.x, acc); acc = fmaf(q1.w, k3.y, acc);
+          part[hh] = acc;
+        }
+#pragma unroll
+        for (int hh = 0; hh < HPB; ++hh) s[cb * HPB + hh] = part[hh];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars->rope_empty[slot]));
+        ++rope_n;
+      }
+      if (!ok) break;
+      // ---- latent part from TMEM
+      ok = mbar_wait(smem_u32(&bars->s_full), tile & 1, s_abort);
+      if (!ok) break;
+      tc_fence_after();
+      {
+        float sv[32];
+        tc_ld32(tmem_s + lane_base, sv);
+        tc_wait_ld();
+#pragma unroll
+        for (int h = 0; h < N; ++h) {
+          const float x = (s[h] + sv[h]) * a.scale_log2e;
+          s[h] = trow < nvalid ? x : -INFINITY;
+        }
+      }
+      // ---- per-head max over the 128 tokens of the tile
+      float wm = -INFINITY;
+#pragma unroll
+      for (int h = 0; h < N; ++h) {
+        const float v = ord2f(__reduce_max_sync(0xffffffffu, f2ord(s[h])));
+        if (lane == h) wm = v;
+      }
+      s_wmax[quarter * N + lane] = wm;
+      named_bar_sync(1, kSoftmaxThreads);
+      float tm = fmaxf(fmaxf(s_wmax[lane], s_wmax[N + lane]), fmaxf(s_wmax[2 * N + lane], s_wmax[3 * N + lane]));
+      // reference max moves only when the tile max exceeds it by more than 2^8
+      const bool move = tm > m_ref + 8.f;
+      const float m_new = move ? tm : m_ref;
+      const float corr = move ? exp2f(m_ref - m_new) : 1.f;      // 0 on the first tile
+      m_ref = m_new;
+      const bool any_move = __any_sync(0xffffffffu, move);       // same in all four warps
+      if (any_move && quarter == 0) s_corr[lane] = corr;
+      // ---- probabilities, partial sums, P tile in the no-swizzle MN-major layout
+#pragma unroll
+      for (int j = 0; j < N / 8; ++j) {
+        uint32_t packed[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int h0 = j * 8 + 2 * e;
+          const float mh0 = __shfl_sync(0xffffffffu, m_new, h0), mh1 = __shfl_sync(0xffffffffu, m_new, h0 + 1);
+          const float p0 = exp2f(s[h0] - mh0), p1 = exp2f(s[h0 + 1] - mh1);
+          if (any_move) {
+            l_part[h0] *= __shfl_sync(0xffffffffu, corr, h0);
+            l_part[h0 + 1] *= __shfl_sync(0xffffffffu, corr, h0 + 1);
+          }
+          const bf162 pb = __floats2bfloat162_rn(p0, p1);
+          // sum what the tensor core will actually see (bf16-rounded probabilities)
+          const float2 pr = __bfloat1622float2(pb);
+          l_part[h0] += pr.x;
+          l_part[h0 + 1] += pr.y;
+          packed[e] = *(const uint32_t*)&pb;
+        }
+        *(uint4*)(s_p + j * 2048 + (trow >> 3) * 128 + (trow & 7) * 16) =
+            make_uint4(packed[0], packed[1], packed[2], packed[3]);
+      }
+      // ---- rescale the TMEM-resident output when a reference moved (skip on the first tile:
+      //      the first pass-B MMA overwrites)
+      if (any_move && tile > 0) {
+        named_bar_sync(1, kSoftmaxThreads);      // s_corr visible
+        for (int blk = 0; blk < NB; ++blk) {
+          float v[32];
+          tc_ld32(tmem_base + blk * N + lane_base, v);
+          tc_wait_ld();
+#pragma unroll
+          for (int h = 0; h < N; ++h) v[h] *= s_corr[h];
+          tc_st32(tmem_base + blk * N + lane_base, v);
+        }
+        tc_wait_st();
+      }
+      fence_proxy_async();
+      tc_fence_before();
+      mbar_arrive(smem_u32(&bars->p_ready));
+    }
+
+    // ---- epilogue: partial output and softmax statistics of this item
+    if (ok) ok = mbar_wait(smem_u32(&bars->pv_done), (n_tiles - 1) & 1, s_abort);
+    if (ok) {
+      tc_fence_after();
+      float* pa = a.part_acc + (size_t)item * a.n_h * d_c;
+      for (int blk = 0; blk < NB; ++blk) {
+        float v[32];
+        tc_ld32(tmem_base + blk * N + lane_base, v);
+        tc_wait_ld();
+        const int d = blk * 128 + trow;
+#pragma unroll
+        for (int h = 0; h < N; ++h)
+          if (h < a.n_h) pa[(size_t)h * d_c + d] = v[h];
+      }
+      float wl = 0.f;
+#pragma unroll
+      for (int h = 0; h < N; ++h) {
+        const float v = warp_sum(l_part[h]);
+        if (lane == h) wl = v;
+      }
+      named_bar_sync(1, kSoftmaxThreads);
+      s_wmax[quarter * N + lane] = wl;
+      named_bar_sync(1, kSoftmaxThreads);
+      if (quarter == 0 && lane < a.n_h) {
+        const float lsum = s_wmax[lane] + s_wmax[N + lane] + s_wmax[2 * N + lane] + s_wmax[3 * N + lane];
+        a.part_ml[((size_t)item * a.n_h + lane) * 2 + 0] = m_ref;
+        a.part_ml[((size_t)item * a.n_h + lane) * 2 + 1] = lsum;
+      }
+    }
+  }
+
+  // ============================================================== teardown
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *s_abort) ekv_record(a.status, ELITEKV_ERR_TIMEOUT, item, seq);
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+// 2-D bf16 tensor [rows][cols] (cols contiguous), box [box_rows][64], 128-byte swizzle
+int make_map(CUtensorMap* m, const void* ptr, unsigned long long rows, unsigned long long cols, unsigned box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return ELITEKV_ERR_CUDA;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * sizeof(bf16)};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? ELITEKV_OK : ELITEKV_ERR_CUDA;
+}
+
+}  // namespace
+
+int ekv_tc_supported(const elitekv_layer* L, const elitekv_cache* cache) {
+  const int r2 = 2 * L->r;
+  if (L->n_h != 32) return 0;
+  if (L->d_c % 128 != 0 || (L->d_c / 128 + 1) * 32 > 512) return 0;
+  if (!(r2 == 8 || r2 == 16 || r2 == 32)) return 0;
+  if (Smem<32>::total(L->d_c) > L->smem_optin) return 0;
+  if (cache && cache->page_table && (cache->page_size % 64 != 0)) return 0;
+  return 1;
+}
+
+int ekv_tc_max_items(const elitekv_layer* L, int B) { return L->sm_count + B; }
+
+int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, const CacheView& cv,
+                         const void* q_rope, const void* q_abs, int B, const DecodeScratch& ws,
+                         cudaStream_t st) {
+  if (!ekv_tc_supported(L, cache)) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
+  const unsigned long long rows =
+      cv.page_table ? (unsigned long long)cv.num_pages << cv.page_shift : (unsigned long long)cv.max_ctx * cv.n_seqs;
+  CUtensorMap m_lat, m_rope, m_q;
+  int rc = make_map(&m_lat, cache->latent, rows, L->d_c, 64);
+  if (rc == ELITEKV_OK) rc = make_map(&m_rope, cache->rope, rows, (unsigned long long)L->n_h * 2 * L->r, 64);
+  if (rc == ELITEKV_OK) rc = make_map(&m_q, q_abs, (unsigned long long)B * L->n_h, L->d_c, 32);
+  if (rc != ELITEKV_OK) return rc;
+  TcArgs a;
+  a.items = ws.items;
+  a.page_table = cv.page_table;
+  a.part_acc = ws.part_acc;
+  a.part_ml = ws.part_ml;
+  a.q_rope = (const bf16*)q_rope;
+  a.status = L->d_status;
+  a.max_ctx = cv.max_ctx;
+  a.num_pages = cv.num_pages;
+  a.page_shift = cv.page_shift;
+  a.page_mask = cv.page_mask;
+  a.max_pages_per_seq = cv.max_pages_per_seq;
+  a.n_h = L->n_h;
+  a.d_c = L->d_c;
+  a.scale_log2e = L->scale * 1.4426950408889634f;
+  const int smem = Smem<32>::total(L->d_c);
+  auto launch = [&](auto kern) -> int {
+    EKV_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    kern<<<ws.max_items, kThreads, smem, st>>>(m_lat, m_rope, m_q, a);
+    EKV_CUDA_OK(cudaGetLastError());
+    return ELITEKV_OK;
+  };
+  switch (2 * L->r) {
+    case 8: return launch(decode_tc_kernel<32, 8>);
+    case 16: return launch(decode_tc_kernel<32, 16>);
+    default: return launch(decode_tc_kernel<32, 32>);
+  }
+}

@@ -199,6 +199,34 @@ def test_decode_7b_shape_small_context(ek):
     H.check_parity(st, out, H.all_units(st))
 
 
+@pytest.mark.parametrize("kernel", [1, 2], ids=["generic", "tensor-core"])
+def test_decode_7b_shape_ragged_tails_both_kernels(ek, kernel):
+    """Same inputs through the CUDA-core kernel and the tcgen05 kernel: lengths around the
+    16-token MMA step and the 128-token tile."""
+    w = gen.shrink(gen.LLAMA7B_75, B=8, ctx=400)
+    st = H.setup(w, lens=[1, 15, 16, 17, 127, 128, 129, 400], decode_kernel=kernel)
+    out = H.run_decode(st)
+    H.check_parity(st, out, H.all_units(st))
+
+
+@pytest.mark.parametrize("page_size", [64, 128])
+def test_decode_7b_shape_paged_tensor_core(ek, page_size):
+    w = replace(gen.shrink(gen.LLAMA7B_75, B=3, ctx=700), paged=True, page_size=page_size)
+    st = H.setup(w, lens=[700, 64, 193], decode_kernel=2)
+    out = H.run_decode(st)
+    H.check_parity(st, out, H.all_units(st))
+
+
+def test_tensor_core_kernel_refuses_uncovered_shapes(ek):
+    w = replace(SMALL, seed=64)
+    st = H.setup(w, lens=[5, 5, 5], decode_kernel=0)
+    idx = gen.elite_index_sets(w)
+    layer = ek.Layer(w.n_h, w.d_h, w.r, w.d_c, idx, st.W_uk, st.W_uv, 64, decode_kernel=2)
+    with pytest.raises(ek.ElitekvError) as e:
+        ek.elitekv_decode_workspace_size(layer, 3)
+    assert e.value.code == ek.ERR_UNSUPPORTED_SHAPE
+
+
 def test_decode_13b_shape_small_context(ek):
     w = gen.shrink(gen.LLAMA13B_75, B=2, ctx=300)
     st = H.setup(w, lens=[300, 129])

@@ -137,14 +137,28 @@ def oracle_sample(w: gen.Workload, n_units: int, seed_shift: int = 0):
     return dt, len(heads), f"{len(heads)} heads of sequence {b} at full context {n} (of {w.B}x{w.n_h} units)"
 
 
-def cpu_baseline(w: gen.Workload, budget_s: float = 15.0):
-    dt1, u1, _ = oracle_sample(w, 2)
-    units = int(max(2, min(w.n_h, budget_s / max(dt1 / u1, 1e-6))))
-    dt, u, what = oracle_sample(w, units)
-    # tokens/s for the whole step: B sequences need B*n_h units
-    value = (u / w.n_h) / dt
+def cpu_baseline(w: gen.Workload, budget_s: float = 12.0):
+    """Whole sequences (all heads) through the oracle until about `budget_s` seconds are spent."""
+    t_total, units, seqs = 0.0, 0, 0
+    while seqs < w.B and (seqs == 0 or t_total * (seqs + 1) / seqs < budget_s):
+        dt, u, _ = oracle_sample(w, w.n_h, seed_shift=seqs)
+        t_total += dt
+        units += u
+        seqs += 1
+    value = (units / w.n_h) / t_total        # sequences (= decode tokens) per second, one layer
     return {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
-            "sample": what + f"; {dt:.2f} s, scaled by units"}
+            "sample": f"{seqs} of {w.B} sequences, all {w.n_h} heads, full context; "
+                      f"{t_total:.2f} s of oracle time"}
+
+
+def config_of(w: gen.Workload, world: int, cache_bytes=None):
+    c = {"workload": w.name, "n_h": w.n_h, "d_h": w.d_h, "r": w.r, "d_c": w.d_c,
+         "batch_per_gpu": w.B, "context": w.ctx, "paged": w.paged,
+         "l2": "256 MiB flush write before every timed step; cache larger than L2",
+         "parallelism": f"replicas x{world} (independent sequences, no collective)"}
+    if cache_bytes is not None:
+        c["cache_bytes_per_step"] = cache_bytes
+    return c
 
 
 def run_reference(args, w: gen.Workload):
@@ -164,8 +178,7 @@ def run_reference(args, w: gen.Workload):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_unit * w.n_h * w.B * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
-        "config": {"workload": w.name, "n_h": w.n_h, "d_h": w.d_h, "r": w.r, "d_c": w.d_c,
-                   "batch": w.B, "context": w.ctx},
+        "config": config_of(w, max(args.gpus, 1)),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
                          "sample": f"each step {n_units} (sequence, head) units at full context, "
                                    "time scaled to the whole batch"},
@@ -265,6 +278,7 @@ def run_gpu(args, w: gen.Workload):
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local) if rank == 0 else None
     for _ in range(max(args.warmup, 3)):
         step(ek, layer, cache, dev, ws, bufs)
     torch.cuda.synchronize()
@@ -274,7 +288,6 @@ def run_gpu(args, w: gen.Workload):
     ek.elitekv_profile_enable(layer, True)
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
           for _ in range(args.steps)]
-    sampler = ClockSampler(local) if rank == 0 else None
     barrier()
     for a, b in ev:
         flush.fill_(1)
@@ -282,7 +295,6 @@ def run_gpu(args, w: gen.Workload):
         step(ek, layer, cache, dev, ws, bufs)
         b.record()
     barrier()
-    clocks = sampler.stop() if sampler else None
     step_ms = [a.elapsed_time(b) for a, b in ev]
     total_ms = sum(step_ms)
     kern_ms, kern_n = ek.elitekv_profile_collect(layer)
@@ -308,6 +320,31 @@ def run_gpu(args, w: gen.Workload):
         e2e_step()           # no flush here: the 268 MB+ cache does not fit the 126 MB L2
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
+
+    # ---- per-call breakdown (informational; same kernels, a few extra untimed-by-the-metric calls)
+    def timed(fn, n=10):
+        evs = []
+        for _ in range(n):
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            evs.append((a, b))
+        torch.cuda.synchronize()
+        return 1e3 * sum(a.elapsed_time(b) for a, b in evs) / n
+    stages = {
+        "append_us": timed(lambda: ek.elitekv_append(layer, cache, dev["k_e"], dev["c"], dev["seq_id"], dev["pos"])),
+        "absorb_us": timed(lambda: ek.elitekv_absorb_query(layer, dev["q"], dev["pos"], bufs["q_rope"], bufs["q_abs"])),
+        "decode_us": timed(lambda: ek.elitekv_decode(layer, cache, bufs["q_rope"], bufs["q_abs"], dev["lens"], ws, bufs["out"])),
+    }
+    # keep the GPU busy long enough for the clock sampler to see it under load
+    t_busy = time.perf_counter()
+    while time.perf_counter() - t_busy < 0.6:
+        for _ in range(20):
+            step(ek, layer, cache, dev, ws, bufs)
+        torch.cuda.synchronize()
+    clocks = sampler.stop() if sampler else None
     assert ek.elitekv_check_status(layer) == 0
 
     # ---- comparator: uncompressed RoPE-MHA decode at the same shape (rank 0, one GPU)
@@ -361,11 +398,7 @@ def run_gpu(args, w: gen.Workload):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": w.name, "n_h": w.n_h, "d_h": w.d_h, "r": w.r, "d_c": w.d_c,
-                   "batch_per_gpu": w.B, "context": w.ctx, "paged": w.paged,
-                   "cache_bytes_per_step": cache_bytes,
-                   "l2": "256 MiB flush write before every timed step; cache larger than L2",
-                   "parallelism": f"replicas x{world} (independent sequences, no collective)"},
+        "config": config_of(w, world, cache_bytes),
         "hbm_gbs_whole_step": cache_bytes / (ms_per_step * 1e-3) / 1e9,
         "pct_of_nominal_8tbs_whole_step": 100.0 * cache_bytes / (ms_per_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
         "roofline": {"bound": "hbm", "kernel": "split-K decode attention", "achieved": achieved,
@@ -378,6 +411,7 @@ def run_gpu(args, w: gen.Workload):
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": KERNELS_PER_STEP * args.steps,
         "clocks": clocks,
+        "stages": stages,
         "comparator": comparator,
     }
     if not args.no_cpu_baseline and world == 1:

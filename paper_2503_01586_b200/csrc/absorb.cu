@@ -4,16 +4,19 @@
 //   q_rope[b,h,2j:2j+2] = q[b,h,chunk idx[h][j]] . R(q_pos[b] * theta_idx[h][j])
 //   q_abs [b,h,k]       = sum_i q_nope[b,h,i] * W_uk[k][h*dn + i]
 //
-// Grid (n_h, ceil(d_c/256)): a block owns one head and 256 latent coordinates; each thread
-// owns two adjacent coordinates and keeps one fp32 accumulator pair per sequence of the
-// current batch chunk, so every weight element is read once per chunk of 16 sequences.  The
-// weights come regrouped as [n_h][dn][d_c] (d_c contiguous), which makes the reads coalesced.
+// Grid (n_h, ceil(d_c/128)): a block owns one head and 128 latent coordinates.  Its 256 threads
+// are 64 coordinate pairs x 4 groups over the head's un-rotated dims; every thread keeps one fp32
+// accumulator pair per sequence of the current chunk of 16 sequences, so each weight element is
+// read once per chunk, and the four groups are added through shared memory.  The weights come
+// regrouped as [n_h][dn][d_c] (d_c contiguous), which makes the reads coalesced.
 #include "common.cuh"
 
 namespace {
 
 constexpr int kAbsorbBatch = 16;
-constexpr int kAbsorbThreads = 128;
+constexpr int kAbsorbThreads = 256;
+constexpr int kAbsorbGroups = 4;
+constexpr int kAbsorbCoords = 128;
 
 __global__ void __launch_bounds__(kAbsorbThreads)
 absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int B,
@@ -21,10 +24,13 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
               const int32_t* __restrict__ idx, const float2* __restrict__ cs, bf16* __restrict__ q_rope,
               bf16* __restrict__ q_abs, int n_h, int d_h, int r, int d_c, int max_pos,
               int32_t* status) {
-  extern __shared__ float q_nope[];   // [kAbsorbBatch][dn]
+  extern __shared__ __align__(16) float smem_f[];
   const int h = blockIdx.x;
   const int dn = d_h - 2 * r;
-  const int k = (blockIdx.y * kAbsorbThreads + threadIdx.x) * 2;
+  float* q_nope = smem_f;                                   // [dn][16] (sequence fastest)
+  float* red = smem_f + (size_t)(dn > 0 ? dn : 1) * kAbsorbBatch;   // [3][16][128]
+  const int pair = threadIdx.x & 63, grp = threadIdx.x >> 6;
+  const int k = blockIdx.y * kAbsorbCoords + 2 * pair;
   const int32_t* dims = qdims + (size_t)h * d_h;
 
   // rope part: one block per head does it
@@ -46,33 +52,56 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
     }
   }
 
+  const int per_grp = (dn + kAbsorbGroups - 1) / kAbsorbGroups;
+  const int i_lo = min(dn, grp * per_grp), i_hi = min(dn, i_lo + per_grp);
   for (int b0 = 0; b0 < B; b0 += kAbsorbBatch) {
     const int nb = min(kAbsorbBatch, B - b0);
     __syncthreads();
-    for (int e = threadIdx.x; e < nb * dn; e += blockDim.x) {
-      const int bb = e / dn, i = e % dn;
-      q_nope[bb * dn + i] = __bfloat162float(q[((size_t)(b0 + bb) * n_h + h) * d_h + dims[2 * r + i]]);
+    for (int e = threadIdx.x; e < kAbsorbBatch * dn; e += blockDim.x) {
+      const int i = e / kAbsorbBatch, bb = e % kAbsorbBatch;
+      q_nope[e] = bb < nb ? __bfloat162float(q[((size_t)(b0 + bb) * n_h + h) * d_h + dims[2 * r + i]]) : 0.f;
     }
     __syncthreads();
-    if (k < d_c) {
-      float a0[kAbsorbBatch], a1[kAbsorbBatch];
+    float a0[kAbsorbBatch], a1[kAbsorbBatch];
 #pragma unroll
-      for (int bb = 0; bb < kAbsorbBatch; ++bb) a0[bb] = a1[bb] = 0.f;
+    for (int bb = 0; bb < kAbsorbBatch; ++bb) a0[bb] = a1[bb] = 0.f;
+    if (k < d_c) {
       const bf16* wp = WukT + (size_t)h * dn * d_c + k;
 #pragma unroll 4
-      for (int i = 0; i < dn; ++i) {
+      for (int i = i_lo; i < i_hi; ++i) {
         const float2 w = __bfloat1622float2(*(const bf162*)(wp + (size_t)i * d_c));
+        const float4* xr = (const float4*)(q_nope + (size_t)i * kAbsorbBatch);
 #pragma unroll
-        for (int bb = 0; bb < kAbsorbBatch; ++bb) {
-          const float x = q_nope[bb * dn + i];   // rows beyond nb hold stale values; results unused
-          a0[bb] = fmaf(x, w.x, a0[bb]);
-          a1[bb] = fmaf(x, w.y, a1[bb]);
+        for (int v = 0; v < kAbsorbBatch / 4; ++v) {
+          const float4 x = xr[v];
+          a0[4 * v + 0] = fmaf(x.x, w.x, a0[4 * v + 0]); a1[4 * v + 0] = fmaf(x.x, w.y, a1[4 * v + 0]);
+          a0[4 * v + 1] = fmaf(x.y, w.x, a0[4 * v + 1]); a1[4 * v + 1] = fmaf(x.y, w.y, a1[4 * v + 1]);
+          a0[4 * v + 2] = fmaf(x.z, w.x, a0[4 * v + 2]); a1[4 * v + 2] = fmaf(x.z, w.y, a1[4 * v + 2]);
+          a0[4 * v + 3] = fmaf(x.w, w.x, a0[4 * v + 3]); a1[4 * v + 3] = fmaf(x.w, w.y, a1[4 * v + 3]);
         }
       }
+    }
+    if (grp > 0) {
 #pragma unroll
       for (int bb = 0; bb < kAbsorbBatch; ++bb)
-        if (bb < nb)
-          *(bf162*)(q_abs + ((size_t)(b0 + bb) * n_h + h) * d_c + k) = __floats2bfloat162_rn(a0[bb], a1[bb]);
+        *(float2*)(red + ((size_t)(grp - 1) * kAbsorbBatch + bb) * kAbsorbCoords + 2 * pair) =
+            make_float2(a0[bb], a1[bb]);
+    }
+    __syncthreads();
+    if (grp == 0 && k < d_c) {
+#pragma unroll
+      for (int bb = 0; bb < kAbsorbBatch; ++bb) {
+        if (bb < nb) {
+          float s0 = a0[bb], s1 = a1[bb];
+#pragma unroll
+          for (int g = 0; g < kAbsorbGroups - 1; ++g) {
+            const float2 t = *(const float2*)(red + ((size_t)g * kAbsorbBatch + bb) * kAbsorbCoords + 2 * pair);
+            s0 += t.x;
+            s1 += t.y;
+          }
+          *(bf162*)(q_abs + ((size_t)(b0 + bb) * n_h + h) * d_c + k) = __floats2bfloat162_rn(s0, s1);
+        }
+      }
     }
   }
 }
@@ -82,8 +111,10 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
 int ekv_launch_absorb(const elitekv_layer* L, const void* q, const int32_t* q_pos, int B,
                       void* q_rope, void* q_abs, cudaStream_t st) {
   if (B == 0) return ELITEKV_OK;
-  dim3 grid(L->n_h, (L->d_c + 2 * kAbsorbThreads - 1) / (2 * kAbsorbThreads));
-  size_t smem = sizeof(float) * kAbsorbBatch * (size_t)(L->dn > 0 ? L->dn : 1);
+  dim3 grid(L->n_h, (L->d_c + kAbsorbCoords - 1) / kAbsorbCoords);
+  size_t smem = sizeof(float) * (kAbsorbBatch * (size_t)(L->dn > 0 ? L->dn : 1) +
+                                 (size_t)(kAbsorbGroups - 1) * kAbsorbBatch * kAbsorbCoords);
+  EKV_CUDA_OK(cudaFuncSetAttribute(absorb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   absorb_kernel<<<grid, kAbsorbThreads, smem, st>>>(
       (const bf16*)q, q_pos, B, L->d_WukT, L->d_qdims, L->d_idx, L->d_cs, (bf16*)q_rope,
       (bf16*)q_abs, L->n_h, L->d_h, L->r, L->d_c, L->max_pos, L->d_status);

@@ -31,7 +31,7 @@ int max_items_any(const elitekv_layer* L, int B) {
 }
 
 struct Carve {
-  size_t off_items, off_first, off_ml, off_acc, total;
+  size_t off_items, off_first, off_ml, off_acc, off_slice, off_cnt, total;
 };
 
 Carve carve(const elitekv_layer* L, int B, int max_items) {
@@ -41,6 +41,8 @@ Carve carve(const elitekv_layer* L, int B, int max_items) {
   c.off_first = o; o = align256(o + sizeof(int32_t) * ((size_t)B + 1));
   c.off_ml = o;    o = align256(o + sizeof(float) * 2 * (size_t)max_items * L->n_h);
   c.off_acc = o;   o = align256(o + sizeof(float) * (size_t)max_items * L->n_h * L->d_c);
+  c.off_slice = o; o = align256(o + ekv_combine_scratch_bytes(L, B));
+  c.off_cnt = o;   o = align256(o + sizeof(int32_t) * (size_t)ekv_combine_counters(L, B));
   c.total = o;
   return c;
 }
@@ -99,9 +101,12 @@ extern "C" int elitekv_decode(const elitekv_layer* L, const elitekv_cache* cache
   ws.seq_first = (int32_t*)(base + cw.off_first);
   ws.part_ml = (float*)(base + cw.off_ml);
   ws.part_acc = (float*)(base + cw.off_acc);
+  ws.slice_out = (float*)(base + cw.off_slice);
+  ws.counters = (int32_t*)(base + cw.off_cnt);
+  ws.n_counters = ekv_combine_counters(L, B);
   cudaStream_t st = (cudaStream_t)stream;
   rc = ekv_launch_plan(seq_lens, B, kernel == 2 ? 128 : ELITEKV_TILE_TOKENS, max_items, ws.items,
-                       ws.seq_first, st);
+                       ws.seq_first, ws.counters, ws.n_counters, st);
   if (rc != ELITEKV_OK) return rc;
   EkvProfile* prof = (L->prof && L->prof->enabled && L->prof->count < kProfileSlots) ? L->prof : nullptr;
   if (prof) EKV_CUDA_OK(cudaEventRecord(prof->ev[2 * prof->count], st));

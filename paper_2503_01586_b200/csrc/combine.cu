@@ -5,13 +5,139 @@
 //   M = max_s m_s,  L = sum_s l_s 2^(m_s - M),  o_lat = sum_s acc_s 2^(m_s - M) / L
 //   o[b,h,:] = o_lat . W_uv[:, h*d_h:(h+1)*d_h]        (B^v folded outwards, Section 5;
 //                                                      V = c W_uv of Section 3.2)
-// Grid (n_h, ceil(B/8)): a block owns one head and up to 8 sequences, so W_uv's head slice is
-// read once per 8 sequences.  Threads are (output dim pair) x (k group); the latent axis is
-// walked in chunks of 128 that are merged into shared memory first.
+//
+// Fast kernel (d_h = 128, d_c % 128 == 0): grid (n_h, d_c/128).  A block owns one head and one
+// 128-wide slice of the latent axis: it stages W_uv's [128 x 128] sub-block in shared memory
+// once, then for every group of 16 sequences merges the items' partial outputs of its slice
+// (16-byte loads, weights 2^(m_s-M)/L) and multiplies.  The d_c/128 slice results of a head are
+// written to scratch; the block that finishes last for that (head, sequence group) adds them in
+// a fixed order and writes bf16, so the result does not depend on scheduling.
+//
+// Generic kernel: any even d_h <= 512, any d_c; block per (head, 8 sequences).
 #include "common.cuh"
 
 namespace {
 
+// ------------------------------------------------------------------ fast path
+constexpr int kFB = 16;          // sequences per group
+constexpr int kFK = 128;         // latent slice
+constexpr int kFD = 128;         // head dim
+constexpr int kFThreads = 256;
+
+__global__ void __launch_bounds__(kFThreads)
+combine_fast_kernel(const float* __restrict__ part_acc, const float* __restrict__ part_ml,
+                    const int32_t* __restrict__ seq_first, const bf16* __restrict__ Wuv,
+                    float* __restrict__ slice_out /* [n_slices][B][n_h][128] */,
+                    int32_t* __restrict__ counters /* [n_h][n_groups], zeroed by the plan kernel */,
+                    bf16* __restrict__ out, int B, int n_h, int d_c) {
+  __shared__ __align__(16) bf16 s_w[kFK][kFD];          // 32 KB
+  __shared__ __align__(16) float s_x[kFB][kFK];         // 8 KB merged latent outputs
+  __shared__ float s_M[kFB], s_invL[kFB];
+  __shared__ int s_first[kFB + 1];
+  __shared__ int s_last;
+  const int h = blockIdx.x, slice = blockIdx.y, n_slices = gridDim.y;
+  const int k0 = slice * kFK;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  // W_uv[k0 + k][h*128 + d] -> shared, 16 bytes per thread per step
+  for (int e = tid; e < kFK * (kFD / 8); e += kFThreads) {
+    const int k = e / (kFD / 8), v = e % (kFD / 8);
+    *(uint4*)&s_w[k][v * 8] =
+        __ldg((const uint4*)(Wuv + (size_t)(k0 + k) * n_h * kFD + (size_t)h * kFD + v * 8));
+  }
+
+  const int n_groups = (B + kFB - 1) / kFB;
+  for (int g = 0; g < n_groups; ++g) {
+    const int b0 = g * kFB, nb = min(kFB, B - b0);
+    __syncthreads();
+    if (tid <= nb) s_first[tid] = seq_first[b0 + tid];
+    __syncthreads();
+    // softmax statistics per sequence: one warp each
+    for (int bb = warp; bb < nb; bb += kFThreads / 32) {
+      const int i0 = s_first[bb], i1 = s_first[bb + 1];
+      float M = -INFINITY;
+      for (int i = i0 + lane; i < i1; i += 32) M = fmaxf(M, part_ml[((size_t)i * n_h + h) * 2]);
+      M = warp_max(M);
+      float Ls = 0.f;
+      for (int i = i0 + lane; i < i1; i += 32) {
+        const float* ml = part_ml + ((size_t)i * n_h + h) * 2;
+        Ls += ml[1] * exp2f(ml[0] - M);
+      }
+      Ls = warp_sum(Ls);
+      if (lane == 0) {
+        s_M[bb] = M;
+        s_invL[bb] = (i1 > i0 && Ls > 0.f) ? 1.f / Ls : 0.f;
+      }
+    }
+    __syncthreads();
+    // merge the items of each sequence on this latent slice
+    for (int e = tid; e < kFB * (kFK / 4); e += kFThreads) {
+      const int bb = e / (kFK / 4), v = e % (kFK / 4);
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (bb < nb) {
+        const float M = s_M[bb];
+        for (int i = s_first[bb]; i < s_first[bb + 1]; ++i) {
+          const float w = exp2f(part_ml[((size_t)i * n_h + h) * 2] - M);
+          const float4 p = __ldg((const float4*)(part_acc + ((size_t)i * n_h + h) * d_c + k0 + v * 4));
+          acc.x = fmaf(w, p.x, acc.x); acc.y = fmaf(w, p.y, acc.y);
+          acc.z = fmaf(w, p.z, acc.z); acc.w = fmaf(w, p.w, acc.w);
+        }
+        const float il = s_invL[bb];
+        acc.x *= il; acc.y *= il; acc.z *= il; acc.w *= il;
+      }
+      *(float4*)&s_x[bb][v * 4] = acc;
+    }
+    __syncthreads();
+    // [16 x 128] . [128 x 128]: thread = (dim pair, group of 4 sequences)
+    {
+      const int pair = tid & 63, bg = tid >> 6;
+      float a0[4] = {0.f, 0.f, 0.f, 0.f}, a1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 2
+      for (int k = 0; k < kFK; k += 4) {
+        float4 x[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) x[j] = *(const float4*)&s_x[bg * 4 + j][k];
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+          const float2 w = __bfloat1622float2(*(const bf162*)&s_w[k + kk][2 * pair]);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const float xv = kk == 0 ? x[j].x : kk == 1 ? x[j].y : kk == 2 ? x[j].z : x[j].w;
+            a0[j] = fmaf(xv, w.x, a0[j]);
+            a1[j] = fmaf(xv, w.y, a1[j]);
+          }
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int bb = bg * 4 + j;
+        if (bb < nb)
+          *(float2*)(slice_out + (((size_t)slice * B + b0 + bb) * n_h + h) * kFD + 2 * pair) =
+              make_float2(a0[j], a1[j]);
+      }
+    }
+    // last block of this (head, group) adds the slices in order
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = atomicAdd(&counters[h * n_groups + g], 1) == n_slices - 1;
+    __syncthreads();
+    if (s_last) {
+      __threadfence();
+      for (int e = tid; e < nb * (kFD / 2); e += kFThreads) {
+        const int bb = e / (kFD / 2), p2 = e % (kFD / 2);
+        float2 v = make_float2(0.f, 0.f);
+        for (int s = 0; s < n_slices; ++s) {
+          const float2 t = __ldcg((const float2*)(slice_out + (((size_t)s * B + b0 + bb) * n_h + h) * kFD + 2 * p2));
+          v.x += t.x;
+          v.y += t.y;
+        }
+        *(bf162*)(out + ((size_t)(b0 + bb) * n_h + h) * kFD + 2 * p2) = __floats2bfloat162_rn(v.x, v.y);
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------ generic path
 constexpr int kCombBatch = 8;
 constexpr int kCombThreads = 256;
 constexpr int kCombChunk = 128;
@@ -35,7 +161,6 @@ combine_upproj_kernel(const float* __restrict__ part_acc, const float* __restric
 
   if (threadIdx.x <= nb) s_first[threadIdx.x] = seq_first[b0 + threadIdx.x];
   __syncthreads();
-  // softmax statistics of each sequence: one warp per sequence
   {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int bb = warp; bb < nb; bb += kCombThreads / 32) {
@@ -63,7 +188,6 @@ combine_upproj_kernel(const float* __restrict__ part_acc, const float* __restric
 
   for (int k0 = 0; k0 < d_c; k0 += kCombChunk) {
     const int kc = min(kCombChunk, d_c - k0);
-    // merge the items of each sequence for this slice of the latent axis
     for (int e = threadIdx.x; e < kCombBatch * kCombChunk; e += kCombThreads) {
       const int bb = e / kCombChunk, k = e % kCombChunk;
       float v = 0.f;
@@ -93,7 +217,6 @@ combine_upproj_kernel(const float* __restrict__ part_acc, const float* __restric
     __syncthreads();
   }
 
-  // reduce over k groups
   if (worker) {
 #pragma unroll
     for (int bb = 0; bb < kCombBatch; ++bb) {
@@ -112,8 +235,27 @@ combine_upproj_kernel(const float* __restrict__ part_acc, const float* __restric
 
 }  // namespace
 
+int ekv_combine_fast_ok(const elitekv_layer* L) { return L->d_h == kFD && L->d_c % kFK == 0; }
+
+size_t ekv_combine_scratch_bytes(const elitekv_layer* L, int B) {
+  if (!ekv_combine_fast_ok(L)) return 0;
+  return sizeof(float) * (size_t)(L->d_c / kFK) * B * L->n_h * kFD;
+}
+
+int ekv_combine_counters(const elitekv_layer* L, int B) {
+  return ekv_combine_fast_ok(L) ? L->n_h * ((B + kFB - 1) / kFB) : 0;
+}
+
 int ekv_launch_combine(const elitekv_layer* L, int B, const DecodeScratch& ws, void* out,
                        cudaStream_t st) {
+  if (ekv_combine_fast_ok(L)) {
+    dim3 grid(L->n_h, L->d_c / kFK);
+    combine_fast_kernel<<<grid, kFThreads, 0, st>>>(ws.part_acc, ws.part_ml, ws.seq_first, L->d_Wuv,
+                                                    ws.slice_out, ws.counters, (bf16*)out, B, L->n_h,
+                                                    L->d_c);
+    EKV_CUDA_OK(cudaGetLastError());
+    return ELITEKV_OK;
+  }
   const int npair = L->d_h / 2;
   if (npair > kCombThreads) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
   const int kgroups = kCombThreads / npair > 0 ? kCombThreads / npair : 1;

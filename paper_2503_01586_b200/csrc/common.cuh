@@ -119,7 +119,7 @@ int ekv_launch_append(const elitekv_layer* L, const elitekv_cache* cache, const 
 int ekv_launch_absorb(const elitekv_layer* L, const void* q, const int32_t* q_pos, int B,
                       void* q_rope, void* q_abs, cudaStream_t st);
 int ekv_launch_plan(const int32_t* seq_lens, int B, int tile_tokens, int max_items, int32_t* items,
-                    int32_t* seq_first_item, cudaStream_t st);
+                    int32_t* seq_first_item, int32_t* zero_ints, int n_zero, cudaStream_t st);
 
 struct DecodeScratch {
   int max_items;          // capacity of the plan
@@ -127,7 +127,14 @@ struct DecodeScratch {
   int32_t* seq_first;     // [B+1]
   float* part_acc;        // [max_items][n_h][d_c]
   float* part_ml;         // [max_items][n_h][2]  (running max in log2 units, running sum)
+  float* slice_out;       // combine: per latent slice partial outputs [d_c/128][B][n_h][128]
+  int32_t* counters;      // combine: arrival counters, zeroed by the plan kernel
+  int n_counters;
 };
+
+int ekv_combine_fast_ok(const elitekv_layer* L);
+size_t ekv_combine_scratch_bytes(const elitekv_layer* L, int B);
+int ekv_combine_counters(const elitekv_layer* L, int B);
 
 int ekv_generic_supported(const elitekv_layer* L);
 int ekv_generic_max_items(const elitekv_layer* L, int B);

@@ -11,31 +11,39 @@
 
 namespace {
 
-constexpr int kPlanThreads = 1024;
+constexpr int kPlanThreads = 256;
 
-__device__ __forceinline__ int block_exclusive_scan(int v, int* smem, int* total) {
-  // Hillis-Steele over blockDim.x entries
-  const int t = threadIdx.x;
-  smem[t] = v;
-  __syncthreads();
-  for (int o = 1; o < blockDim.x; o <<= 1) {
-    int x = t >= o ? smem[t - o] : 0;
-    __syncthreads();
-    smem[t] += x;
-    __syncthreads();
+// exclusive scan over the block (warp shuffles + one shared array of warp totals)
+__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int x = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += x;
   }
-  int incl = smem[t];
-  *total = smem[blockDim.x - 1];
+  if (lane == 31) warp_tot[warp] = incl;
   __syncthreads();
-  return incl - v;
+  int before = 0, all = 0;
+#pragma unroll
+  for (int w = 0; w < kPlanThreads / 32; ++w) {
+    const int t = warp_tot[w];
+    if (w < warp) before += t;
+    all += t;
+  }
+  __syncthreads();
+  *total = all;
+  return before + incl - v;
 }
 
 __global__ void __launch_bounds__(kPlanThreads)
 plan_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int max_items,
-            int32_t* __restrict__ items, int32_t* __restrict__ seq_first) {
-  __shared__ int scan[kPlanThreads];
+            int32_t* __restrict__ items, int32_t* __restrict__ seq_first,
+            int32_t* __restrict__ zero_ints, int n_zero) {
+  __shared__ int warp_tot[kPlanThreads / 32];
   __shared__ long long s_total;
   const int t = threadIdx.x;
+  for (int i = t; i < n_zero; i += blockDim.x) zero_ints[i] = 0;
   if (t == 0) s_total = 0;
   __syncthreads();
   long long local = 0;
@@ -43,7 +51,7 @@ plan_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int max_items
     int n = seq_lens[b];
     local += n > 0 ? (n + tile - 1) / tile : 0;
   }
-  atomicAdd((unsigned long long*)&s_total, (unsigned long long)local);
+  if (local) atomicAdd((unsigned long long*)&s_total, (unsigned long long)local);
   __syncthreads();
   const long long total = s_total;
   const long long budget = max_items - B > 0 ? max_items - B : 1;
@@ -60,7 +68,7 @@ plan_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int max_items
       pieces = (int)((tiles + target - 1) / target);
     }
     int chunk_total;
-    const int first = carry + block_exclusive_scan(pieces, scan, &chunk_total);
+    const int first = carry + block_exclusive_scan(pieces, warp_tot, &chunk_total);
     if (b < B) {
       seq_first[b] = first;
       for (int j = 0; j < pieces; ++j) {
@@ -69,30 +77,21 @@ plan_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int max_items
         const int tok0 = ta * tile;
         const int tok1 = min(tb * tile, n);
         const int it = first + j;
-        if (it < max_items) {
-          items[4 * it + 0] = b;
-          items[4 * it + 1] = tok0;
-          items[4 * it + 2] = tok1 - tok0;
-          items[4 * it + 3] = 0;
-        }
+        if (it < max_items) *(int4*)(items + 4 * it) = make_int4(b, tok0, tok1 - tok0, 0);
       }
     }
     carry += chunk_total;
   }
   if (t == 0) seq_first[B] = carry;
-  for (int it = carry + t; it < max_items; it += blockDim.x) {
-    items[4 * it + 0] = -1;
-    items[4 * it + 1] = 0;
-    items[4 * it + 2] = 0;
-    items[4 * it + 3] = 0;
-  }
+  for (int it = carry + t; it < max_items; it += blockDim.x) *(int4*)(items + 4 * it) = make_int4(-1, 0, 0, 0);
 }
 
 }  // namespace
 
 int ekv_launch_plan(const int32_t* seq_lens, int B, int tile_tokens, int max_items, int32_t* items,
-                    int32_t* seq_first_item, cudaStream_t st) {
-  plan_kernel<<<1, kPlanThreads, 0, st>>>(seq_lens, B, tile_tokens, max_items, items, seq_first_item);
+                    int32_t* seq_first_item, int32_t* zero_ints, int n_zero, cudaStream_t st) {
+  plan_kernel<<<1, kPlanThreads, 0, st>>>(seq_lens, B, tile_tokens, max_items, items, seq_first_item,
+                                          zero_ints, n_zero);
   EKV_CUDA_OK(cudaGetLastError());
   return ELITEKV_OK;
 }
@@ -102,6 +101,7 @@ extern "C" int elitekv_plan(const int32_t* seq_lens, int32_t B, int32_t tile_tok
                             elitekv_stream_t stream) {
   if (!seq_lens || !items || !seq_first_item || B <= 0 || tile_tokens <= 0 || max_items <= B)
     return ELITEKV_ERR_INVALID_ARG;
-  return ekv_launch_plan(seq_lens, B, tile_tokens, max_items, items, seq_first_item,
+  if ((uintptr_t)items & 15) return ELITEKV_ERR_INVALID_ARG;
+  return ekv_launch_plan(seq_lens, B, tile_tokens, max_items, items, seq_first_item, nullptr, 0,
                          (cudaStream_t)stream);
 }

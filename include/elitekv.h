@@ -73,9 +73,11 @@ typedef struct {
                                  precision at create time.  With a caller table the rotated
                                  values are a pure function of the table (each product and sum
                                  rounded separately in fp32, then bf16 nearest-even).          */
-  int32_t decode_kernel;      /* 0 = choose by shape; 1 = generic CUDA-core kernel;
-                                 2 = tensor-core (tcgen05) kernel, error if the shape is not
-                                 covered.                                                      */
+  int32_t decode_kernel;      /* 0 = choose by shape; 1 = generic CUDA-core kernel; 2 = tcgen05
+                                 kernel, one block per item (latent streamed twice); 3 = tcgen05
+                                 kernel on block pairs (latent axis split over a 2-block
+                                 cluster).  2 and 3 fail with UNSUPPORTED_SHAPE when the shape
+                                 is not covered.                                               */
 } elitekv_params;
 
 /* The two cache planes.  Contiguous (page_table == NULL): sequence s, position p live in row

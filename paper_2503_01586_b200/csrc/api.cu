@@ -9,29 +9,38 @@ inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 // tensor-core kernel, -1 = none.  `cache` may be null (shape-only question).
 int select_kernel(const elitekv_layer* L, const elitekv_cache* cache) {
   const bool tc = ekv_tc_supported(L, cache) != 0;
+  const bool tc2 = ekv_tc2_supported(L, cache) != 0;
+  if (L->decode_kernel == 3) return tc2 ? 3 : -1;
   if (L->decode_kernel == 2) return tc ? 2 : -1;
   if (L->decode_kernel == 1) return ekv_generic_supported(L) ? 1 : -1;
+  if (tc2) return 3;
   if (tc) return 2;
   return ekv_generic_supported(L) ? 1 : -1;
 }
 
 int max_items_for(const elitekv_layer* L, int B, int kernel) {
+  if (kernel == 3) return ekv_tc2_max_items(L, B);
   return kernel == 2 ? ekv_tc_max_items(L, B) : ekv_generic_max_items(L, B);
 }
 
 // The workspace is sized for whichever kernel may be picked once the cache layout is known.
 int max_items_any(const elitekv_layer* L, int B) {
   int m = 0;
-  if (ekv_generic_supported(L) && L->decode_kernel != 2) m = ekv_generic_max_items(L, B);
-  if (ekv_tc_supported(L, nullptr) && L->decode_kernel != 1) {
+  const int want = L->decode_kernel;
+  if (ekv_generic_supported(L) && (want == 0 || want == 1)) m = ekv_generic_max_items(L, B);
+  if (ekv_tc_supported(L, nullptr) && (want == 0 || want == 2)) {
     const int t = ekv_tc_max_items(L, B);
+    if (t > m) m = t;
+  }
+  if (ekv_tc2_supported(L, nullptr) && (want == 0 || want == 3)) {
+    const int t = ekv_tc2_max_items(L, B);
     if (t > m) m = t;
   }
   return m;
 }
 
 struct Carve {
-  size_t off_items, off_first, off_ml, off_acc, off_slice, off_cnt, total;
+  size_t off_items, off_first, off_ml, off_acc, off_slice, off_cnt, off_wfirst, total;
 };
 
 Carve carve(const elitekv_layer* L, int B, int max_items) {
@@ -43,6 +52,7 @@ Carve carve(const elitekv_layer* L, int B, int max_items) {
   c.off_acc = o;   o = align256(o + sizeof(float) * (size_t)max_items * L->n_h * L->d_c);
   c.off_slice = o; o = align256(o + ekv_combine_scratch_bytes(L, B));
   c.off_cnt = o;   o = align256(o + sizeof(int32_t) * (size_t)ekv_combine_counters(L, B));
+  c.off_wfirst = o; o = align256(o + sizeof(int32_t) * ((size_t)L->sm_count / 2 + 2));
   c.total = o;
   return c;
 }
@@ -104,14 +114,21 @@ extern "C" int elitekv_decode(const elitekv_layer* L, const elitekv_cache* cache
   ws.slice_out = (float*)(base + cw.off_slice);
   ws.counters = (int32_t*)(base + cw.off_cnt);
   ws.n_counters = ekv_combine_counters(L, B);
+  ws.worker_first = (int32_t*)(base + cw.off_wfirst);
+  ws.n_workers = kernel == 3 ? ekv_tc2_workers(L) : 0;
   cudaStream_t st = (cudaStream_t)stream;
-  rc = ekv_launch_plan(seq_lens, B, kernel == 2 ? 128 : ELITEKV_TILE_TOKENS, max_items, ws.items,
-                       ws.seq_first, ws.counters, ws.n_counters, st);
+  if (kernel == 3)
+    rc = ekv_launch_plan_balanced(seq_lens, B, 32, ws.n_workers, max_items, ws.items, ws.seq_first,
+                                  ws.worker_first, ws.counters, ws.n_counters, st);
+  else
+    rc = ekv_launch_plan(seq_lens, B, kernel == 2 ? 128 : ELITEKV_TILE_TOKENS, max_items, ws.items,
+                         ws.seq_first, ws.counters, ws.n_counters, st);
   if (rc != ELITEKV_OK) return rc;
   EkvProfile* prof = (L->prof && L->prof->enabled && L->prof->count < kProfileSlots) ? L->prof : nullptr;
   if (prof) EKV_CUDA_OK(cudaEventRecord(prof->ev[2 * prof->count], st));
-  rc = kernel == 2 ? ekv_launch_decode_tc(L, cache, cv, q_rope, q_abs, B, ws, st)
-                   : ekv_launch_decode_generic(L, cache, cv, q_rope, q_abs, B, ws, st);
+  rc = kernel == 3   ? ekv_launch_decode_tc2(L, cache, cv, q_rope, q_abs, B, ws, st)
+       : kernel == 2 ? ekv_launch_decode_tc(L, cache, cv, q_rope, q_abs, B, ws, st)
+                     : ekv_launch_decode_generic(L, cache, cv, q_rope, q_abs, B, ws, st);
   if (rc != ELITEKV_OK) return rc;
   if (prof) {
     EKV_CUDA_OK(cudaEventRecord(prof->ev[2 * prof->count + 1], st));

@@ -121,6 +121,10 @@ int ekv_launch_absorb(const elitekv_layer* L, const void* q, const int32_t* q_po
 int ekv_launch_plan(const int32_t* seq_lens, int B, int tile_tokens, int max_items, int32_t* items,
                     int32_t* seq_first_item, int32_t* zero_ints, int n_zero, cudaStream_t st);
 
+int ekv_launch_plan_balanced(const int32_t* seq_lens, int B, int tile_tokens, int n_workers,
+                             int max_items, int32_t* items, int32_t* seq_first_item,
+                             int32_t* worker_first, int32_t* zero_ints, int n_zero, cudaStream_t st);
+
 struct DecodeScratch {
   int max_items;          // capacity of the plan
   int32_t* items;         // [max_items][4]
@@ -130,6 +134,8 @@ struct DecodeScratch {
   float* slice_out;       // combine: per latent slice partial outputs [d_c/128][B][n_h][128]
   int32_t* counters;      // combine: arrival counters, zeroed by the plan kernel
   int n_counters;
+  int32_t* worker_first;  // balanced plan: [n_workers+1] first item of each worker
+  int n_workers;
 };
 
 int ekv_combine_fast_ok(const elitekv_layer* L);
@@ -146,5 +152,11 @@ int ekv_tc_max_items(const elitekv_layer* L, int B);
 int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, const CacheView& cv,
                          const void* q_rope, const void* q_abs, int B, const DecodeScratch& ws,
                          cudaStream_t st);
+int ekv_tc2_supported(const elitekv_layer* L, const elitekv_cache* cache);  // cache may be null
+int ekv_tc2_workers(const elitekv_layer* L);
+int ekv_tc2_max_items(const elitekv_layer* L, int B);
+int ekv_launch_decode_tc2(const elitekv_layer* L, const elitekv_cache* cache, const CacheView& cv,
+                          const void* q_rope, const void* q_abs, int B, const DecodeScratch& ws,
+                          cudaStream_t st);
 int ekv_launch_combine(const elitekv_layer* L, int B, const DecodeScratch& ws, void* out,
                        cudaStream_t st);

@@ -36,7 +36,7 @@ extern "C" int elitekv_layer_create(const elitekv_params* p, elitekv_layer** out
   if (!p->W_uv || (p->d_h - 2 * p->r > 0 && !p->W_uk)) return ELITEKV_ERR_INVALID_ARG;
   if (p->max_pos <= 0 || !(p->rope_base > 0.f)) return ELITEKV_ERR_INVALID_ARG;
   if (p->pair_mode != 0 && p->pair_mode != 1) return ELITEKV_ERR_INVALID_ARG;
-  if (p->decode_kernel < 0 || p->decode_kernel > 2) return ELITEKV_ERR_INVALID_ARG;
+  if (p->decode_kernel < 0 || p->decode_kernel > 3) return ELITEKV_ERR_INVALID_ARG;
   if (p->d_c % 8 != 0 || p->d_h > 512) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
   if (((uintptr_t)p->W_uv & 15) || ((uintptr_t)p->W_uk & 15)) return ELITEKV_ERR_INVALID_ARG;
   const int n_h = p->n_h, d_h = p->d_h, r = p->r, half = d_h / 2;

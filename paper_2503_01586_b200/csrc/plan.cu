@@ -86,7 +86,91 @@ plan_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int max_items
   for (int it = carry + t; it < max_items; it += blockDim.x) *(int4*)(items + 4 * it) = make_int4(-1, 0, 0, 0);
 }
 
+// Balanced plan for kernels whose blocks walk several items: worker w of `n_workers` owns the
+// global tile range [w*quota, (w+1)*quota), quota = ceil(total / n_workers); an item is the
+// intersection of one worker's range with one sequence.  Items come out in global order, so they
+// are grouped by sequence (seq_first) and by worker (worker_first).  items[i] = (sequence, first
+// token, token count, worker).
+__global__ void __launch_bounds__(kPlanThreads)
+plan_balanced_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int n_workers,
+                     int max_items, int32_t* __restrict__ items, int32_t* __restrict__ seq_first,
+                     int32_t* __restrict__ worker_first, int32_t* __restrict__ zero_ints, int n_zero) {
+  __shared__ int warp_tot[kPlanThreads / 32];
+  __shared__ long long s_total;
+  const int t = threadIdx.x;
+  for (int i = t; i < n_zero; i += blockDim.x) zero_ints[i] = 0;
+  if (t == 0) s_total = 0;
+  __syncthreads();
+  long long local = 0;
+  for (int b = t; b < B; b += blockDim.x) {
+    int n = seq_lens[b];
+    local += n > 0 ? (n + tile - 1) / tile : 0;
+  }
+  if (local) atomicAdd((unsigned long long*)&s_total, (unsigned long long)local);
+  __syncthreads();
+  const long long total = s_total;
+  long long quota = (total + n_workers - 1) / n_workers;
+  if (quota < 1) quota = 1;
+
+  // pass 1: count items to know n_items (default of worker_first)
+  int carry_tiles = 0, carry_items = 0;
+  // per-thread record of its sequences is recomputed in pass 2; B is small compared to the block
+  for (int pass = 0; pass < 2; ++pass) {
+    carry_tiles = 0;
+    carry_items = 0;
+    for (int b0 = 0; b0 < B; b0 += blockDim.x) {
+      const int b = b0 + t;
+      int n = 0, tiles = 0;
+      if (b < B) {
+        n = seq_lens[b];
+        tiles = n > 0 ? (n + tile - 1) / tile : 0;
+      }
+      int chunk_tiles;
+      const int g0 = carry_tiles + block_exclusive_scan(tiles, warp_tot, &chunk_tiles);
+      int pieces = 0, w0 = 0;
+      if (tiles > 0) {
+        w0 = (int)(g0 / quota);
+        const int w1 = (int)((g0 + tiles - 1) / quota);
+        pieces = w1 - w0 + 1;
+      }
+      int chunk_items;
+      const int first = carry_items + block_exclusive_scan(pieces, warp_tot, &chunk_items);
+      if (pass == 1 && b < B) {
+        seq_first[b] = first;
+        for (int j = 0; j < pieces; ++j) {
+          const long long ga = max((long long)g0, (w0 + j) * quota);
+          const long long gb = min((long long)g0 + tiles, (w0 + j + 1) * quota);
+          const int tok0 = (int)(ga - g0) * tile;
+          const int tok1 = min((int)(gb - g0) * tile, n);
+          const int it = first + j;
+          if (it < max_items) {
+            *(int4*)(items + 4 * it) = make_int4(b, tok0, tok1 - tok0, w0 + j);
+            if (ga == (w0 + j) * quota) worker_first[w0 + j] = it;
+          }
+        }
+      }
+      carry_tiles += chunk_tiles;
+      carry_items += chunk_items;
+    }
+    if (pass == 0) {
+      for (int w = t; w <= n_workers; w += blockDim.x) worker_first[w] = carry_items;
+      __syncthreads();
+    }
+  }
+  if (t == 0) seq_first[B] = carry_items;
+  for (int it = carry_items + t; it < max_items; it += blockDim.x) *(int4*)(items + 4 * it) = make_int4(-1, 0, 0, 0);
+}
+
 }  // namespace
+
+int ekv_launch_plan_balanced(const int32_t* seq_lens, int B, int tile_tokens, int n_workers,
+                             int max_items, int32_t* items, int32_t* seq_first_item,
+                             int32_t* worker_first, int32_t* zero_ints, int n_zero, cudaStream_t st) {
+  plan_balanced_kernel<<<1, kPlanThreads, 0, st>>>(seq_lens, B, tile_tokens, n_workers, max_items, items,
+                                                   seq_first_item, worker_first, zero_ints, n_zero);
+  EKV_CUDA_OK(cudaGetLastError());
+  return ELITEKV_OK;
+}
 
 int ekv_launch_plan(const int32_t* seq_lens, int B, int tile_tokens, int max_items, int32_t* items,
                     int32_t* seq_first_item, int32_t* zero_ints, int n_zero, cudaStream_t st) {

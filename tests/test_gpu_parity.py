@@ -199,7 +199,7 @@ def test_decode_7b_shape_small_context(ek):
     H.check_parity(st, out, H.all_units(st))
 
 
-@pytest.mark.parametrize("kernel", [1, 2], ids=["generic", "tensor-core"])
+@pytest.mark.parametrize("kernel", [1, 2, 3], ids=["generic", "tensor-core", "tensor-core-pair"])
 def test_decode_7b_shape_ragged_tails_both_kernels(ek, kernel):
     """Same inputs through the CUDA-core kernel and the tcgen05 kernel: lengths around the
     16-token MMA step and the 128-token tile."""
@@ -209,10 +209,28 @@ def test_decode_7b_shape_ragged_tails_both_kernels(ek, kernel):
     H.check_parity(st, out, H.all_units(st))
 
 
+@pytest.mark.parametrize("kernel", [2, 3], ids=["tensor-core", "tensor-core-pair"])
 @pytest.mark.parametrize("page_size", [64, 128])
-def test_decode_7b_shape_paged_tensor_core(ek, page_size):
+def test_decode_7b_shape_paged_tensor_core(ek, page_size, kernel):
     w = replace(gen.shrink(gen.LLAMA7B_75, B=3, ctx=700), paged=True, page_size=page_size)
-    st = H.setup(w, lens=[700, 64, 193], decode_kernel=2)
+    st = H.setup(w, lens=[700, 64, 193], decode_kernel=kernel)
+    out = H.run_decode(st)
+    H.check_parity(st, out, H.all_units(st))
+
+
+def test_pair_kernel_many_items_per_worker(ek):
+    """More sequences than workers can split evenly: workers walk several items, some of them
+    a few tiles long, and sequences are cut at arbitrary 32-token boundaries."""
+    w = gen.shrink(gen.LLAMA7B_75, B=40, ctx=300)
+    lens = [1 + (37 * i) % 300 for i in range(40)]
+    st = H.setup(w, lens=lens, decode_kernel=3)
+    out = H.run_decode(st)
+    H.check_parity(st, out, H.sample_units(st, 96))
+
+
+def test_pair_kernel_87_5pct_shape(ek):
+    w = gen.shrink(gen.SWEEP_875, B=3, ctx=500)
+    st = H.setup(w, lens=[500, 33, 160], decode_kernel=3)
     out = H.run_decode(st)
     H.check_parity(st, out, H.all_units(st))
 

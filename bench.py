@@ -191,14 +191,15 @@ def run_reference(args, w: gen.Workload):
 # ---------------------------------------------------------------------------------------------
 # GPU leg
 # ---------------------------------------------------------------------------------------------
-def build_workload(w: gen.Workload, ek, device):
+def build_workload(w: gen.Workload, ek, device, decode_kernel: int = 0):
     """Cache prefilled with len-1 tokens per sequence; the step appends the last one."""
     idx = gen.elite_index_sets(w)
     W_uk, W_uv = gen.up_projections(w, device)
     lens = gen.sequence_lengths(w)                       # tokens INCLUDING the decoded one
     B = w.B
     max_pos = int(lens.max()) + 1
-    layer = ek.Layer(w.n_h, w.d_h, w.r, w.d_c, idx, W_uk, W_uv, max_pos, rope_base=w.rope_base)
+    layer = ek.Layer(w.n_h, w.d_h, w.r, w.d_c, idx, W_uk, W_uv, max_pos, rope_base=w.rope_base,
+                     decode_kernel=decode_kernel)
     rope_w = w.n_h * 2 * w.r
     page_table = None
     if w.paged:
@@ -267,7 +268,7 @@ def run_gpu(args, w: gen.Workload):
         dist = dist_mod
 
     w_rank = gen.replace(w, seed=w.seed + 100 * rank) if rank else w
-    layer, cache, lens, host, dev, ws, bufs, keep = build_workload(w_rank, ek, device)
+    layer, cache, lens, host, dev, ws, bufs, keep = build_workload(w_rank, ek, device, args.kernel)
     total_tokens = int(lens.sum())
     bytes_per_token = 2 * w.cache_elems_per_token
     cache_bytes = total_tokens * bytes_per_token
@@ -435,6 +436,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=gen.LLAMA7B_75.name, choices=sorted(gen.CONFIGS))
+    ap.add_argument("--kernel", type=int, default=0,
+                    help="split-K kernel: 0 auto, 1 CUDA-core, 2 tcgen05 single block, 3 tcgen05 pair")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-comparator", action="store_true")
     args = ap.parse_args()

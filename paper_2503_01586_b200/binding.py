@@ -13,7 +13,7 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libelitekv.so")
+LIB_PATH = os.environ.get("ELITEKV_LIB", os.path.join(_HERE, "libelitekv.so"))
 
 OK = 0
 ERR_INVALID_ARG = -1

@@ -104,6 +104,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   volatile int* s_abort = (volatile int*)(s_tmem + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  EKV_STAMP_DECL;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < kLatSlots; ++i) {
@@ -175,6 +176,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
           if (!mbar_wait(smem_u32(&bars->lat_empty[slot]), ((lat_n / kLatSlots) & 1) ^ 1, s_abort)) return false;
           const uint32_t fb = smem_u32(&bars->lat_full[slot]);
           mbar_expect_tx(fb, (uint32_t)(halves * 8192));
+          EKV_STAMP(0, 100 + kc, tile);
           for (int hf = 0; hf < halves; ++hf)
             tma_load_2d(smem_u32(s_lat + slot * kChunkBytes + hf * 8192), &map_lat, kc * 64, (int)row[hf], fb);
           ++lat_n;
@@ -248,12 +250,16 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         ++lat_n;
       }
       if (!ok) break;
-      if (lane == 0) tc_commit(smem_u32(&bars->s_full));
+      if (lane == 0) {
+        tc_commit(smem_u32(&bars->s_full));
+        EKV_STAMP(1, 20, tile);
+      }
       __syncwarp();
       // ---- wait for P (and the rescaled output) of this tile
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_ready), tile & 1, s_abort));
       if (!ok) break;
       tc_fence_after();
+      if (lane == 0) EKV_STAMP(1, 21, tile);
       // ---- pass B
       const int ksteps = (nvalid + 15) >> 4;
       const int zero_from = nvalid, zero_to = ksteps * 16;
@@ -288,7 +294,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         lat_n += 2;
       }
       if (!ok) break;
-      if (lane == 0) tc_commit(smem_u32(&bars->pv_done));
+      if (lane == 0) {
+        tc_commit(smem_u32(&bars->pv_done));
+        EKV_STAMP(1, 22, tile);
+      }
       __syncwarp();
     }
   }
@@ -344,10 +353,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         ++rope_n;
       }
       if (!ok) break;
+      if (threadIdx.x == 64) EKV_STAMP(2, 30, tile);
       // ---- latent part from TMEM
       ok = mbar_wait(smem_u32(&bars->s_full), tile & 1, s_abort);
       if (!ok) break;
       tc_fence_after();
+      if (threadIdx.x == 64) EKV_STAMP(2, 31, tile);
       {
         float sv[32];
         tc_ld32(tmem_s + lane_base, sv);
@@ -415,6 +426,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       fence_proxy_async();
       tc_fence_before();
       mbar_arrive(smem_u32(&bars->p_ready));
+      if (threadIdx.x == 64) EKV_STAMP(2, 41, tile);
     }
 
     // ---- epilogue: partial output and softmax statistics of this item
@@ -511,3 +523,14 @@ int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, con
     default: return launch(decode_tc_kernel<32, 32>);
   }
 }
+
+#ifdef EKV_TIMELINE
+extern "C" int elitekv_debug_timeline(unsigned long long* host_out, int max_words, int reset) {
+  void* p = nullptr;
+  if (cudaGetSymbolAddress(&p, g_ekv_timeline) != cudaSuccess) return ELITEKV_ERR_CUDA;
+  if (host_out && cudaMemcpy(host_out, p, sizeof(unsigned long long) * (size_t)max_words, cudaMemcpyDeviceToHost) != cudaSuccess)
+    return ELITEKV_ERR_CUDA;
+  if (reset && cudaMemset(p, 0, sizeof(unsigned long long) * 3 * 8192) != cudaSuccess) return ELITEKV_ERR_CUDA;
+  return ELITEKV_OK;
+}
+#endif

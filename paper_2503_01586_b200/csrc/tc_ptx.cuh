@@ -9,6 +9,26 @@
 
 constexpr unsigned kWaitLimit = 1u << 20;   // polls of mbarrier.try_wait before giving up
 
+// Optional in-kernel event timeline (compiled in with -DEKV_TIMELINE): four roles of block 0
+// append (event code, tile, nanosecond timer) records; elitekv_debug_timeline copies them out.
+#ifdef EKV_TIMELINE
+__device__ unsigned long long g_ekv_timeline[3 * 8192];
+__device__ __forceinline__ void ekv_stamp(int role, unsigned& idx, int code, int tile) {
+  if (blockIdx.x != 0 || idx >= 2048) return;
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  const unsigned i = role * 2048 + idx++;
+  g_ekv_timeline[3 * i] = (unsigned long long)code;
+  g_ekv_timeline[3 * i + 1] = (unsigned long long)tile;
+  g_ekv_timeline[3 * i + 2] = t;
+}
+#define EKV_STAMP_DECL unsigned ekv_stamp_idx = 0
+#define EKV_STAMP(role, code, tile) ekv_stamp(role, ekv_stamp_idx, code, tile)
+#else
+#define EKV_STAMP_DECL
+#define EKV_STAMP(role, code, tile) ((void)0)
+#endif
+
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);

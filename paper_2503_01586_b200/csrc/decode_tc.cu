@@ -199,25 +199,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
           if (ok) ok = load_lat(kc);
         }
         while (cb < NRB && ok) ok = load_rope(cb++);
-        // while pass B re-reads this tile from L2, pull the next tile from HBM into L2
-        if (tile + 1 < n_tiles) {
-          const int t_next = t_abs + kTile;
-          const int nv_next = min(kTile, ntok - (tile + 1) * kTile);
-          for (int hf = 0; hf < (nv_next > 64 ? 2 : 1); ++hf) {
-            const int t = t_next + 64 * hf;
-            long long prow;
-            if (a.page_table == nullptr) {
-              prow = (long long)seq * a.max_ctx + t;
-            } else {
-              const int pi = t >> a.page_shift;
-              const int page = pi < a.max_pages_per_seq ? a.page_table[(long long)seq * a.max_pages_per_seq + pi] : -1;
-              if (page < 0 || page >= a.num_pages) continue;
-              prow = ((long long)page << a.page_shift) + (t & a.page_mask);
-            }
-            for (int b = 0; b < NRB; ++b) tma_prefetch_2d(&map_rope, b * 64, (int)prow);
-            for (int kc = 0; kc < NKC; ++kc) tma_prefetch_2d(&map_lat, kc * 64, (int)prow);
-          }
-        }
         // pass B: the same latent chunks again (served by L2)
         for (int kc = 0; kc < NKC && ok; ++kc) ok = load_lat(kc);
       }

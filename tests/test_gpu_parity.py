@@ -245,6 +245,24 @@ def test_tensor_core_kernel_refuses_uncovered_shapes(ek):
     assert e.value.code == ek.ERR_UNSUPPORTED_SHAPE
 
 
+def test_decode_only_parity_from_the_gpu_cache(ek):
+    """Decode in isolation: the oracle reads the rope rows the GPU appended (bf16, downloaded)
+    instead of rotating the raw keys itself, so append rounding cannot mask a decode error."""
+    w = gen.shrink(gen.LLAMA7B_75, B=2, ctx=300)
+    lens = [300, 131]
+    st = H.setup(w, lens=lens)
+    out = H.f64(H.run_decode(st))
+    W_uk, W_uv, idx = H.f64(st.W_uk), H.f64(st.W_uv), st.idx.numpy().astype(np.int64)
+    max_ctx = st.cache.max_ctx
+    for b, n in enumerate(lens):
+        rows = slice(b * max_ctx, b * max_ctx + n)
+        k_rope = H.f64(st.rope_plane[rows]).reshape(n, w.n_h, 2 * w.r)
+        c = H.f64(st.latent_plane[rows])
+        want = O.decode(H.f64(st.q[b]), n - 1, k_rope, c, W_uk, W_uv, idx, w.d_h, base=w.rope_base)
+        rel, mx = H.errors(out[b], want)
+        assert rel <= H.REL_L2_TOL and mx <= H.MAX_ABS_TOL, (b, rel, mx)
+
+
 def test_decode_13b_shape_small_context(ek):
     w = gen.shrink(gen.LLAMA13B_75, B=2, ctx=300)
     st = H.setup(w, lens=[300, 129])

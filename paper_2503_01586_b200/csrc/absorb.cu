@@ -4,18 +4,19 @@
 //   q_rope[b,h,2j:2j+2] = q[b,h,chunk idx[h][j]] . R(q_pos[b] * theta_idx[h][j])
 //   q_abs [b,h,k]       = sum_i q_nope[b,h,i] * W_uk[k][h*dn + i]
 //
-// Grid (n_h, ceil(d_c/128)): a block owns one head and 128 latent coordinates.  Its 256 threads
-// are 64 coordinate pairs x 4 groups over the head's un-rotated dims; every thread keeps one fp32
+// Grid (n_h, ceil(d_c/128)): a block owns one head and 128 latent coordinates.  Its 512 threads
+// are 64 coordinate pairs x 8 groups over the head's un-rotated dims; every thread keeps one fp32
 // accumulator pair per sequence of the current chunk of 16 sequences, so each weight element is
-// read once per chunk, and the four groups are added through shared memory.  The weights come
+// read once per chunk, and the eight groups are added through shared memory.  The weights come
 // regrouped as [n_h][dn][d_c] (d_c contiguous), which makes the reads coalesced.
 #include "common.cuh"
 
 namespace {
 
 constexpr int kAbsorbBatch = 16;
-constexpr int kAbsorbThreads = 256;
-constexpr int kAbsorbGroups = 4;
+constexpr int kAbsorbThreads = 512;
+constexpr int kAbsorbGroups = 8;
+constexpr int kAbsorbMaxPer = 16;   // un-rotated dims per group held in registers
 constexpr int kAbsorbCoords = 128;
 
 __global__ void __launch_bounds__(kAbsorbThreads)
@@ -28,7 +29,7 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
   const int h = blockIdx.x;
   const int dn = d_h - 2 * r;
   float* q_nope = smem_f;                                   // [dn][16] (sequence fastest)
-  float* red = smem_f + (size_t)(dn > 0 ? dn : 1) * kAbsorbBatch;   // [3][16][128]
+  float* red = smem_f + (size_t)(dn > 0 ? dn : 1) * kAbsorbBatch;   // [7][16][128]
   const int pair = threadIdx.x & 63, grp = threadIdx.x >> 6;
   const int k = blockIdx.y * kAbsorbCoords + 2 * pair;
   const int32_t* dims = qdims + (size_t)h * d_h;
@@ -52,7 +53,7 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
     }
   }
 
-  const int per_grp = (dn + kAbsorbGroups - 1) / kAbsorbGroups;
+  const int per_grp = (dn + kAbsorbGroups - 1) / kAbsorbGroups;   // <= kAbsorbMaxPer (d_h <= 128), checked by the launcher
   const int i_lo = min(dn, grp * per_grp), i_hi = min(dn, i_lo + per_grp);
   for (int b0 = 0; b0 < B; b0 += kAbsorbBatch) {
     const int nb = min(kAbsorbBatch, B - b0);
@@ -67,9 +68,15 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
     for (int bb = 0; bb < kAbsorbBatch; ++bb) a0[bb] = a1[bb] = 0.f;
     if (k < d_c) {
       const bf16* wp = WukT + (size_t)h * dn * d_c + k;
-#pragma unroll 4
-      for (int i = i_lo; i < i_hi; ++i) {
-        const float2 w = __bfloat1622float2(*(const bf162*)(wp + (size_t)i * d_c));
+      // all weights of this thread's slice first (independent loads), then the arithmetic
+      bf162 wreg[kAbsorbMaxPer];
+#pragma unroll
+      for (int j = 0; j < kAbsorbMaxPer; ++j)
+        wreg[j] = (i_lo + j < i_hi) ? __ldg((const bf162*)(wp + (size_t)(i_lo + j) * d_c)) : __floats2bfloat162_rn(0.f, 0.f);
+#pragma unroll
+      for (int j = 0; j < kAbsorbMaxPer; ++j) {
+        const int i = max(0, min(i_lo + j, dn - 1));
+        const float2 w = __bfloat1622float2(wreg[j]);
         const float4* xr = (const float4*)(q_nope + (size_t)i * kAbsorbBatch);
 #pragma unroll
         for (int v = 0; v < kAbsorbBatch / 4; ++v) {
@@ -111,6 +118,7 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
 int ekv_launch_absorb(const elitekv_layer* L, const void* q, const int32_t* q_pos, int B,
                       void* q_rope, void* q_abs, cudaStream_t st) {
   if (B == 0) return ELITEKV_OK;
+  if ((L->dn + kAbsorbGroups - 1) / kAbsorbGroups > kAbsorbMaxPer) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
   dim3 grid(L->n_h, (L->d_c + kAbsorbCoords - 1) / kAbsorbCoords);
   size_t smem = sizeof(float) * (kAbsorbBatch * (size_t)(L->dn > 0 ? L->dn : 1) +
                                  (size_t)(kAbsorbGroups - 1) * kAbsorbBatch * kAbsorbCoords);

@@ -23,6 +23,7 @@ constexpr int kFB = 16;          // sequences per group
 constexpr int kFK = 128;         // latent slice
 constexpr int kFD = 128;         // head dim
 constexpr int kFThreads = 256;
+constexpr int kFI = 16;          // items per sequence whose merge weights are staged in shared memory
 
 __global__ void __launch_bounds__(kFThreads)
 combine_fast_kernel(const float* __restrict__ part_acc, const float* __restrict__ part_ml,
@@ -33,6 +34,7 @@ combine_fast_kernel(const float* __restrict__ part_acc, const float* __restrict_
   __shared__ __align__(16) bf16 s_w[kFK][kFD];          // 32 KB
   __shared__ __align__(16) float s_x[kFB][kFK];         // 8 KB merged latent outputs
   __shared__ float s_M[kFB], s_invL[kFB];
+  __shared__ float s_wt[kFB][kFI];
   __shared__ int s_first[kFB + 1];
   __shared__ int s_last;
   const int h = blockIdx.x, slice = blockIdx.y, n_slices = gridDim.y;
@@ -70,20 +72,39 @@ combine_fast_kernel(const float* __restrict__ part_acc, const float* __restrict_
       }
     }
     __syncthreads();
-    // merge the items of each sequence on this latent slice
+    // normalised merge weights 2^(m_s - M) / L of the first kFI items of every sequence
+    for (int e = tid; e < kFB * kFI; e += kFThreads) {
+      const int bb = e / kFI, j = e % kFI;
+      float wv = 0.f;
+      if (bb < nb) {
+        const int i = s_first[bb] + j;
+        if (i < s_first[bb + 1]) wv = exp2f(part_ml[((size_t)i * n_h + h) * 2] - s_M[bb]) * s_invL[bb];
+      }
+      s_wt[bb][j] = wv;
+    }
+    __syncthreads();
+    // merge the items of each sequence on this latent slice (independent 16-byte loads)
     for (int e = tid; e < kFB * (kFK / 4); e += kFThreads) {
       const int bb = e / (kFK / 4), v = e % (kFK / 4);
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
       if (bb < nb) {
-        const float M = s_M[bb];
-        for (int i = s_first[bb]; i < s_first[bb + 1]; ++i) {
-          const float w = exp2f(part_ml[((size_t)i * n_h + h) * 2] - M);
-          const float4 p = __ldg((const float4*)(part_acc + ((size_t)i * n_h + h) * d_c + k0 + v * 4));
+        const int i0 = s_first[bb], ni = s_first[bb + 1] - i0;
+        const float* src = part_acc + ((size_t)i0 * n_h + h) * d_c + k0 + v * 4;
+        const size_t stride = (size_t)n_h * d_c;
+        const int nfast = min(ni, kFI);
+#pragma unroll 4
+        for (int j = 0; j < nfast; ++j) {
+          const float w = s_wt[bb][j];
+          const float4 p = __ldg((const float4*)(src + (size_t)j * stride));
           acc.x = fmaf(w, p.x, acc.x); acc.y = fmaf(w, p.y, acc.y);
           acc.z = fmaf(w, p.z, acc.z); acc.w = fmaf(w, p.w, acc.w);
         }
-        const float il = s_invL[bb];
-        acc.x *= il; acc.y *= il; acc.z *= il; acc.w *= il;
+        for (int j = kFI; j < ni; ++j) {     // rare: a sequence cut into more than kFI items
+          const float w = exp2f(part_ml[((size_t)(i0 + j) * n_h + h) * 2] - s_M[bb]) * s_invL[bb];
+          const float4 p = __ldg((const float4*)(src + (size_t)j * stride));
+          acc.x = fmaf(w, p.x, acc.x); acc.y = fmaf(w, p.y, acc.y);
+          acc.z = fmaf(w, p.z, acc.z); acc.w = fmaf(w, p.w, acc.w);
+        }
       }
       *(float4*)&s_x[bb][v * 4] = acc;
     }

@@ -1,6 +1,13 @@
 // C entry points: argument checks, workspace carving, kernel selection.
 #include "common.cuh"
 
+// Diagnostic build (-DEKV_SYNC_EACH): synchronise after every launch and report which stage failed.
+#ifdef EKV_SYNC_EACH
+#define EKV_STAGE_CHECK(st, stage) do { if (cudaStreamSynchronize(st) != cudaSuccess) return -100 - (stage); } while (0)
+#else
+#define EKV_STAGE_CHECK(st, stage) do { } while (0)
+#endif
+
 namespace {
 
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -70,7 +77,9 @@ extern "C" int elitekv_append(const elitekv_layer* L, const elitekv_cache* cache
   CacheView cv;
   int rc = ekv_make_view(cache, &cv);
   if (rc != ELITEKV_OK) return rc;
-  return ekv_launch_append(L, cache, cv, k_e, c, seq_id, pos, T, (cudaStream_t)stream);
+  rc = ekv_launch_append(L, cache, cv, k_e, c, seq_id, pos, T, (cudaStream_t)stream);
+  EKV_STAGE_CHECK((cudaStream_t)stream, 1);
+  return rc;
 }
 
 extern "C" int elitekv_absorb_query(const elitekv_layer* L, const void* q, const int32_t* q_pos,
@@ -78,7 +87,9 @@ extern "C" int elitekv_absorb_query(const elitekv_layer* L, const void* q, const
   if (!L || !q || !q_pos || !q_abs || B < 0 || (L->r > 0 && !q_rope)) return ELITEKV_ERR_INVALID_ARG;
   if (((uintptr_t)q & 15) || ((uintptr_t)q_abs & 15) || ((uintptr_t)q_rope & 3))
     return ELITEKV_ERR_INVALID_ARG;
-  return ekv_launch_absorb(L, q, q_pos, B, q_rope, q_abs, (cudaStream_t)stream);
+  int rc = ekv_launch_absorb(L, q, q_pos, B, q_rope, q_abs, (cudaStream_t)stream);
+  EKV_STAGE_CHECK((cudaStream_t)stream, 2);
+  return rc;
 }
 
 extern "C" int elitekv_decode_workspace_size(const elitekv_layer* L, int32_t B, size_t* bytes) {
@@ -125,6 +136,7 @@ extern "C" int elitekv_decode(const elitekv_layer* L, const elitekv_cache* cache
     rc = ekv_launch_plan(seq_lens, B, kernel == 2 ? 128 : ELITEKV_TILE_TOKENS, max_items, ws.items,
                          ws.seq_first, ws.counters, ws.n_counters, st);
   if (rc != ELITEKV_OK) return rc;
+  EKV_STAGE_CHECK(st, 3);
   EkvProfile* prof = (L->prof && L->prof->enabled && L->prof->count < kProfileSlots) ? L->prof : nullptr;
   if (prof) EKV_CUDA_OK(cudaEventRecord(prof->ev[2 * prof->count], st));
   rc = kernel == 3   ? ekv_launch_decode_tc2(L, cache, cv, q_rope, q_abs, B, ws, st)
@@ -135,5 +147,8 @@ extern "C" int elitekv_decode(const elitekv_layer* L, const elitekv_cache* cache
     EKV_CUDA_OK(cudaEventRecord(prof->ev[2 * prof->count + 1], st));
     prof->count++;
   }
-  return ekv_launch_combine(L, B, ws, out, st);
+  EKV_STAGE_CHECK(st, 4);
+  rc = ekv_launch_combine(L, B, ws, out, st);
+  EKV_STAGE_CHECK(st, 5);
+  return rc;
 }

@@ -13,6 +13,15 @@
 
 namespace {
 
+#ifdef EKV_SYNC_EACH
+struct AbsorbLimits { long long q, qpos, wuk, qdims, idx, cs, qrope, qabs; };
+__device__ AbsorbLimits g_absorb_lim;
+#define ABS_CHK(site, index, limit) \
+  if ((long long)(index) < 0 || (long long)(index) >= g_absorb_lim.limit) { ekv_record(status, -900 - (site), (int)blockIdx.x, (int)(index)); continue; }
+#else
+#define ABS_CHK(site, index, limit)
+#endif
+
 constexpr int kAbsorbBatch = 16;
 constexpr int kAbsorbThreads = 512;
 constexpr int kAbsorbGroups = 8;
@@ -38,11 +47,18 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
   if (blockIdx.y == 0) {
     for (int e = threadIdx.x; e < B * r; e += blockDim.x) {
       const int b = e / r, j = e % r;
+      ABS_CHK(1, b, qpos)
       int p = q_pos[b];
       if (p < 0 || p >= max_pos) {
         ekv_record(status, ELITEKV_ERR_BAD_POSITION, b, p);
         p = 0;
       }
+      ABS_CHK(2, h * r + j, idx)
+      ABS_CHK(3, (size_t)p * (d_h / 2) + idx[h * r + j], cs)
+      ABS_CHK(4, (size_t)h * d_h + 2 * j + 1, qdims)
+      ABS_CHK(5, ((size_t)b * n_h + h) * d_h + dims[2 * j + 1], q)
+      ABS_CHK(6, ((size_t)b * n_h + h) * d_h + dims[2 * j], q)
+      ABS_CHK(7, ((size_t)b * n_h + h) * 2 * r + 2 * j + 1, qrope)
       const float2 w = cs[(size_t)p * (d_h / 2) + idx[h * r + j]];
       const bf16* qq = q + ((size_t)b * n_h + h) * d_h;
       const float x0 = __bfloat162float(qq[dims[2 * j]]), x1 = __bfloat162float(qq[dims[2 * j + 1]]);
@@ -60,19 +76,27 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
     __syncthreads();
     for (int e = threadIdx.x; e < kAbsorbBatch * dn; e += blockDim.x) {
       const int i = e / kAbsorbBatch, bb = e % kAbsorbBatch;
+      ABS_CHK(8, (size_t)h * d_h + 2 * r + i, qdims)
+      if (bb < nb) { ABS_CHK(9, ((size_t)(b0 + bb) * n_h + h) * d_h + dims[2 * r + i], q) }
       q_nope[e] = bb < nb ? __bfloat162float(q[((size_t)(b0 + bb) * n_h + h) * d_h + dims[2 * r + i]]) : 0.f;
     }
     __syncthreads();
     float a0[kAbsorbBatch], a1[kAbsorbBatch];
 #pragma unroll
     for (int bb = 0; bb < kAbsorbBatch; ++bb) a0[bb] = a1[bb] = 0.f;
-    if (k < d_c) {
+    if (k < d_c && dn > 0) {
       const bf16* wp = WukT + (size_t)h * dn * d_c + k;
       // all weights of this thread's slice first (independent loads), then the arithmetic
       bf162 wreg[kAbsorbMaxPer];
 #pragma unroll
-      for (int j = 0; j < kAbsorbMaxPer; ++j)
-        wreg[j] = (i_lo + j < i_hi) ? __ldg((const bf162*)(wp + (size_t)(i_lo + j) * d_c)) : __floats2bfloat162_rn(0.f, 0.f);
+      for (int j = 0; j < kAbsorbMaxPer; ++j) {
+        // always a valid address (clamped into the head's rows); slots past the group's range
+        // are zeroed after the load instead of predicating the load itself
+        const int ii = max(0, min(i_lo + j, dn - 1));
+        ABS_CHK(10, (size_t)h * dn * d_c + k + (size_t)ii * d_c + 1, wuk)
+        const bf162 wv = __ldg((const bf162*)(wp + (size_t)ii * d_c));
+        wreg[j] = (i_lo + j < i_hi) ? wv : __floats2bfloat162_rn(0.f, 0.f);
+      }
 #pragma unroll
       for (int j = 0; j < kAbsorbMaxPer; ++j) {
         const int i = max(0, min(i_lo + j, dn - 1));
@@ -99,6 +123,7 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
 #pragma unroll
       for (int bb = 0; bb < kAbsorbBatch; ++bb) {
         if (bb < nb) {
+          ABS_CHK(11, ((size_t)(b0 + bb) * n_h + h) * d_c + k + 1, qabs)
           float s0 = a0[bb], s1 = a1[bb];
 #pragma unroll
           for (int g = 0; g < kAbsorbGroups - 1; ++g) {
@@ -123,6 +148,20 @@ int ekv_launch_absorb(const elitekv_layer* L, const void* q, const int32_t* q_po
   size_t smem = sizeof(float) * (kAbsorbBatch * (size_t)(L->dn > 0 ? L->dn : 1) +
                                  (size_t)(kAbsorbGroups - 1) * kAbsorbBatch * kAbsorbCoords);
   EKV_CUDA_OK(cudaFuncSetAttribute(absorb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+#ifdef EKV_SYNC_EACH
+  {
+    AbsorbLimits lim;
+    lim.q = (long long)B * L->n_h * L->d_h;
+    lim.qpos = B;
+    lim.wuk = (long long)L->n_h * L->dn * L->d_c;
+    lim.qdims = (long long)L->n_h * L->d_h;
+    lim.idx = (long long)L->n_h * L->r;
+    lim.cs = (long long)L->max_pos * (L->d_h / 2);
+    lim.qrope = (long long)B * L->n_h * 2 * L->r;
+    lim.qabs = (long long)B * L->n_h * L->d_c;
+    EKV_CUDA_OK(cudaMemcpyToSymbolAsync(g_absorb_lim, &lim, sizeof(lim), 0, cudaMemcpyHostToDevice, st));
+  }
+#endif
   absorb_kernel<<<grid, kAbsorbThreads, smem, st>>>(
       (const bf16*)q, q_pos, B, L->d_WukT, L->d_qdims, L->d_idx, L->d_cs, (bf16*)q_rope,
       (bf16*)q_abs, L->n_h, L->d_h, L->r, L->d_c, L->max_pos, L->d_status);

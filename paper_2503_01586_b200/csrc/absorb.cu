@@ -4,28 +4,18 @@
 //   q_rope[b,h,2j:2j+2] = q[b,h,chunk idx[h][j]] . R(q_pos[b] * theta_idx[h][j])
 //   q_abs [b,h,k]       = sum_i q_nope[b,h,i] * W_uk[k][h*dn + i]
 //
-// Grid (n_h, ceil(d_c/128)): a block owns one head and 128 latent coordinates.  Its 512 threads
-// are 64 coordinate pairs x 8 groups over the head's un-rotated dims; every thread keeps one fp32
+// Grid (n_h, ceil(d_c/128)): a block owns one head and 128 latent coordinates.  Its 256 threads
+// are 64 coordinate pairs x 4 groups over the head's un-rotated dims; every thread keeps one fp32
 // accumulator pair per sequence of the current chunk of 16 sequences, so each weight element is
-// read once per chunk, and the eight groups are added through shared memory.  The weights come
+// read once per chunk, and the four groups are added through shared memory.  The weights come
 // regrouped as [n_h][dn][d_c] (d_c contiguous), which makes the reads coalesced.
 #include "common.cuh"
 
 namespace {
 
-#ifdef EKV_SYNC_EACH
-struct AbsorbLimits { long long q, qpos, wuk, qdims, idx, cs, qrope, qabs; };
-__device__ AbsorbLimits g_absorb_lim;
-#define ABS_CHK(site, index, limit) \
-  if ((long long)(index) < 0 || (long long)(index) >= g_absorb_lim.limit) { ekv_record(status, -900 - (site), (int)blockIdx.x, (int)(index)); continue; }
-#else
-#define ABS_CHK(site, index, limit)
-#endif
-
 constexpr int kAbsorbBatch = 16;
-constexpr int kAbsorbThreads = 512;
-constexpr int kAbsorbGroups = 8;
-constexpr int kAbsorbMaxPer = 16;   // un-rotated dims per group held in registers
+constexpr int kAbsorbThreads = 256;
+constexpr int kAbsorbGroups = 4;
 constexpr int kAbsorbCoords = 128;
 
 __global__ void __launch_bounds__(kAbsorbThreads)
@@ -38,7 +28,7 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
   const int h = blockIdx.x;
   const int dn = d_h - 2 * r;
   float* q_nope = smem_f;                                   // [dn][16] (sequence fastest)
-  float* red = smem_f + (size_t)(dn > 0 ? dn : 1) * kAbsorbBatch;   // [7][16][128]
+  float* red = smem_f + (size_t)(dn > 0 ? dn : 1) * kAbsorbBatch;   // [3][16][128]
   const int pair = threadIdx.x & 63, grp = threadIdx.x >> 6;
   const int k = blockIdx.y * kAbsorbCoords + 2 * pair;
   const int32_t* dims = qdims + (size_t)h * d_h;
@@ -47,18 +37,11 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
   if (blockIdx.y == 0) {
     for (int e = threadIdx.x; e < B * r; e += blockDim.x) {
       const int b = e / r, j = e % r;
-      ABS_CHK(1, b, qpos)
       int p = q_pos[b];
       if (p < 0 || p >= max_pos) {
         ekv_record(status, ELITEKV_ERR_BAD_POSITION, b, p);
         p = 0;
       }
-      ABS_CHK(2, h * r + j, idx)
-      ABS_CHK(3, (size_t)p * (d_h / 2) + idx[h * r + j], cs)
-      ABS_CHK(4, (size_t)h * d_h + 2 * j + 1, qdims)
-      ABS_CHK(5, ((size_t)b * n_h + h) * d_h + dims[2 * j + 1], q)
-      ABS_CHK(6, ((size_t)b * n_h + h) * d_h + dims[2 * j], q)
-      ABS_CHK(7, ((size_t)b * n_h + h) * 2 * r + 2 * j + 1, qrope)
       const float2 w = cs[(size_t)p * (d_h / 2) + idx[h * r + j]];
       const bf16* qq = q + ((size_t)b * n_h + h) * d_h;
       const float x0 = __bfloat162float(qq[dims[2 * j]]), x1 = __bfloat162float(qq[dims[2 * j + 1]]);
@@ -69,38 +52,24 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
     }
   }
 
-  const int per_grp = (dn + kAbsorbGroups - 1) / kAbsorbGroups;   // <= kAbsorbMaxPer (d_h <= 128), checked by the launcher
+  const int per_grp = (dn + kAbsorbGroups - 1) / kAbsorbGroups;
   const int i_lo = min(dn, grp * per_grp), i_hi = min(dn, i_lo + per_grp);
   for (int b0 = 0; b0 < B; b0 += kAbsorbBatch) {
     const int nb = min(kAbsorbBatch, B - b0);
     __syncthreads();
     for (int e = threadIdx.x; e < kAbsorbBatch * dn; e += blockDim.x) {
       const int i = e / kAbsorbBatch, bb = e % kAbsorbBatch;
-      ABS_CHK(8, (size_t)h * d_h + 2 * r + i, qdims)
-      if (bb < nb) { ABS_CHK(9, ((size_t)(b0 + bb) * n_h + h) * d_h + dims[2 * r + i], q) }
       q_nope[e] = bb < nb ? __bfloat162float(q[((size_t)(b0 + bb) * n_h + h) * d_h + dims[2 * r + i]]) : 0.f;
     }
     __syncthreads();
     float a0[kAbsorbBatch], a1[kAbsorbBatch];
 #pragma unroll
     for (int bb = 0; bb < kAbsorbBatch; ++bb) a0[bb] = a1[bb] = 0.f;
-    if (k < d_c && dn > 0) {
+    if (k < d_c) {
       const bf16* wp = WukT + (size_t)h * dn * d_c + k;
-      // all weights of this thread's slice first (independent loads), then the arithmetic
-      bf162 wreg[kAbsorbMaxPer];
-#pragma unroll
-      for (int j = 0; j < kAbsorbMaxPer; ++j) {
-        // always a valid address (clamped into the head's rows); slots past the group's range
-        // are zeroed after the load instead of predicating the load itself
-        const int ii = max(0, min(i_lo + j, dn - 1));
-        ABS_CHK(10, (size_t)h * dn * d_c + k + (size_t)ii * d_c + 1, wuk)
-        const bf162 wv = __ldg((const bf162*)(wp + (size_t)ii * d_c));
-        wreg[j] = (i_lo + j < i_hi) ? wv : __floats2bfloat162_rn(0.f, 0.f);
-      }
-#pragma unroll
-      for (int j = 0; j < kAbsorbMaxPer; ++j) {
-        const int i = max(0, min(i_lo + j, dn - 1));
-        const float2 w = __bfloat1622float2(wreg[j]);
+#pragma unroll 4
+      for (int i = i_lo; i < i_hi; ++i) {
+        const float2 w = __bfloat1622float2(*(const bf162*)(wp + (size_t)i * d_c));
         const float4* xr = (const float4*)(q_nope + (size_t)i * kAbsorbBatch);
 #pragma unroll
         for (int v = 0; v < kAbsorbBatch / 4; ++v) {
@@ -123,7 +92,6 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
 #pragma unroll
       for (int bb = 0; bb < kAbsorbBatch; ++bb) {
         if (bb < nb) {
-          ABS_CHK(11, ((size_t)(b0 + bb) * n_h + h) * d_c + k + 1, qabs)
           float s0 = a0[bb], s1 = a1[bb];
 #pragma unroll
           for (int g = 0; g < kAbsorbGroups - 1; ++g) {
@@ -143,25 +111,10 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
 int ekv_launch_absorb(const elitekv_layer* L, const void* q, const int32_t* q_pos, int B,
                       void* q_rope, void* q_abs, cudaStream_t st) {
   if (B == 0) return ELITEKV_OK;
-  if ((L->dn + kAbsorbGroups - 1) / kAbsorbGroups > kAbsorbMaxPer) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
   dim3 grid(L->n_h, (L->d_c + kAbsorbCoords - 1) / kAbsorbCoords);
   size_t smem = sizeof(float) * (kAbsorbBatch * (size_t)(L->dn > 0 ? L->dn : 1) +
                                  (size_t)(kAbsorbGroups - 1) * kAbsorbBatch * kAbsorbCoords);
   EKV_CUDA_OK(cudaFuncSetAttribute(absorb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-#ifdef EKV_SYNC_EACH
-  {
-    AbsorbLimits lim;
-    lim.q = (long long)B * L->n_h * L->d_h;
-    lim.qpos = B;
-    lim.wuk = (long long)L->n_h * L->dn * L->d_c;
-    lim.qdims = (long long)L->n_h * L->d_h;
-    lim.idx = (long long)L->n_h * L->r;
-    lim.cs = (long long)L->max_pos * (L->d_h / 2);
-    lim.qrope = (long long)B * L->n_h * 2 * L->r;
-    lim.qabs = (long long)B * L->n_h * L->d_c;
-    EKV_CUDA_OK(cudaMemcpyToSymbolAsync(g_absorb_lim, &lim, sizeof(lim), 0, cudaMemcpyHostToDevice, st));
-  }
-#endif
   absorb_kernel<<<grid, kAbsorbThreads, smem, st>>>(
       (const bf16*)q, q_pos, B, L->d_WukT, L->d_qdims, L->d_idx, L->d_cs, (bf16*)q_rope,
       (bf16*)q_abs, L->n_h, L->d_h, L->r, L->d_c, L->max_pos, L->d_status);

@@ -50,6 +50,7 @@ struct TcArgs {
   long long num_pages;
   int page_shift, page_mask, max_pages_per_seq;
   int n_h, d_c;
+  int n_groups;             // head groups of N heads; blockIdx.x = item * n_groups + group
   float scale_log2e;
 };
 
@@ -78,7 +79,9 @@ __global__ void __launch_bounds__(kThreads, 1)
 decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_constant__ CUtensorMap map_rope,
                  const __grid_constant__ CUtensorMap map_q, const TcArgs a) {
   extern __shared__ unsigned char smem_raw[];
-  const int item = blockIdx.x;
+  const int item = blockIdx.x / a.n_groups;
+  const int h0 = (blockIdx.x % a.n_groups) * N;       // first head of this block's group
+  const int nh_here = min(N, a.n_h - h0);
   const int seq = a.items[4 * item + 0];
   if (seq < 0) return;
   const int tok0 = a.items[4 * item + 1];
@@ -126,7 +129,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   // rotated query chunks of this sequence as fp32 (broadcast operand of the rope dot products)
   for (int e = threadIdx.x; e < N * R2; e += kThreads) {
     const int h = e / R2;
-    s_qrope[e] = h < a.n_h ? __bfloat162float(a.q_rope[((size_t)seq * a.n_h + h) * R2 + (e % R2)]) : 0.f;
+    s_qrope[e] = h < nh_here ? __bfloat162float(a.q_rope[((size_t)seq * a.n_h + h0 + h) * R2 + (e % R2)]) : 0.f;
   }
   const int tmem_cols_needed = NB * N + N;
   uint32_t tmem_cols = 32;
@@ -147,7 +150,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       const uint32_t qbar = smem_u32(&bars->q_full);
       mbar_expect_tx(qbar, (uint32_t)(NKC * N * 128));
       for (int kc = 0; kc < NKC; ++kc)
-        tma_load_2d(smem_u32(s_q + kc * N * 128), &map_q, kc * 64, seq * a.n_h, qbar);
+        tma_load_2d(smem_u32(s_q + kc * N * 128), &map_q, kc * 64, seq * a.n_h + h0, qbar);
 
       unsigned lat_n = 0, rope_n = 0;      // chunks issued so far
       bool ok = true;
@@ -188,7 +191,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
           const uint32_t fb = smem_u32(&bars->rope_full[slot]);
           mbar_expect_tx(fb, (uint32_t)(halves * 8192));
           for (int hf = 0; hf < halves; ++hf)
-            tma_load_2d(smem_u32(s_rope + slot * kChunkBytes + hf * 8192), &map_rope, cb * 64, (int)row[hf], fb);
+            tma_load_2d(smem_u32(s_rope + slot * kChunkBytes + hf * 8192), &map_rope, h0 * R2 + cb * 64, (int)row[hf], fb);
           ++rope_n;
           return true;
         };
@@ -293,7 +296,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
     float m_ref = -INFINITY;                      // lane h holds head h's reference max (N <= 32 per group)
     unsigned rope_n = 0;
     bool ok = true;
-    static_assert(N == 32, "softmax threads keep one head per lane");
+    static_assert(N == 16 || N == 32, "softmax threads keep one head per lane (lanes >= N idle)");
 
     for (int tile = 0; tile < n_tiles && ok; ++tile) {
       const int nvalid = min(kTile, ntok - tile * kTile);
@@ -341,8 +344,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       tc_fence_after();
       if (threadIdx.x == 64) EKV_STAMP(2, 31, tile);
       {
-        float sv[32];
-        tc_ld32(tmem_s + lane_base, sv);
+        float sv[N];
+        tc_ld_cols<N>(tmem_s + lane_base, sv);
         tc_wait_ld();
 #pragma unroll
         for (int h = 0; h < N; ++h) {
@@ -357,16 +360,17 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         const float v = ord2f(__reduce_max_sync(0xffffffffu, f2ord(s[h])));
         if (lane == h) wm = v;
       }
-      s_wmax[quarter * N + lane] = wm;
+      if (lane < N) s_wmax[quarter * N + lane] = wm;
       named_bar_sync(1, kSoftmaxThreads);
-      float tm = fmaxf(fmaxf(s_wmax[lane], s_wmax[N + lane]), fmaxf(s_wmax[2 * N + lane], s_wmax[3 * N + lane]));
+      const int hl = lane & (N - 1);
+      float tm = fmaxf(fmaxf(s_wmax[hl], s_wmax[N + hl]), fmaxf(s_wmax[2 * N + hl], s_wmax[3 * N + hl]));
       // reference max moves only when the tile max exceeds it by more than 2^8
       const bool move = tm > m_ref + 8.f;
       const float m_new = move ? tm : m_ref;
       const float corr = move ? exp2f(m_ref - m_new) : 1.f;      // 0 on the first tile
       m_ref = m_new;
       const bool any_move = __any_sync(0xffffffffu, move);       // same in all four warps
-      if (any_move && quarter == 0) s_corr[lane] = corr;
+      if (any_move && quarter == 0 && lane < N) s_corr[lane] = corr;
       // ---- probabilities, partial sums, P tile in the no-swizzle MN-major layout
 #pragma unroll
       for (int j = 0; j < N / 8; ++j) {
@@ -395,12 +399,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       if (any_move && tile > 0) {
         named_bar_sync(1, kSoftmaxThreads);      // s_corr visible
         for (int blk = 0; blk < NB; ++blk) {
-          float v[32];
-          tc_ld32(tmem_base + blk * N + lane_base, v);
+          float v[N];
+          tc_ld_cols<N>(tmem_base + blk * N + lane_base, v);
           tc_wait_ld();
 #pragma unroll
           for (int h = 0; h < N; ++h) v[h] *= s_corr[h];
-          tc_st32(tmem_base + blk * N + lane_base, v);
+          tc_st_cols<N>(tmem_base + blk * N + lane_base, v);
         }
         tc_wait_st();
       }
@@ -414,15 +418,15 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
     if (ok) ok = mbar_wait(smem_u32(&bars->pv_done), (n_tiles - 1) & 1, s_abort);
     if (ok) {
       tc_fence_after();
-      float* pa = a.part_acc + (size_t)item * a.n_h * d_c;
+      float* pa = a.part_acc + ((size_t)item * a.n_h + h0) * d_c;
       for (int blk = 0; blk < NB; ++blk) {
-        float v[32];
-        tc_ld32(tmem_base + blk * N + lane_base, v);
+        float v[N];
+        tc_ld_cols<N>(tmem_base + blk * N + lane_base, v);
         tc_wait_ld();
         const int d = blk * 128 + trow;
 #pragma unroll
         for (int h = 0; h < N; ++h)
-          if (h < a.n_h) pa[(size_t)h * d_c + d] = v[h];
+          if (h < nh_here) pa[(size_t)h * d_c + d] = v[h];
       }
       float wl = 0.f;
 #pragma unroll
@@ -431,12 +435,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         if (lane == h) wl = v;
       }
       named_bar_sync(1, kSoftmaxThreads);
-      s_wmax[quarter * N + lane] = wl;
+      if (lane < N) s_wmax[quarter * N + lane] = wl;
       named_bar_sync(1, kSoftmaxThreads);
-      if (quarter == 0 && lane < a.n_h) {
+      if (quarter == 0 && lane < nh_here) {
         const float lsum = s_wmax[lane] + s_wmax[N + lane] + s_wmax[2 * N + lane] + s_wmax[3 * N + lane];
-        a.part_ml[((size_t)item * a.n_h + lane) * 2 + 0] = m_ref;
-        a.part_ml[((size_t)item * a.n_h + lane) * 2 + 1] = lsum;
+        a.part_ml[((size_t)item * a.n_h + h0 + lane) * 2 + 0] = m_ref;
+        a.part_ml[((size_t)item * a.n_h + h0 + lane) * 2 + 1] = lsum;
       }
     }
   }
@@ -453,17 +457,34 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
 
 }  // namespace
 
+// Heads per block: all 32 when the fp32 output of every head fits TMEM's 512 columns, else
+// groups of 16 heads (each group streams the token tile itself; the groups of an item are
+// adjacent blocks so that the second and third reader hit L2).
+static int tc_pick_n(const elitekv_layer* L) {
+  const int nb = L->d_c / 128;
+  if (L->n_h == 32 && (nb + 1) * 32 <= 512) return 32;
+  if ((nb + 1) * 16 <= 512) return 16;
+  return 0;
+}
+
 int ekv_tc_supported(const elitekv_layer* L, const elitekv_cache* cache) {
   const int r2 = 2 * L->r;
-  if (L->n_h != 32) return 0;
-  if (L->d_c % 128 != 0 || (L->d_c / 128 + 1) * 32 > 512) return 0;
+  if (L->d_c % 128 != 0) return 0;
   if (!(r2 == 8 || r2 == 16 || r2 == 32)) return 0;
-  if (Smem<32>::total(L->d_c) > L->smem_optin) return 0;
+  const int n = tc_pick_n(L);
+  if (n == 0) return 0;
+  if ((L->n_h * r2) % 64 != 0 || L->n_h % 8 != 0) return 0;
+  if ((n == 32 ? Smem<32>::total(L->d_c) : Smem<16>::total(L->d_c)) > L->smem_optin) return 0;
   if (cache && cache->page_table && (cache->page_size % 64 != 0)) return 0;
   return 1;
 }
 
-int ekv_tc_max_items(const elitekv_layer* L, int B) { return L->sm_count + B; }
+static int tc_groups(const elitekv_layer* L) {
+  const int n = tc_pick_n(L);
+  return n ? (L->n_h + n - 1) / n : 1;
+}
+
+int ekv_tc_max_items(const elitekv_layer* L, int B) { return L->sm_count / tc_groups(L) + B; }
 
 int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, const CacheView& cv,
                          const void* q_rope, const void* q_abs, int B, const DecodeScratch& ws,
@@ -471,10 +492,12 @@ int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, con
   if (!ekv_tc_supported(L, cache)) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
   const unsigned long long rows =
       cv.page_table ? (unsigned long long)cv.num_pages << cv.page_shift : (unsigned long long)cv.max_ctx * cv.n_seqs;
+  if (rows >= (1ull << 31)) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
   CUtensorMap m_lat, m_rope, m_q;
   int rc = make_map(&m_lat, cache->latent, rows, L->d_c, 64);
   if (rc == ELITEKV_OK) rc = make_map(&m_rope, cache->rope, rows, (unsigned long long)L->n_h * 2 * L->r, 64);
-  if (rc == ELITEKV_OK) rc = make_map(&m_q, q_abs, (unsigned long long)B * L->n_h, L->d_c, 32);
+  const int N = tc_pick_n(L);
+  if (rc == ELITEKV_OK) rc = make_map(&m_q, q_abs, (unsigned long long)B * L->n_h, L->d_c, N);
   if (rc != ELITEKV_OK) return rc;
   TcArgs a;
   a.items = ws.items;
@@ -490,18 +513,26 @@ int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, con
   a.max_pages_per_seq = cv.max_pages_per_seq;
   a.n_h = L->n_h;
   a.d_c = L->d_c;
+  a.n_groups = tc_groups(L);
   a.scale_log2e = L->scale * 1.4426950408889634f;
-  const int smem = Smem<32>::total(L->d_c);
+  const int smem = N == 32 ? Smem<32>::total(L->d_c) : Smem<16>::total(L->d_c);
   auto launch = [&](auto kern) -> int {
     EKV_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    kern<<<ws.max_items, kThreads, smem, st>>>(m_lat, m_rope, m_q, a);
+    kern<<<ws.max_items * a.n_groups, kThreads, smem, st>>>(m_lat, m_rope, m_q, a);
     EKV_CUDA_OK(cudaGetLastError());
     return ELITEKV_OK;
   };
+  if (N == 32) {
+    switch (2 * L->r) {
+      case 8: return launch(decode_tc_kernel<32, 8>);
+      case 16: return launch(decode_tc_kernel<32, 16>);
+      default: return launch(decode_tc_kernel<32, 32>);
+    }
+  }
   switch (2 * L->r) {
-    case 8: return launch(decode_tc_kernel<32, 8>);
-    case 16: return launch(decode_tc_kernel<32, 16>);
-    default: return launch(decode_tc_kernel<32, 32>);
+    case 8: return launch(decode_tc_kernel<16, 8>);
+    case 16: return launch(decode_tc_kernel<16, 16>);
+    default: return launch(decode_tc_kernel<16, 32>);
   }
 }
 

@@ -60,7 +60,7 @@ Carve carve(const elitekv_layer* L, int B, int max_items) {
   c.off_acc = o;   o = align256(o + sizeof(float) * (size_t)max_items * L->n_h * L->d_c);
   c.off_slice = o; o = align256(o + ekv_combine_scratch_bytes(L, B));
   c.off_cnt = o;   o = align256(o + sizeof(int32_t) * (size_t)ekv_combine_counters(L, B));
-  c.off_wfirst = o; o = align256(o + sizeof(int32_t) * ((size_t)L->sm_count / 2 + 2));
+  c.off_wfirst = o; o = align256(o + sizeof(int32_t) * ((size_t)L->sm_count + 2));
   c.total = o;
   return c;
 }
@@ -127,11 +127,11 @@ extern "C" int elitekv_decode(const elitekv_layer* L, const elitekv_cache* cache
   ws.counters = (int32_t*)(base + cw.off_cnt);
   ws.n_counters = ekv_combine_counters(L, B);
   ws.worker_first = (int32_t*)(base + cw.off_wfirst);
-  ws.n_workers = kernel == 3 ? ekv_tc2_workers(L) : 0;
+  ws.n_workers = kernel == 3 ? ekv_tc2_workers(L) : kernel == 2 ? ekv_tc_workers(L) : 0;
   cudaStream_t st = (cudaStream_t)stream;
-  if (kernel == 3)
-    rc = ekv_launch_plan_balanced(seq_lens, B, 32, ws.n_workers, max_items, ws.items, ws.seq_first,
-                                  ws.worker_first, ws.counters, ws.n_counters, st);
+  if (kernel == 3 || kernel == 2)
+    rc = ekv_launch_plan_balanced(seq_lens, B, kernel == 3 ? 32 : 128, ws.n_workers, max_items, ws.items,
+                                  ws.seq_first, ws.worker_first, ws.counters, ws.n_counters, st);
   else
     rc = ekv_launch_plan(seq_lens, B, kernel == 2 ? 128 : ELITEKV_TILE_TOKENS, max_items, ws.items,
                          ws.seq_first, ws.counters, ws.n_counters, st);

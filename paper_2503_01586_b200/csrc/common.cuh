@@ -149,6 +149,7 @@ int ekv_launch_decode_generic(const elitekv_layer* L, const elitekv_cache* cache
                               const DecodeScratch& ws, cudaStream_t st);
 int ekv_tc_supported(const elitekv_layer* L, const elitekv_cache* cache);   // cache may be null
 int ekv_tc_max_items(const elitekv_layer* L, int B);
+int ekv_tc_workers(const elitekv_layer* L);
 int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, const CacheView& cv,
                          const void* q_rope, const void* q_abs, int B, const DecodeScratch& ws,
                          cudaStream_t st);

@@ -41,6 +41,7 @@ constexpr int kSoftmaxThreads = 128;
 
 struct TcArgs {
   const int32_t* items;
+  const int32_t* worker_first;
   const int32_t* page_table;
   float* part_acc;
   float* part_ml;
@@ -79,14 +80,11 @@ __global__ void __launch_bounds__(kThreads, 1)
 decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_constant__ CUtensorMap map_rope,
                  const __grid_constant__ CUtensorMap map_q, const TcArgs a) {
   extern __shared__ unsigned char smem_raw[];
-  const int item = blockIdx.x / a.n_groups;
+  const int worker = blockIdx.x / a.n_groups;         // persistent worker: walks its plan items
   const int h0 = (blockIdx.x % a.n_groups) * N;       // first head of this block's group
   const int nh_here = min(N, a.n_h - h0);
-  const int seq = a.items[4 * item + 0];
-  if (seq < 0) return;
-  const int tok0 = a.items[4 * item + 1];
-  const int ntok = a.items[4 * item + 2];
-  const int n_tiles = (ntok + kTile - 1) / kTile;
+  const int item_lo = a.worker_first[worker], item_hi = a.worker_first[worker + 1];
+  if (item_lo >= item_hi) return;
   const int d_c = a.d_c;
   const int NKC = d_c >> 6;      // 64-wide latent chunks
   const int NB = d_c >> 7;       // 128-row output blocks
@@ -126,11 +124,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
   }
-  // rotated query chunks of this sequence as fp32 (broadcast operand of the rope dot products)
-  for (int e = threadIdx.x; e < N * R2; e += kThreads) {
-    const int h = e / R2;
-    s_qrope[e] = h < nh_here ? __bfloat162float(a.q_rope[((size_t)seq * a.n_h + h0 + h) * R2 + (e % R2)]) : 0.f;
-  }
   const int tmem_cols_needed = NB * N + N;
   uint32_t tmem_cols = 32;
   while ((int)tmem_cols < tmem_cols_needed) tmem_cols <<= 1;
@@ -144,6 +137,22 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   const uint32_t tmem_base = *s_tmem;
   const uint32_t tmem_s = tmem_base + NB * N;     // S columns after the NB output blocks
 
+  // running counters (each role advances its own copies identically): ring uses, tiles, items
+  unsigned lat_n = 0, rope_n = 0, tbase = 0;
+  int seq = -1;
+  for (int item = item_lo; item < item_hi; ++item) {
+  seq = a.items[4 * item + 0];
+  const int tok0 = a.items[4 * item + 1];
+  const int ntok = a.items[4 * item + 2];
+  const int n_tiles = (ntok + kTile - 1) / kTile;
+  const unsigned item_n = (unsigned)(item - item_lo);
+  // rotated query chunks of this sequence as fp32 (broadcast operand of the rope dot products)
+  for (int e = threadIdx.x; e < N * R2; e += kThreads) {
+    const int h = e / R2;
+    s_qrope[e] = h < nh_here ? __bfloat162float(a.q_rope[((size_t)seq * a.n_h + h0 + h) * R2 + (e % R2)]) : 0.f;
+  }
+  __syncthreads();
+
   // ============================================================== warp 0: TMA producer
   if (warp == 0) {
     if (lane == 0) {
@@ -152,7 +161,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       for (int kc = 0; kc < NKC; ++kc)
         tma_load_2d(smem_u32(s_q + kc * N * 128), &map_q, kc * 64, seq * a.n_h + h0, qbar);
 
-      unsigned lat_n = 0, rope_n = 0;      // chunks issued so far
       bool ok = true;
       for (int tile = 0; tile < n_tiles && ok; ++tile) {
         const int t_abs = tok0 + tile * kTile;
@@ -211,8 +219,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   else if (warp == 1) {
     constexpr uint32_t idesc_s = make_idesc(128, N, 0, 0);    // S = C . Q^T   (both K-major)
     constexpr uint32_t idesc_pv = make_idesc(128, N, 1, 1);   // acc = C^T . P (both MN-major)
-    bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->q_full), 0, s_abort));
-    unsigned lat_n = 0;
+    bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->q_full), item_n & 1, s_abort));
     for (int tile = 0; tile < n_tiles && ok; ++tile) {
       const int nvalid = min(kTile, ntok - tile * kTile);
       // ---- pass A
@@ -240,7 +247,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       }
       __syncwarp();
       // ---- wait for P (and the rescaled output) of this tile
-      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_ready), tile & 1, s_abort));
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_ready), (tbase + tile) & 1, s_abort));
       if (!ok) break;
       tc_fence_after();
       if (lane == 0) EKV_STAMP(1, 21, tile);
@@ -294,7 +301,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
 #pragma unroll
     for (int h = 0; h < N; ++h) l_part[h] = 0.f;
     float m_ref = -INFINITY;                      // lane h holds head h's reference max (N <= 32 per group)
-    unsigned rope_n = 0;
     bool ok = true;
     static_assert(N == 16 || N == 32, "softmax threads keep one head per lane (lanes >= N idle)");
 
@@ -339,7 +345,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       if (!ok) break;
       if (threadIdx.x == 64) EKV_STAMP(2, 30, tile);
       // ---- latent part from TMEM
-      ok = mbar_wait(smem_u32(&bars->s_full), tile & 1, s_abort);
+      ok = mbar_wait(smem_u32(&bars->s_full), (tbase + tile) & 1, s_abort);
       if (!ok) break;
       tc_fence_after();
       if (threadIdx.x == 64) EKV_STAMP(2, 31, tile);
@@ -415,7 +421,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
     }
 
     // ---- epilogue: partial output and softmax statistics of this item
-    if (ok) ok = mbar_wait(smem_u32(&bars->pv_done), (n_tiles - 1) & 1, s_abort);
+    if (ok) ok = mbar_wait(smem_u32(&bars->pv_done), (tbase + n_tiles - 1) & 1, s_abort);
     if (ok) {
       tc_fence_after();
       float* pa = a.part_acc + ((size_t)item * a.n_h + h0) * d_c;
@@ -445,10 +451,17 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
     }
   }
 
+  // ---- end of item: every role is done with the queries, the P tile and the output columns
+  tbase += (unsigned)n_tiles;
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  }
+
   // ============================================================== teardown
   tc_fence_before();
   __syncthreads();
-  if (threadIdx.x == 0 && *s_abort) ekv_record(a.status, ELITEKV_ERR_TIMEOUT, item, seq);
+  if (threadIdx.x == 0 && *s_abort) ekv_record(a.status, ELITEKV_ERR_TIMEOUT, worker, seq);
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
@@ -484,7 +497,9 @@ static int tc_groups(const elitekv_layer* L) {
   return n ? (L->n_h + n - 1) / n : 1;
 }
 
-int ekv_tc_max_items(const elitekv_layer* L, int B) { return L->sm_count / tc_groups(L) + B; }
+// One persistent worker (a block per head group) per SM share; items = workers + sequences at most.
+int ekv_tc_workers(const elitekv_layer* L) { return L->sm_count / tc_groups(L) > 0 ? L->sm_count / tc_groups(L) : 1; }
+int ekv_tc_max_items(const elitekv_layer* L, int B) { return ekv_tc_workers(L) + B; }
 
 int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, const CacheView& cv,
                          const void* q_rope, const void* q_abs, int B, const DecodeScratch& ws,
@@ -501,6 +516,7 @@ int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, con
   if (rc != ELITEKV_OK) return rc;
   TcArgs a;
   a.items = ws.items;
+  a.worker_first = ws.worker_first;
   a.page_table = cv.page_table;
   a.part_acc = ws.part_acc;
   a.part_ml = ws.part_ml;
@@ -518,7 +534,7 @@ int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, con
   const int smem = N == 32 ? Smem<32>::total(L->d_c) : Smem<16>::total(L->d_c);
   auto launch = [&](auto kern) -> int {
     EKV_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    kern<<<ws.max_items * a.n_groups, kThreads, smem, st>>>(m_lat, m_rope, m_q, a);
+    kern<<<ws.n_workers * a.n_groups, kThreads, smem, st>>>(m_lat, m_rope, m_q, a);
     EKV_CUDA_OK(cudaGetLastError());
     return ELITEKV_OK;
   };

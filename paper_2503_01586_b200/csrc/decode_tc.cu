@@ -34,7 +34,7 @@ namespace {
 
 constexpr int kTile = 128;            // tokens per tile
 constexpr int kChunkBytes = 16384;    // [128 tokens][64 bf16] with 128-byte rows
-constexpr int kLatSlots = 4;
+constexpr int kLatSlots = 8;          // ring slots: one latent chunk + the matching query chunk each
 constexpr int kRopeSlots = 3;
 constexpr int kThreads = 192;
 constexpr int kSoftmaxThreads = 128;
@@ -58,15 +58,17 @@ struct TcArgs {
 struct __align__(8) TcBarriers {
   uint64_t lat_full[kLatSlots], lat_empty[kLatSlots];
   uint64_t rope_full[kRopeSlots], rope_empty[kRopeSlots];
-  uint64_t q_full, s_full, p_ready, pv_done;
+  uint64_t s_full, p_ready, pv_done;
 };
 
 // shared-memory carve-up (offsets from a 1024-byte aligned base)
 template <int N>
 struct Smem {
-  __host__ __device__ static constexpr int q_bytes(int d_c) { return (d_c / 64) * N * 128; }
-  __host__ __device__ static constexpr int lat_off(int d_c) { return q_bytes(d_c); }
-  __host__ __device__ static constexpr int rope_off(int d_c) { return lat_off(d_c) + kLatSlots * kChunkBytes; }
+  // a ring slot holds a latent chunk [128 tokens][64] and, behind it, the absorbed-query chunk
+  // [N heads][64] of the same latent coordinates (used by pass A only)
+  static constexpr int slot_bytes = kChunkBytes + N * 128;
+  __host__ __device__ static constexpr int lat_off(int) { return 0; }
+  __host__ __device__ static constexpr int rope_off(int d_c) { return lat_off(d_c) + kLatSlots * slot_bytes; }
   __host__ __device__ static constexpr int p_off(int d_c) { return rope_off(d_c) + kRopeSlots * kChunkBytes; }
   static constexpr int p_bytes = kTile * N * 2;
   __host__ __device__ static constexpr int misc_off(int d_c) { return p_off(d_c) + p_bytes; }
@@ -92,7 +94,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   constexpr int HPB = 64 / R2;       // heads per rope box
 
   unsigned char* base = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  unsigned char* s_q = base;
+  constexpr int kSlot = Smem<N>::slot_bytes;
   unsigned char* s_lat = base + Smem<N>::lat_off(d_c);
   unsigned char* s_rope = base + Smem<N>::rope_off(d_c);
   unsigned char* s_p = base + Smem<N>::p_off(d_c);
@@ -116,7 +118,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       mbar_init(smem_u32(&bars->rope_full[i]), 1);
       mbar_init(smem_u32(&bars->rope_empty[i]), kSoftmaxThreads / 32);
     }
-    mbar_init(smem_u32(&bars->q_full), 1);
     mbar_init(smem_u32(&bars->s_full), 1);
     mbar_init(smem_u32(&bars->p_ready), kSoftmaxThreads);
     mbar_init(smem_u32(&bars->pv_done), 1);
@@ -145,7 +146,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   const int tok0 = a.items[4 * item + 1];
   const int ntok = a.items[4 * item + 2];
   const int n_tiles = (ntok + kTile - 1) / kTile;
-  const unsigned item_n = (unsigned)(item - item_lo);
   // rotated query chunks of this sequence as fp32 (broadcast operand of the rope dot products)
   for (int e = threadIdx.x; e < N * R2; e += kThreads) {
     const int h = e / R2;
@@ -156,11 +156,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   // ============================================================== warp 0: TMA producer
   if (warp == 0) {
     if (lane == 0) {
-      const uint32_t qbar = smem_u32(&bars->q_full);
-      mbar_expect_tx(qbar, (uint32_t)(NKC * N * 128));
-      for (int kc = 0; kc < NKC; ++kc)
-        tma_load_2d(smem_u32(s_q + kc * N * 128), &map_q, kc * 64, seq * a.n_h + h0, qbar);
-
       bool ok = true;
       for (int tile = 0; tile < n_tiles && ok; ++tile) {
         const int t_abs = tok0 + tile * kTile;
@@ -182,14 +177,16 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
             row[hf] = ((long long)page << a.page_shift) + (t & a.page_mask);
           }
         }
-        auto load_lat = [&](int kc) -> bool {
+        auto load_lat = [&](int kc, bool with_q) -> bool {
           const unsigned slot = lat_n % kLatSlots;
           if (!mbar_wait(smem_u32(&bars->lat_empty[slot]), ((lat_n / kLatSlots) & 1) ^ 1, s_abort)) return false;
           const uint32_t fb = smem_u32(&bars->lat_full[slot]);
-          mbar_expect_tx(fb, (uint32_t)(halves * 8192));
+          mbar_expect_tx(fb, (uint32_t)(halves * 8192 + (with_q ? N * 128 : 0)));
+          if (with_q)   // the sequence's absorbed queries for these 64 latent coordinates (L2-resident)
+            tma_load_2d(smem_u32(s_lat + slot * kSlot + kChunkBytes), &map_q, kc * 64, seq * a.n_h + h0, fb);
           EKV_STAMP(0, 100 + kc, tile);
           for (int hf = 0; hf < halves; ++hf)
-            tma_load_2d(smem_u32(s_lat + slot * kChunkBytes + hf * 8192), &map_lat, kc * 64, (int)row[hf], fb);
+            tma_load_2d(smem_u32(s_lat + slot * kSlot + hf * 8192), &map_lat, kc * 64, (int)row[hf], fb);
           ++lat_n;
           return true;
         };
@@ -207,11 +204,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         int cb = 0;
         for (int kc = 0; kc < NKC && ok; ++kc) {
           if (cb < NRB && (long long)kc * NRB >= (long long)cb * NKC) ok = load_rope(cb++);
-          if (ok) ok = load_lat(kc);
+          if (ok) ok = load_lat(kc, true);
         }
         while (cb < NRB && ok) ok = load_rope(cb++);
         // pass B: the same latent chunks again (served by L2)
-        for (int kc = 0; kc < NKC && ok; ++kc) ok = load_lat(kc);
+        for (int kc = 0; kc < NKC && ok; ++kc) ok = load_lat(kc, false);
       }
     }
   }
@@ -219,7 +216,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   else if (warp == 1) {
     constexpr uint32_t idesc_s = make_idesc(128, N, 0, 0);    // S = C . Q^T   (both K-major)
     constexpr uint32_t idesc_pv = make_idesc(128, N, 1, 1);   // acc = C^T . P (both MN-major)
-    bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->q_full), item_n & 1, s_abort));
+    bool ok = true;
     for (int tile = 0; tile < n_tiles && ok; ++tile) {
       const int nvalid = min(kTile, ntok - tile * kTile);
       // ---- pass A
@@ -229,8 +226,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         if (!ok) break;
         tc_fence_after();
         if (lane == 0) {
-          const uint32_t a_addr = smem_u32(s_lat + slot * kChunkBytes);
-          const uint32_t b_addr = smem_u32(s_q + kc * N * 128);
+          const uint32_t a_addr = smem_u32(s_lat + slot * kSlot);
+          const uint32_t b_addr = a_addr + kChunkBytes;
 #pragma unroll
           for (int k = 0; k < 4; ++k)
             tc_mma(tmem_s, make_desc(a_addr + k * 32, 16, 1024, 2), make_desc(b_addr + k * 32, 16, 1024, 2),
@@ -265,7 +262,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
           // exact zeros so that 0-probability rows cannot inject NaN/Inf bit patterns
           for (int e = lane; e < (zero_to - zero_from) * 16; e += 32) {
             const int rrow = zero_from + (e >> 4), c16 = e & 15;
-            unsigned char* p = s_lat + (c16 < 8 ? s0 : s1) * kChunkBytes + rrow * 128 + (c16 & 7) * 16;
+            unsigned char* p = s_lat + (c16 < 8 ? s0 : s1) * kSlot + rrow * 128 + (c16 & 7) * 16;
             *(uint4*)p = make_uint4(0, 0, 0, 0);
           }
           fence_proxy_async();
@@ -273,10 +270,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         }
         tc_fence_after();
         if (lane == 0) {
-          const uint32_t a_addr = smem_u32(s_lat + s0 * kChunkBytes);
+          const uint32_t a_addr = smem_u32(s_lat + s0 * kSlot);
           const uint32_t b_addr = smem_u32(s_p);
           for (int k = 0; k < ksteps; ++k)
-            tc_mma(tmem_base + blk * N, make_desc(a_addr + k * 2048, kChunkBytes, 1024, 2),
+            tc_mma(tmem_base + blk * N, make_desc(a_addr + k * 2048, kSlot, 1024, 2),
                    make_desc(b_addr + k * 256, 128, 2048, 0), idesc_pv, (tile | k) != 0);
           tc_commit(smem_u32(&bars->lat_empty[s0]));
           tc_commit(smem_u32(&bars->lat_empty[s1]));

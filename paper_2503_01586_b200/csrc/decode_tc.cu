@@ -80,7 +80,8 @@ struct Smem {
 template <int N, int R2>
 __global__ void __launch_bounds__(kThreads, 1)
 decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_constant__ CUtensorMap map_rope,
-                 const __grid_constant__ CUtensorMap map_q, const TcArgs a) {
+                 const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_lat128,
+                 const __grid_constant__ CUtensorMap map_rope128, const TcArgs a) {
   extern __shared__ unsigned char smem_raw[];
   const int worker = blockIdx.x / a.n_groups;         // persistent worker: walks its plan items
   const int h0 = (blockIdx.x % a.n_groups) * N;       // first head of this block's group
@@ -177,6 +178,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
             row[hf] = ((long long)page << a.page_shift) + (t & a.page_mask);
           }
         }
+        // both 64-row halves adjacent in the cache: one 128-row box instead of two
+        const bool whole = halves == 2 && row[1] == row[0] + 64;
         auto load_lat = [&](int kc, bool with_q) -> bool {
           const unsigned slot = lat_n % kLatSlots;
           if (!mbar_wait(smem_u32(&bars->lat_empty[slot]), ((lat_n / kLatSlots) & 1) ^ 1, s_abort)) return false;
@@ -185,8 +188,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
           if (with_q)   // the sequence's absorbed queries for these 64 latent coordinates (L2-resident)
             tma_load_2d(smem_u32(s_lat + slot * kSlot + kChunkBytes), &map_q, kc * 64, seq * a.n_h + h0, fb);
           EKV_STAMP(0, 100 + kc, tile);
-          for (int hf = 0; hf < halves; ++hf)
-            tma_load_2d(smem_u32(s_lat + slot * kSlot + hf * 8192), &map_lat, kc * 64, (int)row[hf], fb);
+          if (whole) {
+            tma_load_2d(smem_u32(s_lat + slot * kSlot), &map_lat128, kc * 64, (int)row[0], fb);
+          } else {
+            for (int hf = 0; hf < halves; ++hf)
+              tma_load_2d(smem_u32(s_lat + slot * kSlot + hf * 8192), &map_lat, kc * 64, (int)row[hf], fb);
+          }
           ++lat_n;
           return true;
         };
@@ -195,8 +202,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
           if (!mbar_wait(smem_u32(&bars->rope_empty[slot]), ((rope_n / kRopeSlots) & 1) ^ 1, s_abort)) return false;
           const uint32_t fb = smem_u32(&bars->rope_full[slot]);
           mbar_expect_tx(fb, (uint32_t)(halves * 8192));
-          for (int hf = 0; hf < halves; ++hf)
-            tma_load_2d(smem_u32(s_rope + slot * kChunkBytes + hf * 8192), &map_rope, h0 * R2 + cb * 64, (int)row[hf], fb);
+          if (whole) {
+            tma_load_2d(smem_u32(s_rope + slot * kChunkBytes), &map_rope128, h0 * R2 + cb * 64, (int)row[0], fb);
+          } else {
+            for (int hf = 0; hf < halves; ++hf)
+              tma_load_2d(smem_u32(s_rope + slot * kChunkBytes + hf * 8192), &map_rope, h0 * R2 + cb * 64, (int)row[hf], fb);
+          }
           ++rope_n;
           return true;
         };
@@ -505,9 +516,11 @@ int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, con
   const unsigned long long rows =
       cv.page_table ? (unsigned long long)cv.num_pages << cv.page_shift : (unsigned long long)cv.max_ctx * cv.n_seqs;
   if (rows >= (1ull << 31)) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
-  CUtensorMap m_lat, m_rope, m_q;
+  CUtensorMap m_lat, m_rope, m_q, m_lat128, m_rope128;
   int rc = make_map(&m_lat, cache->latent, rows, L->d_c, 64);
   if (rc == ELITEKV_OK) rc = make_map(&m_rope, cache->rope, rows, (unsigned long long)L->n_h * 2 * L->r, 64);
+  if (rc == ELITEKV_OK) rc = make_map(&m_lat128, cache->latent, rows, L->d_c, 128);
+  if (rc == ELITEKV_OK) rc = make_map(&m_rope128, cache->rope, rows, (unsigned long long)L->n_h * 2 * L->r, 128);
   const int N = tc_pick_n(L);
   if (rc == ELITEKV_OK) rc = make_map(&m_q, q_abs, (unsigned long long)B * L->n_h, L->d_c, N);
   if (rc != ELITEKV_OK) return rc;
@@ -531,7 +544,7 @@ int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, con
   const int smem = N == 32 ? Smem<32>::total(L->d_c) : Smem<16>::total(L->d_c);
   auto launch = [&](auto kern) -> int {
     EKV_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    kern<<<ws.n_workers * a.n_groups, kThreads, smem, st>>>(m_lat, m_rope, m_q, a);
+    kern<<<ws.n_workers * a.n_groups, kThreads, smem, st>>>(m_lat, m_rope, m_q, m_lat128, m_rope128, a);
     EKV_CUDA_OK(cudaGetLastError());
     return ELITEKV_OK;
   };

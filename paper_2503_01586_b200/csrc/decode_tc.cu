@@ -233,7 +233,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       // ---- pass A
       for (int kc = 0; kc < NKC && ok; ++kc) {
         const unsigned slot = lat_n % kLatSlots;
-        ok = mbar_wait_warp(smem_u32(&bars->lat_full[slot]), (lat_n / kLatSlots) & 1, s_abort);
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->lat_full[slot]), (lat_n / kLatSlots) & 1, s_abort));
         if (!ok) break;
         tc_fence_after();
         if (lane == 0) {
@@ -255,7 +255,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       }
       __syncwarp();
       // ---- wait for P (and the rescaled output) of this tile
-      ok = mbar_wait_warp(smem_u32(&bars->p_ready), (tbase + tile) & 1, s_abort);
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_ready), (tbase + tile) & 1, s_abort));
       if (!ok) break;
       tc_fence_after();
       if (lane == 0) EKV_STAMP(1, 21, tile);
@@ -264,8 +264,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       const int zero_from = nvalid, zero_to = ksteps * 16;
       for (int blk = 0; blk < NB && ok; ++blk) {
         const unsigned s0 = lat_n % kLatSlots, s1 = (lat_n + 1) % kLatSlots;
-        ok = mbar_wait_warp(smem_u32(&bars->lat_full[s0]), (lat_n / kLatSlots) & 1, s_abort) &&
-             mbar_wait_warp(smem_u32(&bars->lat_full[s1]), ((lat_n + 1) / kLatSlots) & 1, s_abort);
+        ok = mbar_wait(smem_u32(&bars->lat_full[s0]), (lat_n / kLatSlots) & 1, s_abort) &&
+             mbar_wait(smem_u32(&bars->lat_full[s1]), ((lat_n + 1) / kLatSlots) & 1, s_abort);
+        ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         if (zero_to > zero_from) {
           // token rows past the end of the sequence inside the last 16-token step: make them
@@ -321,7 +322,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       for (int cb = 0; cb < NRB; ++cb) {
         if (!ok) break;
         const unsigned slot = rope_n % kRopeSlots;
-        ok = mbar_wait_warp(smem_u32(&bars->rope_full[slot]), (rope_n / kRopeSlots) & 1, s_abort);
+        ok = mbar_wait(smem_u32(&bars->rope_full[slot]), (rope_n / kRopeSlots) & 1, s_abort);
         if (!ok) break;
         const unsigned char* rowp = s_rope + slot * kChunkBytes + trow * 128;
         float part[HPB];
@@ -352,7 +353,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       if (!ok) break;
       if (threadIdx.x == 64) EKV_STAMP(2, 30, tile);
       // ---- latent part from TMEM
-      ok = mbar_wait_warp(smem_u32(&bars->s_full), (tbase + tile) & 1, s_abort);
+      ok = mbar_wait(smem_u32(&bars->s_full), (tbase + tile) & 1, s_abort);
       if (!ok) break;
       tc_fence_after();
       if (threadIdx.x == 64) EKV_STAMP(2, 31, tile);
@@ -428,7 +429,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
     }
 
     // ---- epilogue: partial output and softmax statistics of this item
-    if (ok) ok = mbar_wait_warp(smem_u32(&bars->pv_done), (tbase + n_tiles - 1) & 1, s_abort);
+    if (ok) ok = mbar_wait(smem_u32(&bars->pv_done), (tbase + n_tiles - 1) & 1, s_abort);
     if (ok) {
       tc_fence_after();
       float* pa = a.part_acc + ((size_t)item * a.n_h + h0) * d_c;

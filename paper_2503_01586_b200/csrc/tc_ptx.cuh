@@ -60,16 +60,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   *abort_flag = 1;
   return false;
 }
-// Warp-collective wait (all 32 lanes must call it): only lane 0 polls, so that waiting warps do
-// not flood the shared-memory pipe that the tensor core's operand fetch also uses; afterwards
-// every lane confirms the phase itself (immediate) to get its own acquire.  Uniform result.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  bool ok = true;
-  if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag);
-  ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-  if (ok) ok = mbar_try_wait(bar, parity);
-  return __all_sync(0xffffffffu, ok);
-}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"

@@ -36,7 +36,8 @@ constexpr int kTile = 128;            // tokens per tile
 constexpr int kChunkBytes = 16384;    // [128 tokens][64 bf16] with 128-byte rows
 constexpr int kLatSlots = 8;          // ring slots: one latent chunk + the matching query chunk each
 constexpr int kRopeSlots = 3;
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;         // warp 0 latent loads, 1 MMA, 2-5 softmax, 6 rope loads
+constexpr int kProdLanes = 4;
 constexpr int kSoftmaxThreads = 128;
 
 struct TcArgs {
@@ -154,9 +155,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   }
   __syncthreads();
 
-  // ============================================================== warp 0: TMA producer
-  if (warp == 0) {
-    if (lane == 0) {
+  // ============================================================== warp 0: latent TMA producers
+  // One thread can issue a TMA load only every ~0.17 us (wait + expect_tx + issue), i.e. about
+  // 47 GB/s of 8 KB boxes per SM.  Four lanes of this warp therefore run the same loop in
+  // lockstep, lane j owning every fourth ring use, so one warp instruction issues four loads.
+  if (warp == 0 || warp == 6) {
+    const bool rope_role = warp == 6;
+    if ((!rope_role && lane < kProdLanes) || (rope_role && lane == 0)) {
       bool ok = true;
       for (int tile = 0; tile < n_tiles && ok; ++tile) {
         const int t_abs = tok0 + tile * kTile;
@@ -172,7 +177,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
             int page = (hf < halves && pi < a.max_pages_per_seq)
                            ? a.page_table[(long long)seq * a.max_pages_per_seq + pi] : 0;
             if (page < 0 || page >= a.num_pages) {
-              if (hf < halves) ekv_record(a.status, ELITEKV_ERR_BAD_PAGE, seq, page);
+              if (hf < halves && rope_role) ekv_record(a.status, ELITEKV_ERR_BAD_PAGE, seq, page);
               page = 0;
             }
             row[hf] = ((long long)page << a.page_shift) + (t & a.page_mask);
@@ -180,46 +185,45 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         }
         // both 64-row halves adjacent in the cache: one 128-row box instead of two
         const bool whole = halves == 2 && row[1] == row[0] + 64;
-        auto load_lat = [&](int kc, bool with_q) -> bool {
-          const unsigned slot = lat_n % kLatSlots;
-          if (!mbar_wait(smem_u32(&bars->lat_empty[slot]), ((lat_n / kLatSlots) & 1) ^ 1, s_abort)) return false;
-          const uint32_t fb = smem_u32(&bars->lat_full[slot]);
-          mbar_expect_tx(fb, (uint32_t)(halves * 8192 + (with_q ? N * 128 : 0)));
-          if (with_q)   // the sequence's absorbed queries for these 64 latent coordinates (L2-resident)
-            tma_load_2d(smem_u32(s_lat + slot * kSlot + kChunkBytes), &map_q, kc * 64, seq * a.n_h + h0, fb);
-          EKV_STAMP(0, 100 + kc, tile);
-          if (whole) {
-            tma_load_2d(smem_u32(s_lat + slot * kSlot), &map_lat128, kc * 64, (int)row[0], fb);
-          } else {
-            for (int hf = 0; hf < halves; ++hf)
-              tma_load_2d(smem_u32(s_lat + slot * kSlot + hf * 8192), &map_lat, kc * 64, (int)row[hf], fb);
+        if (!rope_role) {
+          // ring uses of this tile: NKC chunks of pass A (each with its query chunk), then the
+          // same NKC chunks again for pass B (served by L2)
+          for (int u = lane; u < 2 * NKC && ok; u += kProdLanes) {
+            const bool with_q = u < NKC;
+            const int kc = with_q ? u : u - NKC;
+            const unsigned n = lat_n + (unsigned)u, slot = n % kLatSlots;
+            ok = mbar_wait(smem_u32(&bars->lat_empty[slot]), ((n / kLatSlots) & 1) ^ 1, s_abort);
+            if (!ok) break;
+            const uint32_t fb = smem_u32(&bars->lat_full[slot]);
+            mbar_expect_tx(fb, (uint32_t)(halves * 8192 + (with_q ? N * 128 : 0)));
+            if (with_q)   // the sequence's absorbed queries for these 64 latent coordinates (L2-resident)
+              tma_load_2d(smem_u32(s_lat + slot * kSlot + kChunkBytes), &map_q, kc * 64, seq * a.n_h + h0, fb);
+            if (lane == 0) EKV_STAMP(0, (with_q ? 100 : 200) + kc, tile);
+            if (whole) {
+              tma_load_2d(smem_u32(s_lat + slot * kSlot), &map_lat128, kc * 64, (int)row[0], fb);
+            } else {
+              for (int hf = 0; hf < halves; ++hf)
+                tma_load_2d(smem_u32(s_lat + slot * kSlot + hf * 8192), &map_lat, kc * 64, (int)row[hf], fb);
+            }
           }
-          ++lat_n;
-          return true;
-        };
-        auto load_rope = [&](int cb) -> bool {
-          const unsigned slot = rope_n % kRopeSlots;
-          if (!mbar_wait(smem_u32(&bars->rope_empty[slot]), ((rope_n / kRopeSlots) & 1) ^ 1, s_abort)) return false;
-          const uint32_t fb = smem_u32(&bars->rope_full[slot]);
-          mbar_expect_tx(fb, (uint32_t)(halves * 8192));
-          if (whole) {
-            tma_load_2d(smem_u32(s_rope + slot * kChunkBytes), &map_rope128, h0 * R2 + cb * 64, (int)row[0], fb);
-          } else {
-            for (int hf = 0; hf < halves; ++hf)
-              tma_load_2d(smem_u32(s_rope + slot * kChunkBytes + hf * 8192), &map_rope, h0 * R2 + cb * 64, (int)row[hf], fb);
+          lat_n += 2u * (unsigned)NKC;
+        } else {
+          // warp 6: the rope boxes of the tile
+          for (int cb = 0; cb < NRB && ok; ++cb) {
+            const unsigned slot = rope_n % kRopeSlots;
+            ok = mbar_wait(smem_u32(&bars->rope_empty[slot]), ((rope_n / kRopeSlots) & 1) ^ 1, s_abort);
+            if (!ok) break;
+            const uint32_t fb = smem_u32(&bars->rope_full[slot]);
+            mbar_expect_tx(fb, (uint32_t)(halves * 8192));
+            if (whole) {
+              tma_load_2d(smem_u32(s_rope + slot * kChunkBytes), &map_rope128, h0 * R2 + cb * 64, (int)row[0], fb);
+            } else {
+              for (int hf = 0; hf < halves; ++hf)
+                tma_load_2d(smem_u32(s_rope + slot * kChunkBytes + hf * 8192), &map_rope, h0 * R2 + cb * 64, (int)row[hf], fb);
+            }
+            ++rope_n;
           }
-          ++rope_n;
-          return true;
-        };
-        // pass A: latent chunks with the rope boxes spread between them
-        int cb = 0;
-        for (int kc = 0; kc < NKC && ok; ++kc) {
-          if (cb < NRB && (long long)kc * NRB >= (long long)cb * NKC) ok = load_rope(cb++);
-          if (ok) ok = load_lat(kc, true);
         }
-        while (cb < NRB && ok) ok = load_rope(cb++);
-        // pass B: the same latent chunks again (served by L2)
-        for (int kc = 0; kc < NKC && ok; ++kc) ok = load_lat(kc, false);
       }
     }
   }

@@ -162,6 +162,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   if (warp == 0 || warp == 6) {
     const bool rope_role = warp == 6;
     if ((!rope_role && lane < kProdLanes) || (rope_role && lane == 0)) {
+      // L2 priorities: a latent chunk read in pass A is read again soon (pass B) -> keep; after
+      // pass B, and for rope rows, the data is dead -> first to go; the queries are re-read by
+      // every tile of the sequence -> keep
+      const uint64_t pol_keep = make_l2_policy_evict_last(), pol_drop = make_l2_policy_evict_first();
       bool ok = true;
       for (int tile = 0; tile < n_tiles && ok; ++tile) {
         const int t_abs = tok0 + tile * kTile;
@@ -197,13 +201,14 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
             const uint32_t fb = smem_u32(&bars->lat_full[slot]);
             mbar_expect_tx(fb, (uint32_t)(halves * 8192 + (with_q ? N * 128 : 0)));
             if (with_q)   // the sequence's absorbed queries for these 64 latent coordinates (L2-resident)
-              tma_load_2d(smem_u32(s_lat + slot * kSlot + kChunkBytes), &map_q, kc * 64, seq * a.n_h + h0, fb);
+              tma_load_2d_hint(smem_u32(s_lat + slot * kSlot + kChunkBytes), &map_q, kc * 64, seq * a.n_h + h0, fb, pol_keep);
             if (lane == 0) EKV_STAMP(0, (with_q ? 100 : 200) + kc, tile);
+            const uint64_t pol = with_q ? pol_keep : pol_drop;
             if (whole) {
-              tma_load_2d(smem_u32(s_lat + slot * kSlot), &map_lat128, kc * 64, (int)row[0], fb);
+              tma_load_2d_hint(smem_u32(s_lat + slot * kSlot), &map_lat128, kc * 64, (int)row[0], fb, pol);
             } else {
               for (int hf = 0; hf < halves; ++hf)
-                tma_load_2d(smem_u32(s_lat + slot * kSlot + hf * 8192), &map_lat, kc * 64, (int)row[hf], fb);
+                tma_load_2d_hint(smem_u32(s_lat + slot * kSlot + hf * 8192), &map_lat, kc * 64, (int)row[hf], fb, pol);
             }
           }
           lat_n += 2u * (unsigned)NKC;
@@ -216,10 +221,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
             const uint32_t fb = smem_u32(&bars->rope_full[slot]);
             mbar_expect_tx(fb, (uint32_t)(halves * 8192));
             if (whole) {
-              tma_load_2d(smem_u32(s_rope + slot * kChunkBytes), &map_rope128, h0 * R2 + cb * 64, (int)row[0], fb);
+              tma_load_2d_hint(smem_u32(s_rope + slot * kChunkBytes), &map_rope128, h0 * R2 + cb * 64, (int)row[0], fb, pol_drop);
             } else {
               for (int hf = 0; hf < halves; ++hf)
-                tma_load_2d(smem_u32(s_rope + slot * kChunkBytes + hf * 8192), &map_rope, h0 * R2 + cb * 64, (int)row[hf], fb);
+                tma_load_2d_hint(smem_u32(s_rope + slot * kChunkBytes + hf * 8192), &map_rope, h0 * R2 + cb * 64, (int)row[hf], fb, pol_drop);
             }
             ++rope_n;
           }

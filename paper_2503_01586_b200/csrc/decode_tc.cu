@@ -36,8 +36,8 @@ constexpr int kTile = 128;            // tokens per tile
 constexpr int kChunkBytes = 16384;    // [128 tokens][64 bf16] with 128-byte rows
 constexpr int kLatSlots = 8;          // ring slots: one latent chunk + the matching query chunk each
 constexpr int kRopeSlots = 3;
-constexpr int kThreads = 224;         // warp 0 latent loads, 1 MMA, 2-5 softmax, 6 rope loads
-constexpr int kProdLanes = 4;
+constexpr int kThreads = 288;         // warp 0 latent loads, 1 MMA, 2-5 softmax, 6 rope loads, 7-8 latent loads
+constexpr int kProdWarps = 3;         // latent-load warps: 0, 7, 8 (one issuing lane each)
 constexpr int kSoftmaxThreads = 128;
 
 struct TcArgs {
@@ -155,13 +155,14 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   }
   __syncthreads();
 
-  // ============================================================== warp 0: latent TMA producers
+  // ============================================================== warps 0, 7, 8: latent TMA producers; warp 6: rope
   // One thread can issue a TMA load only every ~0.17 us (wait + expect_tx + issue), i.e. about
-  // 47 GB/s of 8 KB boxes per SM.  Four lanes of this warp therefore run the same loop in
-  // lockstep, lane j owning every fourth ring use, so one warp instruction issues four loads.
-  if (warp == 0 || warp == 6) {
+  // 47 GB/s of 8 KB boxes per SM, and two issuing warps were measured to double that.  The
+  // latent ring uses are therefore dealt round-robin to kProdWarps warps.
+  if (warp == 0 || warp >= 6) {
     const bool rope_role = warp == 6;
-    if ((!rope_role && lane < kProdLanes) || (rope_role && lane == 0)) {
+    const int prod = warp == 0 ? 0 : warp - 6;          // latent producer index
+    if (lane == 0) {
       // L2 priorities: a latent chunk read in pass A is read again soon (pass B) -> keep; after
       // pass B, and for rope rows, the data is dead -> first to go; the queries are re-read by
       // every tile of the sequence -> keep
@@ -192,7 +193,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         if (!rope_role) {
           // ring uses of this tile: NKC chunks of pass A (each with its query chunk), then the
           // same NKC chunks again for pass B (served by L2)
-          for (int u = lane; u < 2 * NKC && ok; u += kProdLanes) {
+          for (int u = prod; u < 2 * NKC && ok; u += kProdWarps) {
             const bool with_q = u < NKC;
             const int kc = with_q ? u : u - NKC;
             const unsigned n = lat_n + (unsigned)u, slot = n % kLatSlots;
@@ -202,7 +203,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
             mbar_expect_tx(fb, (uint32_t)(halves * 8192 + (with_q ? N * 128 : 0)));
             if (with_q)   // the sequence's absorbed queries for these 64 latent coordinates (L2-resident)
               tma_load_2d_hint(smem_u32(s_lat + slot * kSlot + kChunkBytes), &map_q, kc * 64, seq * a.n_h + h0, fb, pol_keep);
-            if (lane == 0) EKV_STAMP(0, (with_q ? 100 : 200) + kc, tile);
+            if (prod == 0) EKV_STAMP(0, (with_q ? 100 : 200) + kc, tile);
             const uint64_t pol = with_q ? pol_keep : pol_drop;
             if (whole) {
               tma_load_2d_hint(smem_u32(s_lat + slot * kSlot), &map_lat128, kc * 64, (int)row[0], fb, pol);

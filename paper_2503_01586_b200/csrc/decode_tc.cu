@@ -243,8 +243,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       // ---- pass A
       for (int kc = 0; kc < NKC && ok; ++kc) {
         const unsigned slot = lat_n % kLatSlots;
+        if (lane == 0 && (kc & 3) == 0) EKV_STAMP(1, 300 + kc, tile);
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->lat_full[slot]), (lat_n / kLatSlots) & 1, s_abort));
         if (!ok) break;
+        if (lane == 0 && (kc & 3) == 0) EKV_STAMP(1, 400 + kc, tile);
         tc_fence_after();
         if (lane == 0) {
           const uint32_t a_addr = smem_u32(s_lat + slot * kSlot);
@@ -274,10 +276,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       const int zero_from = nvalid, zero_to = ksteps * 16;
       for (int blk = 0; blk < NB && ok; ++blk) {
         const unsigned s0 = lat_n % kLatSlots, s1 = (lat_n + 1) % kLatSlots;
+        if (lane == 0 && (blk & 1) == 0) EKV_STAMP(1, 500 + blk, tile);
         ok = mbar_wait(smem_u32(&bars->lat_full[s0]), (lat_n / kLatSlots) & 1, s_abort) &&
              mbar_wait(smem_u32(&bars->lat_full[s1]), ((lat_n + 1) / kLatSlots) & 1, s_abort);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
+        if (lane == 0 && (blk & 1) == 0) EKV_STAMP(1, 600 + blk, tile);
         if (zero_to > zero_from) {
           // token rows past the end of the sequence inside the last 16-token step: make them
           // exact zeros so that 0-probability rows cannot inject NaN/Inf bit patterns

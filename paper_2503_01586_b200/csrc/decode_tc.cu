@@ -234,57 +234,54 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
     }
   }
   // ============================================================== warp 1: MMA issuer
+  // Lane 0 alone waits, issues and commits (per-chunk warp-wide synchronisation costs as much as
+  // the MMAs themselves); the other lanes only help to zero a ragged tail.
   else if (warp == 1) {
     constexpr uint32_t idesc_s = make_idesc(128, N, 0, 0);    // S = C . Q^T   (both K-major)
     constexpr uint32_t idesc_pv = make_idesc(128, N, 1, 1);   // acc = C^T . P (both MN-major)
     bool ok = true;
     for (int tile = 0; tile < n_tiles && ok; ++tile) {
       const int nvalid = min(kTile, ntok - tile * kTile);
-      // ---- pass A
-      for (int kc = 0; kc < NKC && ok; ++kc) {
-        const unsigned slot = lat_n % kLatSlots;
-        if (lane == 0 && (kc & 3) == 0) EKV_STAMP(1, 300 + kc, tile);
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->lat_full[slot]), (lat_n / kLatSlots) & 1, s_abort));
-        if (!ok) break;
-        if (lane == 0 && (kc & 3) == 0) EKV_STAMP(1, 400 + kc, tile);
-        tc_fence_after();
-        if (lane == 0) {
-          const uint32_t a_addr = smem_u32(s_lat + slot * kSlot);
-          const uint32_t b_addr = a_addr + kChunkBytes;
-#pragma unroll
-          for (int k = 0; k < 4; ++k)
-            tc_mma(tmem_s, make_desc(a_addr + k * 32, 16, 1024, 2), make_desc(b_addr + k * 32, 16, 1024, 2),
-                   idesc_s, (kc | k) != 0);
-          tc_commit(smem_u32(&bars->lat_empty[slot]));
-        }
-        __syncwarp();
-        ++lat_n;
-      }
-      if (!ok) break;
-      if (lane == 0) {
-        tc_commit(smem_u32(&bars->s_full));
-        EKV_STAMP(1, 20, tile);
-      }
-      __syncwarp();
-      // ---- wait for P (and the rescaled output) of this tile
-      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_ready), (tbase + tile) & 1, s_abort));
-      if (!ok) break;
-      tc_fence_after();
-      if (lane == 0) EKV_STAMP(1, 21, tile);
-      // ---- pass B
       const int ksteps = (nvalid + 15) >> 4;
       const int zero_from = nvalid, zero_to = ksteps * 16;
-      for (int blk = 0; blk < NB && ok; ++blk) {
-        const unsigned s0 = lat_n % kLatSlots, s1 = (lat_n + 1) % kLatSlots;
-        if (lane == 0 && (blk & 1) == 0) EKV_STAMP(1, 500 + blk, tile);
-        ok = mbar_wait(smem_u32(&bars->lat_full[s0]), (lat_n / kLatSlots) & 1, s_abort) &&
-             mbar_wait(smem_u32(&bars->lat_full[s1]), ((lat_n + 1) / kLatSlots) & 1, s_abort);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        if (lane == 0 && (blk & 1) == 0) EKV_STAMP(1, 600 + blk, tile);
-        if (zero_to > zero_from) {
-          // token rows past the end of the sequence inside the last 16-token step: make them
-          // exact zeros so that 0-probability rows cannot inject NaN/Inf bit patterns
+      const unsigned n0 = lat_n;                 // first ring use of this tile
+      if (lane == 0) {
+        // ---- pass A
+        for (int kc = 0; kc < NKC && ok; ++kc) {
+          const unsigned n = n0 + kc, slot = n % kLatSlots;
+          if ((kc & 3) == 0) EKV_STAMP(1, 300 + kc, tile);
+          ok = mbar_wait(smem_u32(&bars->lat_full[slot]), (n / kLatSlots) & 1, s_abort);
+          if (!ok) break;
+          const uint32_t a_addr = smem_u32(s_lat + slot * kSlot);
+          const uint64_t da = make_desc(a_addr, 16, 1024, 2), db = make_desc(a_addr + kChunkBytes, 16, 1024, 2);
+#pragma unroll
+          for (int k = 0; k < 4; ++k)      // +32 bytes along K per step = +2 in the address field
+            tc_mma(tmem_s, da + 2 * k, db + 2 * k, idesc_s, (kc | k) != 0);
+          tc_commit(smem_u32(&bars->lat_empty[slot]));
+        }
+        if (ok) {
+          tc_commit(smem_u32(&bars->s_full));
+          EKV_STAMP(1, 20, tile);
+          // ---- wait for P (and the rescaled output) of this tile
+          ok = mbar_wait(smem_u32(&bars->p_ready), (tbase + tile) & 1, s_abort);
+          tc_fence_after();
+          EKV_STAMP(1, 21, tile);
+        }
+      }
+      // ---- pass B
+      const uint32_t p_addr = smem_u32(s_p);
+      if (zero_to > zero_from) {
+        // ragged end of a sequence: rows past its last token inside the last 16-token step are
+        // made exact zeros (warp-cooperatively) so that zero-probability rows cannot inject
+        // NaN/Inf bit patterns
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        for (int blk = 0; blk < NB && ok; ++blk) {
+          const unsigned n = n0 + NKC + 2 * blk, s0 = n % kLatSlots, s1 = (n + 1) % kLatSlots;
+          if (lane == 0)
+            ok = mbar_wait(smem_u32(&bars->lat_full[s0]), (n / kLatSlots) & 1, s_abort) &&
+                 mbar_wait(smem_u32(&bars->lat_full[s1]), ((n + 1) / kLatSlots) & 1, s_abort);
+          ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+          if (!ok) break;
           for (int e = lane; e < (zero_to - zero_from) * 16; e += 32) {
             const int rrow = zero_from + (e >> 4), c16 = e & 15;
             unsigned char* p = s_lat + (c16 < 8 ? s0 : s1) * kSlot + rrow * 128 + (c16 & 7) * 16;
@@ -292,26 +289,36 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
           }
           fence_proxy_async();
           __syncwarp();
+          if (lane == 0) {
+            const uint64_t da = make_desc(smem_u32(s_lat + s0 * kSlot), kSlot, 1024, 2), db = make_desc(p_addr, 128, 2048, 0);
+            for (int k = 0; k < ksteps; ++k)
+              tc_mma(tmem_base + blk * N, da + 128 * k, db + 16 * k, idesc_pv, (tile | k) != 0);
+            tc_commit(smem_u32(&bars->lat_empty[s0]));
+            tc_commit(smem_u32(&bars->lat_empty[s1]));
+          }
+          __syncwarp();
         }
-        tc_fence_after();
-        if (lane == 0) {
-          const uint32_t a_addr = smem_u32(s_lat + s0 * kSlot);
-          const uint32_t b_addr = smem_u32(s_p);
-          for (int k = 0; k < ksteps; ++k)
-            tc_mma(tmem_base + blk * N, make_desc(a_addr + k * 2048, kSlot, 1024, 2),
-                   make_desc(b_addr + k * 256, 128, 2048, 0), idesc_pv, (tile | k) != 0);
+      } else if (lane == 0) {
+        for (int blk = 0; blk < NB && ok; ++blk) {
+          const unsigned n = n0 + NKC + 2 * blk, s0 = n % kLatSlots, s1 = (n + 1) % kLatSlots;
+          if ((blk & 1) == 0) EKV_STAMP(1, 500 + blk, tile);
+          ok = mbar_wait(smem_u32(&bars->lat_full[s0]), (n / kLatSlots) & 1, s_abort) &&
+               mbar_wait(smem_u32(&bars->lat_full[s1]), ((n + 1) / kLatSlots) & 1, s_abort);
+          if (!ok) break;
+          const uint64_t da = make_desc(smem_u32(s_lat + s0 * kSlot), kSlot, 1024, 2), db = make_desc(p_addr, 128, 2048, 0);
+#pragma unroll
+          for (int k = 0; k < 8; ++k)      // +16 tokens: +2048 bytes in A (+128), +256 bytes in P (+16)
+            if (k < ksteps) tc_mma(tmem_base + blk * N, da + 128 * k, db + 16 * k, idesc_pv, (tile | k) != 0);
           tc_commit(smem_u32(&bars->lat_empty[s0]));
           tc_commit(smem_u32(&bars->lat_empty[s1]));
         }
-        __syncwarp();
-        lat_n += 2;
       }
-      if (!ok) break;
-      if (lane == 0) {
+      if (lane == 0 && ok) {
         tc_commit(smem_u32(&bars->pv_done));
         EKV_STAMP(1, 22, tile);
       }
-      __syncwarp();
+      lat_n = n0 + 2u * (unsigned)NKC;
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     }
   }
   // ============================================================== warps 2-5: softmax

@@ -130,7 +130,7 @@ extern "C" int elitekv_decode(const elitekv_layer* L, const elitekv_cache* cache
   ws.n_workers = kernel == 3 ? ekv_tc2_workers(L) : kernel == 2 ? ekv_tc_workers(L) : 0;
   cudaStream_t st = (cudaStream_t)stream;
   if (kernel == 3 || kernel == 2)
-    rc = ekv_launch_plan_balanced(seq_lens, B, kernel == 3 ? 32 : 64, ws.n_workers, max_items, ws.items,
+    rc = ekv_launch_plan_balanced(seq_lens, B, kernel == 3 ? 32 : 128, ws.n_workers, max_items, ws.items,
                                   ws.seq_first, ws.worker_first, ws.counters, ws.n_counters, st);
   else
     rc = ekv_launch_plan(seq_lens, B, kernel == 2 ? 128 : ELITEKV_TILE_TOKENS, max_items, ws.items,

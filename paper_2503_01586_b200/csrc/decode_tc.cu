@@ -10,22 +10,28 @@
 // from the 128-byte-swizzled shared-memory tiles that TMA writes; the narrow per-head rope dot
 // product stays on FP32 FMA in the softmax threads.
 //
-// The absorbed queries of a sequence (n_h x d_c bf16, 96 KB at d_c = 1536) must stay resident
-// beside the token tile, which leaves no room to keep a whole 128 x d_c tile in shared memory.
-// The tile is therefore streamed twice through a small ring of [128 tokens x 64 coords] chunks:
-// pass A accumulates S over the latent axis, the softmax threads turn S (+ rope part) into P,
-// pass B streams the same chunks again (they were just read, so they come from L2, not HBM)
-// and accumulates P-weighted latents into the TMEM-resident output.  HBM sees every cache byte
-// once per step.
+// The absorbed queries of a sequence (n_h x d_c bf16, 96 KB at d_c = 1536) and a whole
+// 128 x d_c token tile do not fit in shared memory together, so nothing is kept resident: the
+// tile is streamed twice through a ring of slots, each slot holding one [128 tokens x 64 coords]
+// latent chunk and, in pass A, the matching [n_h x 64] chunk of the absorbed queries (which
+// stays L2-resident).  Pass A accumulates S over the latent axis, the softmax threads turn S
+// (+ rope part) into P, pass B streams the same latent chunks again and accumulates P-weighted
+// latents into the TMEM-resident output.  L2 eviction hints (keep after pass A, drop after pass
+// B) make the second read an L2 hit, so HBM sees every cache byte once per step.
 //
-// One thread block (192 threads) per plan item:
-//   warp 0    TMA producer (one lane): absorbed queries once, then per tile the latent chunks
-//             of pass A interleaved with the rope boxes, then the latent chunks of pass B
-//   warp 1    TMEM allocation; one lane issues every tcgen05.mma and the commits that free
-//             ring slots; the warp zero-fills token rows past the end of the sequence
-//   warps 2-5 one thread per token row: rope dot products, S from TMEM, masking, running
-//             max / sum in base 2 with a lazily moved reference max, P to shared memory in the
-//             layout the second GEMM wants, TMEM rescale when the reference moves, epilogue
+// A block is a persistent worker: it walks the items of the balanced plan that fall into its
+// share of the batch's tiles and writes one partial result (m, l, acc) per item.  Layers whose
+// fp32 output does not fit TMEM's 512 columns for 32 heads (d_c > 1920 or n_h != 32) run with
+// 16 heads per block; the head groups of an item are adjacent blocks so that they share L2.
+//
+// Roles (288 threads):
+//   warps 0,7,8  latent TMA producers (one lane each, ring uses dealt round-robin)
+//   warp 6       rope TMA producer
+//   warp 1       TMEM allocation; lane 0 issues every tcgen05.mma and the commits that free ring
+//                slots; the warp zero-fills token rows past the end of the sequence
+//   warps 2-5    one thread per token row: rope dot products, S from TMEM, masking, running
+//                max / sum in base 2 with a lazily moved reference max, P to shared memory in the
+//                layout the second GEMM wants, TMEM rescale when the reference moves, epilogue
 // Every wait is bounded: when a limit is hit the block records ELITEKV_ERR_TIMEOUT in the
 // layer's status word, stops issuing work, frees its TMEM and leaves.
 #include "tc_ptx.cuh"

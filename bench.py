@@ -188,6 +188,20 @@ def run_reference(args, w: gen.Workload):
     print(json.dumps(line))
 
 
+def max_over_ranks(dist, values, device):
+    """Element-wise maximum of per-rank timings (ranks are independent replicas: the job is as
+    slow as its slowest rank).  `dist` is torch.distributed or None for a single process."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.tolist()]
+
+
+def aggregate_value(world: int, batch_per_rank: int, ms_per_step: float) -> float:
+    """Whole-job decode tokens/s: every rank advances its own batch each step."""
+    return world * batch_per_rank / (ms_per_step * 1e-3)
+
+
 # ---------------------------------------------------------------------------------------------
 # GPU leg
 # ---------------------------------------------------------------------------------------------
@@ -381,10 +395,7 @@ def run_gpu(args, w: gen.Workload):
             comparator = None
 
     # ---- reduce over ranks
-    t = torch.tensor([total_ms, e2e_s, kern_ms], dtype=torch.float64, device=device)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, e2e_s, kern_ms = (float(x) for x in t.tolist())
+    total_ms, e2e_s, kern_ms = max_over_ranks(dist, [total_ms, e2e_s, kern_ms], device)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -392,7 +403,7 @@ def run_gpu(args, w: gen.Workload):
 
     peak, peak_kind = measured_peaks()
     ms_per_step = total_ms / args.steps
-    value = world * w.B / (ms_per_step * 1e-3)
+    value = aggregate_value(world, w.B, ms_per_step)
     kern_avg_s = (kern_ms / max(kern_n, 1)) * 1e-3
     achieved = cache_bytes / kern_avg_s / 1e9 if kern_n else None
     line = {

@@ -349,7 +349,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       for (int cb = 0; cb < NRB; ++cb) {
         if (!ok) break;
         const unsigned slot = rope_n % kRopeSlots;
-        ok = mbar_wait(smem_u32(&bars->rope_full[slot]), (rope_n / kRopeSlots) & 1, s_abort);
+        ok = mbar_wait_group(smem_u32(&bars->rope_full[slot]), (rope_n / kRopeSlots) & 1, s_abort, threadIdx.x == 64, 2, kSoftmaxThreads);
         if (!ok) break;
         const unsigned char* rowp = s_rope + slot * kChunkBytes + trow * 128;
         float part[HPB];
@@ -380,7 +380,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       if (!ok) break;
       if (threadIdx.x == 64) EKV_STAMP(2, 30, tile);
       // ---- latent part from TMEM
-      ok = mbar_wait(smem_u32(&bars->s_full), (tbase + tile) & 1, s_abort);
+      ok = mbar_wait_group(smem_u32(&bars->s_full), (tbase + tile) & 1, s_abort, threadIdx.x == 64, 2, kSoftmaxThreads);
       if (!ok) break;
       tc_fence_after();
       if (threadIdx.x == 64) EKV_STAMP(2, 31, tile);
@@ -456,7 +456,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
     }
 
     // ---- epilogue: partial output and softmax statistics of this item
-    if (ok) ok = mbar_wait(smem_u32(&bars->pv_done), (tbase + n_tiles - 1) & 1, s_abort);
+    ok = mbar_wait_group(smem_u32(&bars->pv_done), (tbase + n_tiles - 1) & 1, s_abort, threadIdx.x == 64, 2, kSoftmaxThreads) && ok;
     if (ok) {
       tc_fence_after();
       float* pa = a.part_acc + ((size_t)item * a.n_h + h0) * d_c;

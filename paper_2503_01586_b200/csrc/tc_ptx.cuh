@@ -60,6 +60,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   *abort_flag = 1;
   return false;
 }
+// Group wait for long waits of many threads: one leader polls the mbarrier, the others sleep in
+// a hardware named barrier (polling threads hammer the shared-memory pipe that feeds the tensor
+// core).  Afterwards every thread confirms the phase itself (one immediate try_wait = its own
+// acquire); false means the block is aborting.  All `n` threads of barrier `id` must call it.
+__device__ __forceinline__ bool mbar_wait_group(uint32_t bar, uint32_t parity, volatile int* abort_flag, bool leader,
+                                                int id, int n) {
+  if (leader) (void)mbar_wait(bar, parity, abort_flag);
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory");
+  return mbar_try_wait(bar, parity);
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"

@@ -25,10 +25,16 @@
 // 16 heads per block; the head groups of an item are adjacent blocks so that they share L2.
 //
 // Roles (288 threads):
-//   warps 0,7,8  latent TMA producers (one lane each, ring uses dealt round-robin)
+//   warps 0,7,8  latent TMA producers (ring uses dealt round-robin)
 //   warp 6       rope TMA producer
-//   warp 1       TMEM allocation; lane 0 issues every tcgen05.mma and the commits that free ring
-//                slots; the warp zero-fills token rows past the end of the sequence
+//   warp 1       TMEM allocation and MMA issue.  The tensor core finishes a 128 x N x 16 MMA in
+//                about 40 clocks (the time to read the 4 KB A operand from shared memory); the
+//                issuing code keeps up only when it runs warp-uniformly with the tcgen05.mma
+//                itself under an elected lane and the descriptor words built from precomputed
+//                halves plus small immediates (measured: 42 clocks per MMA, against 61 when a
+//                single diverged lane runs the same loop and ~100 with per-MMA 64-bit
+//                descriptor assembly).  The warp also zero-fills token rows past the end of
+//                the sequence.  Producer warps issue TMA the same way.
 //   warps 2-5    one thread per token row: rope dot products, S from TMEM, masking, running
 //                max / sum in base 2 with a lazily moved reference max, P to shared memory in the
 //                layout the second GEMM wants, TMEM rescale when the reference moves, epilogue
@@ -42,8 +48,8 @@ constexpr int kTile = 128;            // tokens per tile
 constexpr int kChunkBytes = 16384;    // [128 tokens][64 bf16] with 128-byte rows
 constexpr int kLatSlots = 8;          // ring slots: one latent chunk + the matching query chunk each
 constexpr int kRopeSlots = 3;
-constexpr int kThreads = 288;         // warp 0 latent loads, 1 MMA, 2-5 softmax, 6 rope loads, 7-8 latent loads
-constexpr int kProdWarps = 3;         // latent-load warps: 0, 7, 8 (one issuing lane each)
+constexpr int kThreads = 288;         // warps 0,7,8 latent loads, 1 MMA, 2-5 softmax, 6 rope loads
+constexpr int kProdWarps = 3;         // latent-load warps: 0, 7, 8
 constexpr int kSoftmaxThreads = 128;
 
 struct TcArgs {
@@ -162,54 +168,57 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   __syncthreads();
 
   // ============================================================== warps 0, 7, 8: latent TMA producers; warp 6: rope
-  // One thread can issue a TMA load only every ~0.17 us (wait + expect_tx + issue), i.e. about
-  // 47 GB/s of 8 KB boxes per SM, and two issuing warps were measured to double that.  The
-  // latent ring uses are therefore dealt round-robin to kProdWarps warps.
+  // Each producer warp runs its loop warp-uniformly and one elected lane issues expect_tx and the
+  // TMA loads.  One warp can issue a box only every ~0.17 us, so the latent ring uses are dealt
+  // round-robin to kProdWarps warps.
   if (warp == 0 || warp >= 6) {
     const bool rope_role = warp == 6;
     const int prod = warp == 0 ? 0 : warp - 6;          // latent producer index
-    if (lane == 0) {
-      // L2 priorities: a latent chunk read in pass A is read again soon (pass B) -> keep; after
-      // pass B, and for rope rows, the data is dead -> first to go; the queries are re-read by
-      // every tile of the sequence -> keep
-      const uint64_t pol_keep = make_l2_policy_evict_last(), pol_drop = make_l2_policy_evict_first();
-      bool ok = true;
-      for (int tile = 0; tile < n_tiles && ok; ++tile) {
-        const int t_abs = tok0 + tile * kTile;
-        const int nvalid = min(kTile, ntok - tile * kTile);
-        const int halves = nvalid > 64 ? 2 : 1;
-        long long row[2];
-        for (int hf = 0; hf < 2; ++hf) {
-          const int t = t_abs + 64 * hf;
-          if (a.page_table == nullptr) {
-            row[hf] = (long long)seq * a.max_ctx + t;
-          } else {
-            const int pi = t >> a.page_shift;
-            int page = (hf < halves && pi < a.max_pages_per_seq)
-                           ? a.page_table[(long long)seq * a.max_pages_per_seq + pi] : 0;
-            if (page < 0 || page >= a.num_pages) {
-              if (hf < halves && rope_role) ekv_record(a.status, ELITEKV_ERR_BAD_PAGE, seq, page);
-              page = 0;
-            }
-            row[hf] = ((long long)page << a.page_shift) + (t & a.page_mask);
+    // L2 priorities: a latent chunk read in pass A is read again soon (pass B) -> keep; after
+    // pass B, and for rope rows, the data is dead -> first to go; the queries are re-read by
+    // every tile of the sequence -> keep
+    const uint64_t pol_keep = make_l2_policy_evict_last(), pol_drop = make_l2_policy_evict_first();
+    bool ok = true;
+    for (int tile = 0; tile < n_tiles && ok; ++tile) {
+      // cache rows of the two 64-token halves of the tile; `whole` = adjacent (one 128-row box)
+      const int t_abs = tok0 + tile * kTile;
+      const int nvalid = min(kTile, ntok - tile * kTile);
+      const int halves = nvalid > 64 ? 2 : 1;
+      long long row[2];
+      for (int hf = 0; hf < 2; ++hf) {
+        const int t = t_abs + 64 * hf;
+        if (a.page_table == nullptr) {
+          row[hf] = (long long)seq * a.max_ctx + t;
+        } else {
+          const int pi = t >> a.page_shift;
+          int page = (hf < halves && pi < a.max_pages_per_seq)
+                         ? a.page_table[(long long)seq * a.max_pages_per_seq + pi] : 0;
+          if (page < 0 || page >= a.num_pages) {
+            if (hf < halves && rope_role && lane == 0) ekv_record(a.status, ELITEKV_ERR_BAD_PAGE, seq, page);
+            page = 0;
           }
+          row[hf] = ((long long)page << a.page_shift) + (t & a.page_mask);
         }
-        // both 64-row halves adjacent in the cache: one 128-row box instead of two
-        const bool whole = halves == 2 && row[1] == row[0] + 64;
-        if (!rope_role) {
-          // ring uses of this tile: NKC chunks of pass A (each with its query chunk), then the
-          // same NKC chunks again for pass B (served by L2)
-          for (int u = prod; u < 2 * NKC && ok; u += kProdWarps) {
-            const bool with_q = u < NKC;
-            const int kc = with_q ? u : u - NKC;
-            const unsigned n = lat_n + (unsigned)u, slot = n % kLatSlots;
-            ok = mbar_wait(smem_u32(&bars->lat_empty[slot]), ((n / kLatSlots) & 1) ^ 1, s_abort);
+      }
+      const bool whole = halves == 2 && row[1] == row[0] + 64;
+      if (!rope_role) {
+        // ring uses of this tile: NKC chunks of pass A (each with its query chunk), then the
+        // same NKC chunks again for pass B (served by L2)
+        for (int u = prod; u < 2 * NKC; u += kProdWarps) {
+          const bool with_q = u < NKC;
+          const int kc = with_q ? u : u - NKC;
+          const unsigned n = lat_n + (unsigned)u, slot = n % kLatSlots;
+          const uint32_t eb = smem_u32(&bars->lat_empty[slot]), epar = ((n / kLatSlots) & 1) ^ 1;
+          if (!mbar_test_wait(eb, epar)) {
+            ok = __all_sync(0xffffffffu, mbar_spin(eb, epar, s_abort, 1));
             if (!ok) break;
+          }
+          if (elect_one()) {
             const uint32_t fb = smem_u32(&bars->lat_full[slot]);
             mbar_expect_tx(fb, (uint32_t)(halves * 8192 + (with_q ? N * 128 : 0)));
             if (with_q)   // the sequence's absorbed queries for these 64 latent coordinates (L2-resident)
               tma_load_2d_hint(smem_u32(s_lat + slot * kSlot + kChunkBytes), &map_q, kc * 64, seq * a.n_h + h0, fb, pol_keep);
-            if (prod == 0) EKV_STAMP(0, (with_q ? 100 : 200) + kc, tile);
+            if (prod == 0 && kc == 0) EKV_STAMP(0, with_q ? 100 : 200, tile);
             const uint64_t pol = with_q ? pol_keep : pol_drop;
             if (whole) {
               tma_load_2d_hint(smem_u32(s_lat + slot * kSlot), &map_lat128, kc * 64, (int)row[0], fb, pol);
@@ -218,13 +227,19 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
                 tma_load_2d_hint(smem_u32(s_lat + slot * kSlot + hf * 8192), &map_lat, kc * 64, (int)row[hf], fb, pol);
             }
           }
-          lat_n += 2u * (unsigned)NKC;
-        } else {
-          // warp 6: the rope boxes of the tile
-          for (int cb = 0; cb < NRB && ok; ++cb) {
-            const unsigned slot = rope_n % kRopeSlots;
-            ok = mbar_wait(smem_u32(&bars->rope_empty[slot]), ((rope_n / kRopeSlots) & 1) ^ 1, s_abort);
+          __syncwarp();
+        }
+        lat_n += 2u * (unsigned)NKC;
+      } else {
+        // warp 6: the rope boxes of the tile
+        for (int cb = 0; cb < NRB; ++cb) {
+          const unsigned slot = rope_n % kRopeSlots;
+          const uint32_t eb = smem_u32(&bars->rope_empty[slot]), epar = ((rope_n / kRopeSlots) & 1) ^ 1;
+          if (!mbar_test_wait(eb, epar)) {
+            ok = __all_sync(0xffffffffu, mbar_spin(eb, epar, s_abort, 2));
             if (!ok) break;
+          }
+          if (elect_one()) {
             const uint32_t fb = smem_u32(&bars->rope_full[slot]);
             mbar_expect_tx(fb, (uint32_t)(halves * 8192));
             if (whole) {
@@ -233,98 +248,115 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
               for (int hf = 0; hf < halves; ++hf)
                 tma_load_2d_hint(smem_u32(s_rope + slot * kChunkBytes + hf * 8192), &map_rope, h0 * R2 + cb * 64, (int)row[hf], fb, pol_drop);
             }
-            ++rope_n;
           }
+          __syncwarp();
+          ++rope_n;
         }
       }
     }
   }
   // ============================================================== warp 1: MMA issuer
-  // Lane 0 alone waits, issues and commits (per-chunk warp-wide synchronisation costs as much as
-  // the MMAs themselves); the other lanes only help to zero a ragged tail.
+  // The whole warp walks the ring (waits, descriptor arithmetic, slot bookkeeping are
+  // warp-uniform) and an elected lane issues the MMAs and the commits that free ring slots;
+  // all lanes help to zero a ragged tail.
   else if (warp == 1) {
     constexpr uint32_t idesc_s = make_idesc(128, N, 0, 0);    // S = C . Q^T   (both K-major)
     constexpr uint32_t idesc_pv = make_idesc(128, N, 1, 1);   // acc = C^T . P (both MN-major)
+    constexpr uint32_t hi_sw = desc_hi(1024, 2);              // 128-byte swizzle, 1024 bytes between 8-row groups
+    constexpr uint32_t hi_p = desc_hi(2048, 0);               // P tile: no swizzle, 2048 bytes between 8-head groups
+    constexpr uint32_t kSlot16 = kSlot >> 4;
+    const uint32_t lat16 = smem_u32(s_lat) >> 4;              // ring base in 16-byte units
+    const uint32_t lo_p = desc_lo(smem_u32(s_p), 128);
+    const uint32_t full0 = smem_u32(&bars->lat_full[0]), empty0 = smem_u32(&bars->lat_empty[0]);
     bool ok = true;
     for (int tile = 0; tile < n_tiles && ok; ++tile) {
       const int nvalid = min(kTile, ntok - tile * kTile);
       const int ksteps = (nvalid + 15) >> 4;
       const int zero_from = nvalid, zero_to = ksteps * 16;
       const unsigned n0 = lat_n;                 // first ring use of this tile
-      if (lane == 0) {
-        // ---- pass A
-        for (int kc = 0; kc < NKC && ok; ++kc) {
-          const unsigned n = n0 + kc, slot = n % kLatSlots;
-          if ((kc & 3) == 0) EKV_STAMP(1, 300 + kc, tile);
-          ok = mbar_wait(smem_u32(&bars->lat_full[slot]), (n / kLatSlots) & 1, s_abort);
+      // ---- pass A: NKC chunks, 4 K-steps of 16 latent coordinates each
+      unsigned slot = n0 % kLatSlots, par = (n0 / kLatSlots) & 1;
+      if (elect_one()) EKV_STAMP(1, 300, tile);
+      for (int kc = 0; kc < NKC; ++kc) {
+        const uint32_t fb = full0 + slot * 8;
+        if (!mbar_test_wait(fb, par)) {
+          ok = __all_sync(0xffffffffu, mbar_spin(fb, par, s_abort, 3));
           if (!ok) break;
-          const uint32_t a_addr = smem_u32(s_lat + slot * kSlot);
-          const uint64_t da = make_desc(a_addr, 16, 1024, 2), db = make_desc(a_addr + kChunkBytes, 16, 1024, 2);
-#pragma unroll
-          for (int k = 0; k < 4; ++k)      // +32 bytes along K per step = +2 in the address field
-            tc_mma(tmem_s, da + 2 * k, db + 2 * k, idesc_s, (kc | k) != 0);
-          tc_commit(smem_u32(&bars->lat_empty[slot]));
         }
-        if (ok) {
-          tc_commit(smem_u32(&bars->s_full));
-          EKV_STAMP(1, 20, tile);
-          // ---- wait for P (and the rescaled output) of this tile
-          ok = mbar_wait(smem_u32(&bars->p_ready), (tbase + tile) & 1, s_abort);
-          tc_fence_after();
-          EKV_STAMP(1, 21, tile);
+        const uint32_t la = (lat16 + slot * kSlot16) | (1u << 16), lb = la + (kChunkBytes >> 4);
+        if (elect_one()) {
+          tc_mma_w(tmem_s, la, hi_sw, lb, hi_sw, idesc_s, kc != 0);
+          tc_mma_w(tmem_s, la + 2, hi_sw, lb + 2, hi_sw, idesc_s, 1);     // +32 bytes along K per step
+          tc_mma_w(tmem_s, la + 4, hi_sw, lb + 4, hi_sw, idesc_s, 1);
+          tc_mma_w(tmem_s, la + 6, hi_sw, lb + 6, hi_sw, idesc_s, 1);
+          tc_commit(empty0 + slot * 8);
         }
+        __syncwarp();
+        if (++slot == kLatSlots) { slot = 0; par ^= 1; }
       }
-      // ---- pass B
-      const uint32_t p_addr = smem_u32(s_p);
-      if (zero_to > zero_from) {
-        // ragged end of a sequence: rows past its last token inside the last 16-token step are
-        // made exact zeros (warp-cooperatively) so that zero-probability rows cannot inject
-        // NaN/Inf bit patterns
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        for (int blk = 0; blk < NB && ok; ++blk) {
-          const unsigned n = n0 + NKC + 2 * blk, s0 = n % kLatSlots, s1 = (n + 1) % kLatSlots;
-          if (lane == 0)
-            ok = mbar_wait(smem_u32(&bars->lat_full[s0]), (n / kLatSlots) & 1, s_abort) &&
-                 mbar_wait(smem_u32(&bars->lat_full[s1]), ((n + 1) / kLatSlots) & 1, s_abort);
-          ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) break;
+      if (elect_one()) {
+        tc_commit(smem_u32(&bars->s_full));
+        EKV_STAMP(1, 20, tile);
+      }
+      __syncwarp();
+      // ---- wait for P (and the rescaled output) of this tile
+      ok = __all_sync(0xffffffffu, mbar_spin(smem_u32(&bars->p_ready), (tbase + tile) & 1, s_abort, 4));
+      if (!ok) break;
+      tc_fence_after();
+      if (elect_one()) EKV_STAMP(1, 21, tile);
+      // ---- pass B: NB output blocks of 128 latent coordinates = one even/odd slot pair each
+      const unsigned nb0 = n0 + NKC;
+      slot = nb0 % kLatSlots;
+      par = (nb0 / kLatSlots) & 1;
+      for (int blk = 0; blk < NB; ++blk) {
+        const uint32_t fb = full0 + slot * 8;
+        if (!(mbar_test_wait(fb, par) && mbar_test_wait(fb + 8, par))) {
+          ok = __all_sync(0xffffffffu, mbar_spin(fb, par, s_abort, 5) && mbar_spin(fb + 8, par, s_abort, 5));
           if (!ok) break;
+        }
+        if (zero_to > zero_from) {
+          // ragged end of a sequence: rows past its last token inside the last 16-token step are
+          // made exact zeros so that zero-probability rows cannot inject NaN/Inf bit patterns
           for (int e = lane; e < (zero_to - zero_from) * 16; e += 32) {
             const int rrow = zero_from + (e >> 4), c16 = e & 15;
-            unsigned char* p = s_lat + (c16 < 8 ? s0 : s1) * kSlot + rrow * 128 + (c16 & 7) * 16;
+            unsigned char* p = s_lat + (slot + (c16 >> 3)) * kSlot + rrow * 128 + (c16 & 7) * 16;
             *(uint4*)p = make_uint4(0, 0, 0, 0);
           }
           fence_proxy_async();
           __syncwarp();
-          if (lane == 0) {
-            const uint64_t da = make_desc(smem_u32(s_lat + s0 * kSlot), kSlot, 1024, 2), db = make_desc(p_addr, 128, 2048, 0);
+        }
+        // A: two 64-coordinate atoms one slot apart; +16 tokens = +2048 bytes in A, +256 bytes in P
+        const uint32_t la = (lat16 + slot * kSlot16) | (kSlot16 << 16);
+        const uint32_t d = tmem_base + blk * N;
+        if (elect_one()) {
+          if (ksteps == 8) {
+            tc_mma_w(d, la, hi_sw, lo_p, hi_p, idesc_pv, tile != 0);
+            tc_mma_w(d, la + 128, hi_sw, lo_p + 16, hi_p, idesc_pv, 1);
+            tc_mma_w(d, la + 256, hi_sw, lo_p + 32, hi_p, idesc_pv, 1);
+            tc_mma_w(d, la + 384, hi_sw, lo_p + 48, hi_p, idesc_pv, 1);
+            tc_mma_w(d, la + 512, hi_sw, lo_p + 64, hi_p, idesc_pv, 1);
+            tc_mma_w(d, la + 640, hi_sw, lo_p + 80, hi_p, idesc_pv, 1);
+            tc_mma_w(d, la + 768, hi_sw, lo_p + 96, hi_p, idesc_pv, 1);
+            tc_mma_w(d, la + 896, hi_sw, lo_p + 112, hi_p, idesc_pv, 1);
+          } else {      // short last tile: only the loaded token rows
             for (int k = 0; k < ksteps; ++k)
-              tc_mma(tmem_base + blk * N, da + 128 * k, db + 16 * k, idesc_pv, (tile | k) != 0);
-            tc_commit(smem_u32(&bars->lat_empty[s0]));
-            tc_commit(smem_u32(&bars->lat_empty[s1]));
+              tc_mma_w(d, la + 128 * k, hi_sw, lo_p + 16 * k, hi_p, idesc_pv, (tile | k) != 0);
           }
-          __syncwarp();
+          tc_commit(empty0 + slot * 8);
+          tc_commit(empty0 + slot * 8 + 8);
         }
-      } else if (lane == 0) {
-        for (int blk = 0; blk < NB && ok; ++blk) {
-          const unsigned n = n0 + NKC + 2 * blk, s0 = n % kLatSlots, s1 = (n + 1) % kLatSlots;
-          if ((blk & 1) == 0) EKV_STAMP(1, 500 + blk, tile);
-          ok = mbar_wait(smem_u32(&bars->lat_full[s0]), (n / kLatSlots) & 1, s_abort) &&
-               mbar_wait(smem_u32(&bars->lat_full[s1]), ((n + 1) / kLatSlots) & 1, s_abort);
-          if (!ok) break;
-          const uint64_t da = make_desc(smem_u32(s_lat + s0 * kSlot), kSlot, 1024, 2), db = make_desc(p_addr, 128, 2048, 0);
-#pragma unroll
-          for (int k = 0; k < 8; ++k)      // +16 tokens: +2048 bytes in A (+128), +256 bytes in P (+16)
-            if (k < ksteps) tc_mma(tmem_base + blk * N, da + 128 * k, db + 16 * k, idesc_pv, (tile | k) != 0);
-          tc_commit(smem_u32(&bars->lat_empty[s0]));
-          tc_commit(smem_u32(&bars->lat_empty[s1]));
-        }
+        __syncwarp();
+        slot += 2;
+        if (slot >= kLatSlots) { slot -= kLatSlots; par ^= 1; }
       }
-      if (lane == 0 && ok) {
+      if (!ok) break;
+      if (elect_one()) {
         tc_commit(smem_u32(&bars->pv_done));
         EKV_STAMP(1, 22, tile);
       }
+      __syncwarp();
       lat_n = n0 + 2u * (unsigned)NKC;
-      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     }
   }
   // ============================================================== warps 2-5: softmax
@@ -349,7 +381,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       for (int cb = 0; cb < NRB; ++cb) {
         if (!ok) break;
         const unsigned slot = rope_n % kRopeSlots;
-        ok = mbar_wait_group(smem_u32(&bars->rope_full[slot]), (rope_n / kRopeSlots) & 1, s_abort, threadIdx.x == 64, 2, kSoftmaxThreads);
+        ok = mbar_wait_group(smem_u32(&bars->rope_full[slot]), (rope_n / kRopeSlots) & 1, s_abort, threadIdx.x == 64, 2, kSoftmaxThreads, 6);
         if (!ok) break;
         const unsigned char* rowp = s_rope + slot * kChunkBytes + trow * 128;
         float part[HPB];
@@ -380,7 +412,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       if (!ok) break;
       if (threadIdx.x == 64) EKV_STAMP(2, 30, tile);
       // ---- latent part from TMEM
-      ok = mbar_wait_group(smem_u32(&bars->s_full), (tbase + tile) & 1, s_abort, threadIdx.x == 64, 2, kSoftmaxThreads);
+      ok = mbar_wait_group(smem_u32(&bars->s_full), (tbase + tile) & 1, s_abort, threadIdx.x == 64, 2, kSoftmaxThreads, 7);
       if (!ok) break;
       tc_fence_after();
       if (threadIdx.x == 64) EKV_STAMP(2, 31, tile);
@@ -456,7 +488,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
     }
 
     // ---- epilogue: partial output and softmax statistics of this item
-    ok = mbar_wait_group(smem_u32(&bars->pv_done), (tbase + n_tiles - 1) & 1, s_abort, threadIdx.x == 64, 2, kSoftmaxThreads) && ok;
+    ok = mbar_wait_group(smem_u32(&bars->pv_done), (tbase + n_tiles - 1) & 1, s_abort, threadIdx.x == 64, 2, kSoftmaxThreads, 8) && ok;
     if (ok) {
       tc_fence_after();
       float* pa = a.part_acc + ((size_t)item * a.n_h + h0) * d_c;
@@ -491,12 +523,15 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (*s_abort) break;      // same value in every thread: nobody is inside a wait here
   }
 
   // ============================================================== teardown
+  if (*s_abort) drain_after_abort();
   tc_fence_before();
   __syncthreads();
-  if (threadIdx.x == 0 && *s_abort) ekv_record(a.status, ELITEKV_ERR_TIMEOUT, worker, seq);
+  // detail: worker in the low 16 bits, the code of the wait that gave up above them
+  if (threadIdx.x == 0 && *s_abort) ekv_record(a.status, ELITEKV_ERR_TIMEOUT, worker | (*s_abort << 16), seq);
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");

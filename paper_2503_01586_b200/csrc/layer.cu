@@ -5,6 +5,8 @@
 
 #include <vector>
 
+#include <stdio.h>
+
 #include "common.cuh"
 
 namespace {
@@ -143,6 +145,9 @@ extern "C" int elitekv_check_status(const elitekv_layer* L, elitekv_stream_t str
   EKV_CUDA_OK(cudaMemcpyAsync(h, L->d_status, sizeof(h), cudaMemcpyDeviceToHost, st));
   EKV_CUDA_OK(cudaMemsetAsync(L->d_status, 0, sizeof(h), st));
   EKV_CUDA_OK(cudaStreamSynchronize(st));
+#ifdef EKV_SYNC_EACH
+  if (h[0] != 0) fprintf(stderr, "elitekv status %d detail %d (0x%x) %d count %d\n", h[0], h[1], h[1], h[2], h[3]);
+#endif
   return h[0];
 }
 

@@ -51,22 +51,66 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait; returns false (and raises the block's abort flag) when the limit is hit.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int why = 1);
+// True in exactly one lane of a fully converged warp.  Code that issues tcgen05.mma or TMA runs
+// warp-uniformly with only the instruction itself under this predicate: operands of those
+// instructions then live in uniform registers, which was measured to matter (42 clocks per
+// 128 x 32 x 16 MMA against 61 for the same loop run by a single diverged lane).
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
+// Non-blocking probe of a phase (try_wait may park the thread for a while before it answers).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded busy wait on test_wait for the threads on the critical hand-off path (MMA issuer, TMA
+// producers): same contract as mbar_wait, 16 times the poll budget because a probe is cheap.
+__device__ __forceinline__ bool mbar_spin(uint32_t bar, uint32_t parity, volatile int* abort_flag, int why = 1) {
+#ifdef EKV_NO_SPIN
+  return mbar_wait(bar, parity, abort_flag, why);
+#else
+  for (unsigned i = 0; i < 16u * kWaitLimit; ++i) {
+    if (mbar_test_wait(bar, parity)) return true;
+    if ((i & 4095) == 4095 && *abort_flag) return false;
+  }
+  if (*abort_flag == 0) *abort_flag = why;
+  return false;
+#endif
+}
+// Bounded wait; returns false when the limit is hit (the block's abort flag is then set to `why`,
+// a small positive code that names the wait) or when another thread has already given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int why) {
   for (unsigned i = 0; i < kWaitLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 1023) == 1023 && *abort_flag) return false;
   }
-  *abort_flag = 1;
+  if (*abort_flag == 0) *abort_flag = why;
   return false;
+}
+// After an abort: give copies and MMAs already in flight a bounded time (~0.1 ms) to land before
+// the block frees its tensor memory and its shared memory goes away.
+__device__ __forceinline__ void drain_after_abort() {
+  for (int i = 0; i < 100; ++i) asm volatile("nanosleep.u32 1000;" ::: "memory");
 }
 // Group wait for long waits of many threads: one leader polls the mbarrier, the others sleep in
 // a hardware named barrier (polling threads hammer the shared-memory pipe that feeds the tensor
 // core).  Afterwards every thread confirms the phase itself (one immediate try_wait = its own
 // acquire); false means the block is aborting.  All `n` threads of barrier `id` must call it.
 __device__ __forceinline__ bool mbar_wait_group(uint32_t bar, uint32_t parity, volatile int* abort_flag, bool leader,
-                                                int id, int n) {
-  if (leader) (void)mbar_wait(bar, parity, abort_flag);
+                                                int id, int n, int why = 1) {
+  if (leader) (void)mbar_spin(bar, parity, abort_flag, why);
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory");
   return mbar_try_wait(bar, parity);
 }
@@ -108,6 +152,19 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Same with the descriptors given as 32-bit halves: the high words (stride offset, version,
+// swizzle mode) are constants and the low words (address, leading offset) advance by small
+// immediates, which keeps the issuing thread's instruction stream short.
+__device__ __forceinline__ void tc_mma_w(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                         uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %2};\n\t"
+      "mov.b64 db, {%3, %4};\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
   uint32_t* r = (uint32_t*)v;
@@ -174,6 +231,13 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
   d |= (uint64_t)1 << 46;
   d |= (uint64_t)layout << 61;
   return d;
+}
+// The two 32-bit halves of the same descriptor.
+__host__ __device__ constexpr uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+  return ((saddr >> 4) & 0x3FFF) | (((lbo_bytes >> 4) & 0x3FFF) << 16);
+}
+__host__ __device__ constexpr uint32_t desc_hi(uint32_t sbo_bytes, uint32_t layout) {
+  return ((sbo_bytes >> 4) & 0x3FFF) | (1u << 14) | (layout << 29);
 }
 // Instruction descriptor for kind::f16 with bf16 inputs and fp32 accumulation.
 __host__ __device__ constexpr uint32_t make_idesc(int M, int N, int a_mn_major, int b_mn_major) {

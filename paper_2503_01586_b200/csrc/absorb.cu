@@ -67,17 +67,26 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
     for (int bb = 0; bb < kAbsorbBatch; ++bb) a0[bb] = a1[bb] = 0.f;
     if (k < d_c) {
       const bf16* wp = WukT + (size_t)h * dn * d_c + k;
-#pragma unroll 4
-      for (int i = i_lo; i < i_hi; ++i) {
-        const float2 w = __bfloat1622float2(*(const bf162*)(wp + (size_t)i * d_c));
-        const float4* xr = (const float4*)(q_nope + (size_t)i * kAbsorbBatch);
+      // eight independent weight loads in flight per thread, then their multiply-adds
+      for (int i0 = i_lo; i0 < i_hi; i0 += 8) {
+        float2 w[8];
 #pragma unroll
-        for (int v = 0; v < kAbsorbBatch / 4; ++v) {
-          const float4 x = xr[v];
-          a0[4 * v + 0] = fmaf(x.x, w.x, a0[4 * v + 0]); a1[4 * v + 0] = fmaf(x.x, w.y, a1[4 * v + 0]);
-          a0[4 * v + 1] = fmaf(x.y, w.x, a0[4 * v + 1]); a1[4 * v + 1] = fmaf(x.y, w.y, a1[4 * v + 1]);
-          a0[4 * v + 2] = fmaf(x.z, w.x, a0[4 * v + 2]); a1[4 * v + 2] = fmaf(x.z, w.y, a1[4 * v + 2]);
-          a0[4 * v + 3] = fmaf(x.w, w.x, a0[4 * v + 3]); a1[4 * v + 3] = fmaf(x.w, w.y, a1[4 * v + 3]);
+        for (int j = 0; j < 8; ++j)
+          w[j] = i0 + j < i_hi ? __bfloat1622float2(__ldg((const bf162*)(wp + (size_t)(i0 + j) * d_c)))
+                               : make_float2(0.f, 0.f);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (i0 + j < i_hi) {
+            const float4* xr = (const float4*)(q_nope + (size_t)(i0 + j) * kAbsorbBatch);
+#pragma unroll
+            for (int v = 0; v < kAbsorbBatch / 4; ++v) {
+              const float4 x = xr[v];
+              a0[4 * v + 0] = fmaf(x.x, w[j].x, a0[4 * v + 0]); a1[4 * v + 0] = fmaf(x.x, w[j].y, a1[4 * v + 0]);
+              a0[4 * v + 1] = fmaf(x.y, w[j].x, a0[4 * v + 1]); a1[4 * v + 1] = fmaf(x.y, w[j].y, a1[4 * v + 1]);
+              a0[4 * v + 2] = fmaf(x.z, w[j].x, a0[4 * v + 2]); a1[4 * v + 2] = fmaf(x.z, w[j].y, a1[4 * v + 2]);
+              a0[4 * v + 3] = fmaf(x.w, w[j].x, a0[4 * v + 3]); a1[4 * v + 3] = fmaf(x.w, w[j].y, a1[4 * v + 3]);
+            }
+          }
         }
       }
     }

@@ -24,6 +24,7 @@ constexpr int kFK = 128;         // latent slice
 constexpr int kFD = 128;         // head dim
 constexpr int kFThreads = 256;
 constexpr int kFI = 16;          // items per sequence whose merge weights are staged in shared memory
+constexpr int kFStage = 512;     // items per sequence group whose (m, l) are staged in shared memory
 
 __global__ void __launch_bounds__(kFThreads)
 combine_fast_kernel(const float* __restrict__ part_acc, const float* __restrict__ part_ml,
@@ -35,18 +36,20 @@ combine_fast_kernel(const float* __restrict__ part_acc, const float* __restrict_
   __shared__ __align__(16) float s_x[kFB][kFK];         // 8 KB merged latent outputs
   __shared__ float s_M[kFB], s_invL[kFB];
   __shared__ float s_wt[kFB][kFI];
+  __shared__ float2 s_ml[kFStage];
   __shared__ int s_first[kFB + 1];
   __shared__ int s_last;
   const int h = blockIdx.x, slice = blockIdx.y, n_slices = gridDim.y;
   const int k0 = slice * kFK;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-  // W_uv[k0 + k][h*128 + d] -> shared, 16 bytes per thread per step
+  // W_uv[k0 + k][h*128 + d] -> shared, 16-byte asynchronous copies that land while the softmax
+  // statistics of the first group are worked out
   for (int e = tid; e < kFK * (kFD / 8); e += kFThreads) {
     const int k = e / (kFD / 8), v = e % (kFD / 8);
-    *(uint4*)&s_w[k][v * 8] =
-        __ldg((const uint4*)(Wuv + (size_t)(k0 + k) * n_h * kFD + (size_t)h * kFD + v * 8));
+    cp_async16(&s_w[k][v * 8], Wuv + (size_t)(k0 + k) * n_h * kFD + (size_t)h * kFD + v * 8);
   }
+  cp_async_commit();
 
   const int n_groups = (B + kFB - 1) / kFB;
   for (int g = 0; g < n_groups; ++g) {
@@ -54,16 +57,24 @@ combine_fast_kernel(const float* __restrict__ part_acc, const float* __restrict_
     __syncthreads();
     if (tid <= nb) s_first[tid] = seq_first[b0 + tid];
     __syncthreads();
+    // (m, l) of the group's items for this head: one trip to global memory, then shared
+    const int gi0 = s_first[0], gin = s_first[nb] - gi0;
+    for (int e = tid; e < min(gin, kFStage); e += kFThreads)
+      s_ml[e] = __ldg((const float2*)(part_ml + ((size_t)(gi0 + e) * n_h + h) * 2));
+    __syncthreads();
+    auto item_ml = [&](int i) -> float2 {
+      return i - gi0 < kFStage ? s_ml[i - gi0] : __ldg((const float2*)(part_ml + ((size_t)i * n_h + h) * 2));
+    };
     // softmax statistics per sequence: one warp each
     for (int bb = warp; bb < nb; bb += kFThreads / 32) {
       const int i0 = s_first[bb], i1 = s_first[bb + 1];
       float M = -INFINITY;
-      for (int i = i0 + lane; i < i1; i += 32) M = fmaxf(M, part_ml[((size_t)i * n_h + h) * 2]);
+      for (int i = i0 + lane; i < i1; i += 32) M = fmaxf(M, item_ml(i).x);
       M = warp_max(M);
       float Ls = 0.f;
       for (int i = i0 + lane; i < i1; i += 32) {
-        const float* ml = part_ml + ((size_t)i * n_h + h) * 2;
-        Ls += ml[1] * exp2f(ml[0] - M);
+        const float2 ml = item_ml(i);
+        Ls += ml.y * exp2f(ml.x - M);
       }
       Ls = warp_sum(Ls);
       if (lane == 0) {
@@ -78,7 +89,7 @@ combine_fast_kernel(const float* __restrict__ part_acc, const float* __restrict_
       float wv = 0.f;
       if (bb < nb) {
         const int i = s_first[bb] + j;
-        if (i < s_first[bb + 1]) wv = exp2f(part_ml[((size_t)i * n_h + h) * 2] - s_M[bb]) * s_invL[bb];
+        if (i < s_first[bb + 1]) wv = exp2f(item_ml(i).x - s_M[bb]) * s_invL[bb];
       }
       s_wt[bb][j] = wv;
     }
@@ -92,15 +103,21 @@ combine_fast_kernel(const float* __restrict__ part_acc, const float* __restrict_
         const float* src = part_acc + ((size_t)i0 * n_h + h) * d_c + k0 + v * 4;
         const size_t stride = (size_t)n_h * d_c;
         const int nfast = min(ni, kFI);
-#pragma unroll 4
-        for (int j = 0; j < nfast; ++j) {
-          const float w = s_wt[bb][j];
-          const float4 p = __ldg((const float4*)(src + (size_t)j * stride));
-          acc.x = fmaf(w, p.x, acc.x); acc.y = fmaf(w, p.y, acc.y);
-          acc.z = fmaf(w, p.z, acc.z); acc.w = fmaf(w, p.w, acc.w);
+        // eight independent 16-byte loads in flight per thread
+        for (int j0 = 0; j0 < nfast; j0 += 8) {
+          float4 p[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            p[j] = j0 + j < nfast ? __ldg((const float4*)(src + (size_t)(j0 + j) * stride)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float w = j0 + j < nfast ? s_wt[bb][j0 + j] : 0.f;
+            acc.x = fmaf(w, p[j].x, acc.x); acc.y = fmaf(w, p[j].y, acc.y);
+            acc.z = fmaf(w, p[j].z, acc.z); acc.w = fmaf(w, p[j].w, acc.w);
+          }
         }
         for (int j = kFI; j < ni; ++j) {     // rare: a sequence cut into more than kFI items
-          const float w = exp2f(part_ml[((size_t)(i0 + j) * n_h + h) * 2] - s_M[bb]) * s_invL[bb];
+          const float w = exp2f(item_ml(i0 + j).x - s_M[bb]) * s_invL[bb];
           const float4 p = __ldg((const float4*)(src + (size_t)j * stride));
           acc.x = fmaf(w, p.x, acc.x); acc.y = fmaf(w, p.y, acc.y);
           acc.z = fmaf(w, p.z, acc.z); acc.w = fmaf(w, p.w, acc.w);
@@ -108,6 +125,7 @@ combine_fast_kernel(const float* __restrict__ part_acc, const float* __restrict_
       }
       *(float4*)&s_x[bb][v * 4] = acc;
     }
+    cp_async_wait<0>();      // the W_uv slice (first group only; later a no-op)
     __syncthreads();
     // [16 x 128] . [128 x 128]: thread = (dim pair, group of 4 sequences)
     {

@@ -209,10 +209,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
           const int kc = with_q ? u : u - NKC;
           const unsigned n = lat_n + (unsigned)u, slot = n % kLatSlots;
           const uint32_t eb = smem_u32(&bars->lat_empty[slot]), epar = ((n / kLatSlots) & 1) ^ 1;
-          if (!mbar_test_wait(eb, epar)) {
-            ok = __all_sync(0xffffffffu, mbar_spin(eb, epar, s_abort, 1));
-            if (!ok) break;
-          }
+          ok = warp_wait(eb, epar, s_abort, 1);
+          if (!ok) break;
           if (elect_one()) {
             const uint32_t fb = smem_u32(&bars->lat_full[slot]);
             mbar_expect_tx(fb, (uint32_t)(halves * 8192 + (with_q ? N * 128 : 0)));
@@ -235,10 +233,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         for (int cb = 0; cb < NRB; ++cb) {
           const unsigned slot = rope_n % kRopeSlots;
           const uint32_t eb = smem_u32(&bars->rope_empty[slot]), epar = ((rope_n / kRopeSlots) & 1) ^ 1;
-          if (!mbar_test_wait(eb, epar)) {
-            ok = __all_sync(0xffffffffu, mbar_spin(eb, epar, s_abort, 2));
-            if (!ok) break;
-          }
+          ok = warp_wait(eb, epar, s_abort, 2);
+          if (!ok) break;
           if (elect_one()) {
             const uint32_t fb = smem_u32(&bars->rope_full[slot]);
             mbar_expect_tx(fb, (uint32_t)(halves * 8192));
@@ -279,10 +275,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       if (elect_one()) EKV_STAMP(1, 300, tile);
       for (int kc = 0; kc < NKC; ++kc) {
         const uint32_t fb = full0 + slot * 8;
-        if (!mbar_test_wait(fb, par)) {
-          ok = __all_sync(0xffffffffu, mbar_spin(fb, par, s_abort, 3));
-          if (!ok) break;
-        }
+        ok = warp_wait(fb, par, s_abort, 3);
+        if (!ok) break;
         const uint32_t la = (lat16 + slot * kSlot16) | (1u << 16), lb = la + (kChunkBytes >> 4);
         if (elect_one()) {
           tc_mma_w(tmem_s, la, hi_sw, lb, hi_sw, idesc_s, kc != 0);
@@ -301,7 +295,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       }
       __syncwarp();
       // ---- wait for P (and the rescaled output) of this tile
-      ok = __all_sync(0xffffffffu, mbar_spin(smem_u32(&bars->p_ready), (tbase + tile) & 1, s_abort, 4));
+      ok = warp_wait(smem_u32(&bars->p_ready), (tbase + tile) & 1, s_abort, 4);
       if (!ok) break;
       tc_fence_after();
       if (elect_one()) EKV_STAMP(1, 21, tile);
@@ -311,10 +305,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       par = (nb0 / kLatSlots) & 1;
       for (int blk = 0; blk < NB; ++blk) {
         const uint32_t fb = full0 + slot * 8;
-        if (!(mbar_test_wait(fb, par) && mbar_test_wait(fb + 8, par))) {
-          ok = __all_sync(0xffffffffu, mbar_spin(fb, par, s_abort, 5) && mbar_spin(fb + 8, par, s_abort, 5));
-          if (!ok) break;
-        }
+        ok = warp_wait(fb, par, s_abort, 5) && warp_wait(fb + 8, par, s_abort, 5);
+        if (!ok) break;
         if (zero_to > zero_from) {
           // ragged end of a sequence: rows past its last token inside the last 16-token step are
           // made exact zeros so that zero-probability rows cannot inject NaN/Inf bit patterns

@@ -89,6 +89,18 @@ __device__ __forceinline__ bool mbar_spin(uint32_t bar, uint32_t parity, volatil
   return false;
 #endif
 }
+// Warp-uniform bounded wait on one phase for a fully converged warp: every lane probes and any
+// lane's success counts for all (a phase that this warp waits for cannot be undone by anybody
+// else), so the lanes can never disagree about the outcome.
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int why) {
+  if (__any_sync(0xffffffffu, mbar_test_wait(bar, parity))) return true;
+  for (unsigned i = 0; i < 16u * kWaitLimit; ++i) {
+    if (__any_sync(0xffffffffu, mbar_test_wait(bar, parity))) return true;
+    if ((i & 4095) == 4095 && __any_sync(0xffffffffu, *abort_flag != 0)) return false;
+  }
+  if (*abort_flag == 0) *abort_flag = why;
+  return false;
+}
 // Bounded wait; returns false when the limit is hit (the block's abort flag is then set to `why`,
 // a small positive code that names the wait) or when another thread has already given up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int why) {

@@ -2,7 +2,8 @@
 """Benchmark of EliteKV decode attention on B200.
 
 One step = one pass of the whole decode hot path for one layer over a batch of sequences:
-    elitekv_append (1 new token per sequence) -> elitekv_absorb_query -> elitekv_decode.
+    elitekv_append (1 new token per sequence) | elitekv_absorb_query -> elitekv_decode
+(the append and the query preparation are independent and run on two streams).
 Metric: decode-attention tokens/s (= sequences advanced per second for one layer), plus the
 achieved cache-read bandwidth.  Workload at one GPU: LLaMA2-7B-shaped layer, 75 % KV reduction
 (r = 8 elite chunks/head, d_c = 1536), batch 16, context 4096, contiguous cache, bf16,
@@ -155,7 +156,8 @@ def config_of(w: gen.Workload, world: int, cache_bytes=None):
     c = {"workload": w.name, "n_h": w.n_h, "d_h": w.d_h, "r": w.r, "d_c": w.d_c,
          "batch_per_gpu": w.B, "context": w.ctx, "paged": w.paged,
          "l2": "256 MiB flush write before every timed step; cache larger than L2",
-         "parallelism": f"replicas x{world} (independent sequences, no collective)"}
+         "parallelism": f"replicas x{world} (independent sequences, no collective)",
+         "streams": "append on a second stream beside absorb_query; joined before decode"}
     if cache_bytes is not None:
         c["cache_bytes_per_step"] = cache_bytes
     return c
@@ -258,9 +260,22 @@ def build_workload(w: gen.Workload, ek, device, decode_kernel: int = 0):
     return layer, cache, lens, host, dev, ws, bufs, keep
 
 
+_SIDE_STREAM = None
+
+
 def step(ek, layer, cache, d, ws, bufs):
-    ek.elitekv_append(layer, cache, d["k_e"], d["c"], d["seq_id"], d["pos"])
+    """One decode step.  The append (writes the cache) and the query preparation (reads only the
+    queries) do not depend on each other, so the append runs on a second stream beside the
+    absorb; both are joined before the attention call."""
+    global _SIDE_STREAM
+    main = torch.cuda.current_stream()
+    if _SIDE_STREAM is None:
+        _SIDE_STREAM = torch.cuda.Stream()
+    _SIDE_STREAM.wait_stream(main)
+    with torch.cuda.stream(_SIDE_STREAM):
+        ek.elitekv_append(layer, cache, d["k_e"], d["c"], d["seq_id"], d["pos"])
     ek.elitekv_absorb_query(layer, d["q"], d["pos"], bufs["q_rope"], bufs["q_abs"])
+    main.wait_stream(_SIDE_STREAM)
     ek.elitekv_decode(layer, cache, bufs["q_rope"], bufs["q_abs"], d["lens"], ws, bufs["out"])
 
 

@@ -123,6 +123,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   EKV_STAMP_DECL;
 
+  if (threadIdx.x == 32) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_lat128) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_q) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_rope128) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_lat) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_rope) : "memory");
+  }
   if (threadIdx.x == 0) {
     for (int i = 0; i < kLatSlots; ++i) {
       mbar_init(smem_u32(&bars->lat_full[i]), 1);
@@ -160,12 +167,15 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   const int tok0 = a.items[4 * item + 1];
   const int ntok = a.items[4 * item + 2];
   const int n_tiles = (ntok + kTile - 1) / kTile;
-  // rotated query chunks of this sequence as fp32 (broadcast operand of the rope dot products)
-  for (int e = threadIdx.x; e < N * R2; e += kThreads) {
-    const int h = e / R2;
-    s_qrope[e] = h < nh_here ? __bfloat162float(a.q_rope[((size_t)seq * a.n_h + h0 + h) * R2 + (e % R2)]) : 0.f;
+  // rotated query chunks of this sequence as fp32 (broadcast operand of the rope dot products):
+  // filled and used by the softmax warps only, so nobody else waits for it
+  if (warp >= 2 && warp <= 5) {
+    for (int e = threadIdx.x - 64; e < N * R2; e += kSoftmaxThreads) {
+      const int h = e / R2;
+      s_qrope[e] = h < nh_here ? __bfloat162float(a.q_rope[((size_t)seq * a.n_h + h0 + h) * R2 + (e % R2)]) : 0.f;
+    }
+    named_bar_sync(1, kSoftmaxThreads);
   }
-  __syncthreads();
 
   // ============================================================== warps 0, 7, 8: latent TMA producers; warp 6: rope
   // Each producer warp runs its loop warp-uniformly and one elected lane issues expect_tx and the

@@ -28,6 +28,7 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
               bf16* __restrict__ q_abs, int n_h, int d_h, int r, int d_c, int max_pos,
               int32_t* status) {
   extern __shared__ __align__(16) float smem_f[];
+  ekv_pdl_trigger();      // nothing later in the stream is held up by this kernel's start
   const int h = blockIdx.x;
   const int dn = d_h - 2 * r;
   float* q_nope = smem_f;                                   // [dn][16] (sequence fastest)

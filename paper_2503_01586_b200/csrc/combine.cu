@@ -50,6 +50,7 @@ combine_fast_kernel(const float* __restrict__ part_acc, const float* __restrict_
     cp_async16(&s_w[k][v * 8], Wuv + (size_t)(k0 + k) * n_h * kFD + (size_t)h * kFD + v * 8);
   }
   cp_async_commit();
+  ekv_pdl_wait();         // the weights above are constant; everything below reads the split-K kernel's output
 
   const int n_groups = (B + kFB - 1) / kFB;
   for (int g = 0; g < n_groups; ++g) {
@@ -289,9 +290,9 @@ int ekv_launch_combine(const elitekv_layer* L, int B, const DecodeScratch& ws, v
                        cudaStream_t st) {
   if (ekv_combine_fast_ok(L)) {
     dim3 grid(L->n_h, L->d_c / kFK);
-    combine_fast_kernel<<<grid, kFThreads, 0, st>>>(ws.part_acc, ws.part_ml, ws.seq_first, L->d_Wuv,
-                                                    ws.slice_out, ws.counters, (bf16*)out, B, L->n_h,
-                                                    L->d_c);
+    EKV_CUDA_OK(ekv_launch_pdl(combine_fast_kernel, grid, dim3(kFThreads), 0, st, (const float*)ws.part_acc,
+                               (const float*)ws.part_ml, (const int32_t*)ws.seq_first, (const bf16*)L->d_Wuv,
+                               ws.slice_out, ws.counters, (bf16*)out, B, L->n_h, L->d_c));
     EKV_CUDA_OK(cudaGetLastError());
     return ELITEKV_OK;
   }

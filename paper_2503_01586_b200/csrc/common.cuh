@@ -80,6 +80,30 @@ __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
 }
 
+// Programmatic dependent launch: the kernels of one decode step are launched with the
+// programmatic-serialisation attribute, so that the next kernel's blocks are scheduled (and run
+// whatever precedes their ekv_pdl_wait) while the previous kernel drains.  ekv_pdl_wait returns
+// once every kernel earlier in the stream has completed and its writes are visible; a kernel
+// launched without the attribute, or after one that never calls ekv_pdl_trigger, behaves as usual.
+__device__ __forceinline__ void ekv_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void ekv_pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t ekv_launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                  Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 // Where a (sequence, position) lives in the cache planes.
 struct CacheView {
   const int32_t* page_table;

@@ -99,8 +99,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   const int worker = blockIdx.x / a.n_groups;         // persistent worker: walks its plan items
   const int h0 = (blockIdx.x % a.n_groups) * N;       // first head of this block's group
   const int nh_here = min(N, a.n_h - h0);
-  const int item_lo = a.worker_first[worker], item_hi = a.worker_first[worker + 1];
-  if (item_lo >= item_hi) return;
   const int d_c = a.d_c;
   const int NKC = d_c >> 6;      // 64-wide latent chunks
   const int NB = d_c >> 7;       // 128-row output blocks
@@ -158,6 +156,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
   const uint32_t tmem_s = tmem_base + NB * N;     // S columns after the NB output blocks
+  // Everything above touched only this block's own state; the plan, the queries and the cache
+  // come from kernels earlier in the stream.  A worker without items falls through to the
+  // teardown (it has allocated tensor memory like everybody else).
+  ekv_pdl_wait();
+  ekv_pdl_trigger();
+  const int item_lo = a.worker_first[worker], item_hi = a.worker_first[worker + 1];
 
   // running counters (each role advances its own copies identically): ring uses, tiles, items
   unsigned lat_n = 0, rope_n = 0, tbase = 0;
@@ -608,7 +612,8 @@ int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, con
   const int smem = N == 32 ? Smem<32>::total(L->d_c) : Smem<16>::total(L->d_c);
   auto launch = [&](auto kern) -> int {
     EKV_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    kern<<<ws.n_workers * a.n_groups, kThreads, smem, st>>>(m_lat, m_rope, m_q, m_lat128, m_rope128, a);
+    EKV_CUDA_OK(ekv_launch_pdl(kern, dim3(ws.n_workers * a.n_groups), dim3(kThreads), (size_t)smem, st, m_lat, m_rope,
+                               m_q, m_lat128, m_rope128, a));
     EKV_CUDA_OK(cudaGetLastError());
     return ELITEKV_OK;
   };

@@ -98,6 +98,8 @@ plan_balanced_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int 
   __shared__ int warp_tot[kPlanThreads / 32];
   __shared__ long long s_total;
   const int t = threadIdx.x;
+  ekv_pdl_wait();         // earlier kernels may still read the arrays written here
+  ekv_pdl_trigger();
   for (int i = t; i < n_zero; i += blockDim.x) zero_ints[i] = 0;
   if (t == 0) s_total = 0;
   __syncthreads();
@@ -166,8 +168,8 @@ plan_balanced_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int 
 int ekv_launch_plan_balanced(const int32_t* seq_lens, int B, int tile_tokens, int n_workers,
                              int max_items, int32_t* items, int32_t* seq_first_item,
                              int32_t* worker_first, int32_t* zero_ints, int n_zero, cudaStream_t st) {
-  plan_balanced_kernel<<<1, kPlanThreads, 0, st>>>(seq_lens, B, tile_tokens, n_workers, max_items, items,
-                                                   seq_first_item, worker_first, zero_ints, n_zero);
+  EKV_CUDA_OK(ekv_launch_pdl(plan_balanced_kernel, dim3(1), dim3(kPlanThreads), 0, st, seq_lens, B, tile_tokens,
+                             n_workers, max_items, items, seq_first_item, worker_first, zero_ints, n_zero));
   EKV_CUDA_OK(cudaGetLastError());
   return ELITEKV_OK;
 }

@@ -279,6 +279,14 @@ def step(ek, layer, cache, d, ws, bufs):
     ek.elitekv_decode(layer, cache, bufs["q_rope"], bufs["q_abs"], d["lens"], ws, bufs["out"])
 
 
+def step_serial(ek, layer, cache, d, ws, bufs):
+    """The same three calls on one stream (used by the end-to-end leg, which is bound by host
+    latency: the second stream's event bookkeeping costs more there than the overlap saves)."""
+    ek.elitekv_append(layer, cache, d["k_e"], d["c"], d["seq_id"], d["pos"])
+    ek.elitekv_absorb_query(layer, d["q"], d["pos"], bufs["q_rope"], bufs["q_abs"])
+    ek.elitekv_decode(layer, cache, bufs["q_rope"], bufs["q_abs"], d["lens"], ws, bufs["out"])
+
+
 KERNELS_PER_STEP = 5   # append, absorb, plan, split-K attention, combine + up-projection
 
 
@@ -345,7 +353,7 @@ def run_gpu(args, w: gen.Workload):
     def e2e_step():
         for k in host:
             staged[k].copy_(host[k], non_blocking=True)
-        step(ek, layer, cache, staged, ws, bufs)
+        step_serial(ek, layer, cache, staged, ws, bufs)
         bufs["out_host"].copy_(bufs["out"], non_blocking=True)
         torch.cuda.synchronize()
 

@@ -78,16 +78,12 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // Bounded busy wait on test_wait for the threads on the critical hand-off path (MMA issuer, TMA
 // producers): same contract as mbar_wait, 16 times the poll budget because a probe is cheap.
 __device__ __forceinline__ bool mbar_spin(uint32_t bar, uint32_t parity, volatile int* abort_flag, int why = 1) {
-#ifdef EKV_NO_SPIN
-  return mbar_wait(bar, parity, abort_flag, why);
-#else
   for (unsigned i = 0; i < 16u * kWaitLimit; ++i) {
     if (mbar_test_wait(bar, parity)) return true;
     if ((i & 4095) == 4095 && *abort_flag) return false;
   }
   if (*abort_flag == 0) *abort_flag = why;
   return false;
-#endif
 }
 // Warp-uniform bounded wait on one phase for a fully converged warp: every lane probes and any
 // lane's success counts for all (a phase that this warp waits for cannot be undone by anybody

@@ -199,6 +199,30 @@ def test_decode_7b_shape_small_context(ek):
     H.check_parity(st, out, H.all_units(st))
 
 
+def test_back_to_back_steps_share_one_workspace(ek):
+    """Two steps queued without a synchronisation in between, same workspace, different queries:
+    the plan / split-K / combine kernels of the second step are launched with programmatic
+    serialisation, so they must still wait for the first step's combine before they touch the
+    shared plan arrays and partial results.  Each output must equal the one the same step gives
+    when run alone, bit for bit, and match the oracle."""
+    w = gen.shrink(gen.LLAMA7B_75, B=4, ctx=900)
+    st = H.setup(w, lens=[900, 641, 130, 64])
+    q2 = torch.flip(st.q, dims=[0]).contiguous()
+    alone1 = H.run_decode(st).clone()
+    st2 = replace(st, q=q2)
+    alone2 = H.run_decode(st2).clone()
+    for _ in range(5):
+        qr1, qa1 = ek.elitekv_absorb_query(st.layer, st.q, st.q_pos)
+        o1 = ek.elitekv_decode(st.layer, st.cache, qr1, qa1, st.lens_dev, st.workspace)
+        qr2, qa2 = ek.elitekv_absorb_query(st.layer, q2, st.q_pos)
+        o2 = ek.elitekv_decode(st.layer, st.cache, qr2, qa2, st.lens_dev, st.workspace)
+        torch.cuda.synchronize()
+        assert ek.elitekv_check_status(st.layer) == 0
+        assert torch.equal(o1, alone1)
+        assert torch.equal(o2, alone2)
+    H.check_parity(st, alone1, H.all_units(st))
+
+
 @pytest.mark.parametrize("kernel", [1, 2, 3], ids=["generic", "tensor-core", "tensor-core-pair"])
 def test_decode_7b_shape_ragged_tails_both_kernels(ek, kernel):
     """Same inputs through the CUDA-core kernel and the tcgen05 kernel: lengths around the

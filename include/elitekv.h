@@ -133,7 +133,11 @@ int elitekv_decode_workspace_size(const elitekv_layer* layer, int32_t B, size_t*
  * its own token).  seq_lens[b] == 0 gives a zero row.
  *   out bf16 [B][n_h][d_h];  workspace: 256-byte aligned, at least
  *   elitekv_decode_workspace_size bytes, private to this call until the stream reaches its end.
- * Launches: plan, split-K attention, combine + up-projection. */
+ * Launches: plan, split-K attention, combine + up-projection.  The three kernels are launched
+ * with programmatic stream serialisation: each may start its private set-up while the kernel
+ * before it on the stream drains, but reads and writes nothing shared before every earlier
+ * kernel on the stream has completed, so the usual stream order holds for the caller (two
+ * calls may share one workspace on one stream). */
 int elitekv_decode(const elitekv_layer* layer, const elitekv_cache* cache, const void* q_rope,
                    const void* q_abs, const int32_t* seq_lens, int32_t B, void* workspace,
                    size_t workspace_bytes, void* out, elitekv_stream_t stream);

@@ -4,22 +4,30 @@
 //   q_rope[b,h,2j:2j+2] = q[b,h,chunk idx[h][j]] . R(q_pos[b] * theta_idx[h][j])
 //   q_abs [b,h,k]       = sum_i q_nope[b,h,i] * W_uk[k][h*dn + i]
 //
-// Grid (n_h, ceil(d_c/128)): a block owns one head and 128 latent coordinates.  Its 256 threads
-// are 64 coordinate pairs x 4 groups over the head's un-rotated dims; every thread keeps one fp32
-// accumulator pair per sequence of the current chunk of 16 sequences, so each weight element is
-// read once per chunk, and the four groups are added through shared memory.  The weights come
-// regrouped as [n_h][dn][d_c] (d_c contiguous); the block's [dn x 128] slab is brought into
-// shared memory by one bulk copy per weight row, all issued at once by one warp, so the whole
-// slab costs one trip to memory (the kernel is bound by latency, not by its 11 MB of traffic)
-// and overlaps the gather of the queries.
+// Grid (n_h, ceil(d_c/128) + 1).  A block of the first rows owns one head and 128 latent
+// coordinates: per chunk of 16 sequences it computes the [16 x dn] . [dn x 128] product with
+// mma.sync (m16n8k16, bf16 in, fp32 accumulate; both operands are bf16 already, so the products
+// are exact), one warp per 16 coordinates.  The weights come regrouped as [n_h][dn][d_c]
+// (d_c contiguous); the block's [dn x 128] slab is brought into shared memory by one bulk copy
+// per weight row, all issued at once by one warp, so the slab costs one trip to memory and
+// overlaps the gather of the queries.  The kernel is bound by latency, not by its 11 MB of
+// traffic or its 0.2 GFLOP.  The blocks of the last grid row do the query RoPE (three dependent
+// loads per element), off the path of the others.
 #include "tc_ptx.cuh"
 
 namespace {
 
-constexpr int kAbsorbBatch = 16;
-constexpr int kAbsorbThreads = 256;
-constexpr int kAbsorbGroups = 4;
+constexpr int kAbsorbBatch = 16;       // sequences per MMA row tile
+constexpr int kAbsorbThreads = 256;    // 8 warps x 16 coordinates
 constexpr int kAbsorbCoords = 128;
+
+__device__ __forceinline__ void mma_bf16_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
 
 __global__ void __launch_bounds__(kAbsorbThreads)
 absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int B,
@@ -27,41 +35,19 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
               const int32_t* __restrict__ idx, const float2* __restrict__ cs, bf16* __restrict__ q_rope,
               bf16* __restrict__ q_abs, int n_h, int d_h, int r, int d_c, int max_pos,
               int32_t* status) {
-  extern __shared__ __align__(16) float smem_f[];
+  extern __shared__ __align__(16) unsigned char smem_b[];
   ekv_pdl_trigger();      // nothing later in the stream is held up by this kernel's start
   const int h = blockIdx.x;
   const int dn = d_h - 2 * r;
-  float* q_nope = smem_f;                                   // [dn][16] (sequence fastest)
-  float* red = smem_f + (size_t)(dn > 0 ? dn : 1) * kAbsorbBatch;   // [3][16][128]
-  bf16* s_w = (bf16*)(red + (size_t)(kAbsorbGroups - 1) * kAbsorbBatch * kAbsorbCoords);   // [dn][128]
+  const int kpad = (dn + 15) & ~15;                  // K of the product, zero-padded to 16
+  const int qpitch = kpad + 8;                       // row pitch of the query tile (bank spread)
+  bf16* s_w = (bf16*)smem_b;                         // [kpad][128] weight slab
+  bf16* s_q = s_w + (size_t)kpad * kAbsorbCoords;    // [16][qpitch] un-rotated query dims
   __shared__ __align__(8) uint64_t w_bar;
   __shared__ int s_abort;
   const bool rope_block = blockIdx.y == gridDim.y - 1;      // last grid row: query RoPE only
-  const int k0 = blockIdx.y * kAbsorbCoords;
-  const int kw = min(kAbsorbCoords, d_c - k0);       // coordinates of this slab (a multiple of 8)
-  if (threadIdx.x == 0) {
-    mbar_init(smem_u32(&w_bar), 1);
-    s_abort = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    fence_proxy_async();
-  }
-  __syncthreads();
-  if (threadIdx.x < 32 && dn > 0 && !rope_block) {
-    if (threadIdx.x == 0) mbar_expect_tx(smem_u32(&w_bar), (uint32_t)(dn * kw * 2));
-    __syncwarp();
-    const bf16* src = WukT + (size_t)h * dn * d_c + k0;
-    for (int i = threadIdx.x; i < dn; i += 32)
-      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                   ::"r"(smem_u32(s_w + (size_t)i * kAbsorbCoords)), "l"(src + (size_t)i * d_c), "r"(kw * 2),
-                     "r"(smem_u32(&w_bar)) : "memory");
-  }
-  bool w_ready = dn == 0;
-  const int pair = threadIdx.x & 63, grp = threadIdx.x >> 6;
-  const int k = blockIdx.y * kAbsorbCoords + 2 * pair;
   const int32_t* dims = qdims + (size_t)h * d_h;
 
-  // rope part: one extra block per head does it (three dependent loads: kept off the path of
-  // the blocks that do the absorption)
   if (rope_block) {
     for (int e = threadIdx.x; e < B * r; e += blockDim.x) {
       const int b = e / r, j = e % r;
@@ -78,22 +64,47 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
       bf162* dst = (bf162*)(q_rope + ((size_t)b * n_h + h) * 2 * r + 2 * j);
       *dst = __floats2bfloat162_rn(y0, y1);
     }
-      return;
+    return;
   }
 
-  const int per_grp = (dn + kAbsorbGroups - 1) / kAbsorbGroups;
-  const int i_lo = min(dn, grp * per_grp), i_hi = min(dn, i_lo + per_grp);
+  const int k0 = blockIdx.y * kAbsorbCoords;
+  const int kw = min(kAbsorbCoords, d_c - k0);       // coordinates of this slab (a multiple of 8)
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&w_bar), 1);
+    s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+  }
+  __syncthreads();
+  if (threadIdx.x < 32 && dn > 0) {
+    if (threadIdx.x == 0) mbar_expect_tx(smem_u32(&w_bar), (uint32_t)(dn * kw * 2));
+    __syncwarp();
+    const bf16* src = WukT + (size_t)h * dn * d_c + k0;
+    for (int i = threadIdx.x; i < dn; i += 32)
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"(smem_u32(s_w + (size_t)i * kAbsorbCoords)), "l"(src + (size_t)i * d_c), "r"(kw * 2),
+                     "r"(smem_u32(&w_bar)) : "memory");
+  }
+  // rows of the slab past dn (K padding) are zeros
+  for (int e = threadIdx.x; e < (kpad - dn) * (kAbsorbCoords / 8); e += blockDim.x)
+    *(uint4*)(s_w + (size_t)(dn + e / (kAbsorbCoords / 8)) * kAbsorbCoords + (e % (kAbsorbCoords / 8)) * 8) =
+        make_uint4(0, 0, 0, 0);
+  bool w_ready = dn == 0;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;             // MMA fragment coordinates of this lane
+  const int n0 = warp * 16;                          // first coordinate (inside the slab) of this warp
   for (int b0 = 0; b0 < B; b0 += kAbsorbBatch) {
     const int nb = min(kAbsorbBatch, B - b0);
     __syncthreads();
-    for (int e = threadIdx.x; e < kAbsorbBatch * dn; e += blockDim.x) {
-      const int i = e / kAbsorbBatch, bb = e % kAbsorbBatch;
-      q_nope[e] = bb < nb ? __bfloat162float(q[((size_t)(b0 + bb) * n_h + h) * d_h + dims[2 * r + i]]) : 0.f;
+    // un-rotated query dims of 16 sequences, bf16 as they come; K padding and missing rows are zeros
+    for (int e = threadIdx.x; e < kAbsorbBatch * kpad; e += blockDim.x) {
+      const int bb = e / kpad, i = e % kpad;
+      bf16 v = __float2bfloat16_rn(0.f);
+      if (bb < nb && i < dn) v = q[((size_t)(b0 + bb) * n_h + h) * d_h + dims[2 * r + i]];
+      s_q[bb * qpitch + i] = v;
     }
     __syncthreads();
-    float a0[kAbsorbBatch], a1[kAbsorbBatch];
-#pragma unroll
-    for (int bb = 0; bb < kAbsorbBatch; ++bb) a0[bb] = a1[bb] = 0.f;
     if (!w_ready) {
       // the weight slab has landed (bounded wait; a timeout is recorded and the block leaves)
       volatile int* abort_flag = &s_abort;
@@ -103,49 +114,33 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
         return;
       }
     }
-    if (k < d_c) {
-      const bf16* wp = s_w + 2 * pair;
-      for (int i0 = i_lo; i0 < i_hi; i0 += 8) {
-        float2 w[8];
+    if (n0 < kw) {
+      float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+      for (int kk = 0; kk < kpad; kk += 16) {
+        // A fragment (16 sequences x 16 dims): rows g and g+8, dim pairs 2t and 2t+8
+        uint32_t a[4];
+        a[0] = *(const uint32_t*)(s_q + g * qpitch + kk + 2 * t);
+        a[1] = *(const uint32_t*)(s_q + (g + 8) * qpitch + kk + 2 * t);
+        a[2] = *(const uint32_t*)(s_q + g * qpitch + kk + 2 * t + 8);
+        a[3] = *(const uint32_t*)(s_q + (g + 8) * qpitch + kk + 2 * t + 8);
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-          w[j] = i0 + j < i_hi ? __bfloat1622float2(*(const bf162*)(wp + (size_t)(i0 + j) * kAbsorbCoords))
-                               : make_float2(0.f, 0.f);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          if (i0 + j < i_hi) {
-            const float4* xr = (const float4*)(q_nope + (size_t)(i0 + j) * kAbsorbBatch);
-#pragma unroll
-            for (int v = 0; v < kAbsorbBatch / 4; ++v) {
-              const float4 x = xr[v];
-              a0[4 * v + 0] = fmaf(x.x, w[j].x, a0[4 * v + 0]); a1[4 * v + 0] = fmaf(x.x, w[j].y, a1[4 * v + 0]);
-              a0[4 * v + 1] = fmaf(x.y, w[j].x, a0[4 * v + 1]); a1[4 * v + 1] = fmaf(x.y, w[j].y, a1[4 * v + 1]);
-              a0[4 * v + 2] = fmaf(x.z, w[j].x, a0[4 * v + 2]); a1[4 * v + 2] = fmaf(x.z, w[j].y, a1[4 * v + 2]);
-              a0[4 * v + 3] = fmaf(x.w, w[j].x, a0[4 * v + 3]); a1[4 * v + 3] = fmaf(x.w, w[j].y, a1[4 * v + 3]);
-            }
-          }
+        for (int nt = 0; nt < 2; ++nt) {
+          // B fragment (16 dims x 8 coordinates): coordinate g, dim pairs 2t and 2t+8
+          const unsigned short* wp = (const unsigned short*)(s_w + (size_t)(kk + 2 * t) * kAbsorbCoords + n0 + nt * 8 + g);
+          const uint32_t b0r = (uint32_t)wp[0] | ((uint32_t)wp[kAbsorbCoords] << 16);
+          const uint32_t b1r = (uint32_t)wp[8 * kAbsorbCoords] | ((uint32_t)wp[9 * kAbsorbCoords] << 16);
+          mma_bf16_16816(acc[nt], a, b0r, b1r);
         }
       }
-    }
-    if (grp > 0) {
+      // C fragment: rows g and g+8, coordinates 2t and 2t+1 of each 8-wide tile
 #pragma unroll
-      for (int bb = 0; bb < kAbsorbBatch; ++bb)
-        *(float2*)(red + ((size_t)(grp - 1) * kAbsorbBatch + bb) * kAbsorbCoords + 2 * pair) =
-            make_float2(a0[bb], a1[bb]);
-    }
-    __syncthreads();
-    if (grp == 0 && k < d_c) {
-#pragma unroll
-      for (int bb = 0; bb < kAbsorbBatch; ++bb) {
-        if (bb < nb) {
-          float s0 = a0[bb], s1 = a1[bb];
-#pragma unroll
-          for (int g = 0; g < kAbsorbGroups - 1; ++g) {
-            const float2 t = *(const float2*)(red + ((size_t)g * kAbsorbBatch + bb) * kAbsorbCoords + 2 * pair);
-            s0 += t.x;
-            s1 += t.y;
-          }
-          *(bf162*)(q_abs + ((size_t)(b0 + bb) * n_h + h) * d_c + k) = __floats2bfloat162_rn(s0, s1);
+      for (int nt = 0; nt < 2; ++nt) {
+        const int k = k0 + n0 + nt * 8 + 2 * t;
+        if (k < d_c) {
+          if (g < nb)
+            *(bf162*)(q_abs + ((size_t)(b0 + g) * n_h + h) * d_c + k) = __floats2bfloat162_rn(acc[nt][0], acc[nt][1]);
+          if (g + 8 < nb)
+            *(bf162*)(q_abs + ((size_t)(b0 + g + 8) * n_h + h) * d_c + k) = __floats2bfloat162_rn(acc[nt][2], acc[nt][3]);
         }
       }
     }
@@ -158,9 +153,8 @@ int ekv_launch_absorb(const elitekv_layer* L, const void* q, const int32_t* q_po
                       void* q_rope, void* q_abs, cudaStream_t st) {
   if (B == 0) return ELITEKV_OK;
   dim3 grid(L->n_h, (L->d_c + kAbsorbCoords - 1) / kAbsorbCoords + 1);   // + one row of rope blocks
-  size_t smem = sizeof(float) * (kAbsorbBatch * (size_t)(L->dn > 0 ? L->dn : 1) +
-                                 (size_t)(kAbsorbGroups - 1) * kAbsorbBatch * kAbsorbCoords) +
-                sizeof(bf16) * (size_t)L->dn * kAbsorbCoords;
+  const int kpad = (L->dn + 15) & ~15;
+  const size_t smem = sizeof(bf16) * ((size_t)kpad * kAbsorbCoords + (size_t)kAbsorbBatch * (kpad + 8)) + 16;
   if ((int)smem > L->smem_optin || L->d_c % 8 != 0) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
   EKV_CUDA_OK(cudaFuncSetAttribute(absorb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   absorb_kernel<<<grid, kAbsorbThreads, smem, st>>>(

@@ -20,6 +20,7 @@ namespace {
 constexpr int kAbsorbBatch = 16;       // sequences per MMA row tile
 constexpr int kAbsorbThreads = 256;    // 8 warps x 16 coordinates
 constexpr int kAbsorbCoords = 128;
+constexpr int kAbsorbPitch = kAbsorbCoords + 8;   // slab row pitch: 16 bytes of padding spread the fragment loads over the banks
 
 __device__ __forceinline__ void mma_bf16_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
   asm volatile(
@@ -41,8 +42,8 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
   const int dn = d_h - 2 * r;
   const int kpad = (dn + 15) & ~15;                  // K of the product, zero-padded to 16
   const int qpitch = kpad + 8;                       // row pitch of the query tile (bank spread)
-  bf16* s_w = (bf16*)smem_b;                         // [kpad][128] weight slab
-  bf16* s_q = s_w + (size_t)kpad * kAbsorbCoords;    // [16][qpitch] un-rotated query dims
+  bf16* s_w = (bf16*)smem_b;                         // [kpad][128 + 8] weight slab
+  bf16* s_q = s_w + (size_t)kpad * kAbsorbPitch;    // [16][qpitch] un-rotated query dims
   __shared__ __align__(8) uint64_t w_bar;
   __shared__ int s_abort;
   const bool rope_block = blockIdx.y == gridDim.y - 1;      // last grid row: query RoPE only
@@ -82,12 +83,12 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
     const bf16* src = WukT + (size_t)h * dn * d_c + k0;
     for (int i = threadIdx.x; i < dn; i += 32)
       asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                   ::"r"(smem_u32(s_w + (size_t)i * kAbsorbCoords)), "l"(src + (size_t)i * d_c), "r"(kw * 2),
+                   ::"r"(smem_u32(s_w + (size_t)i * kAbsorbPitch)), "l"(src + (size_t)i * d_c), "r"(kw * 2),
                      "r"(smem_u32(&w_bar)) : "memory");
   }
   // rows of the slab past dn (K padding) are zeros
   for (int e = threadIdx.x; e < (kpad - dn) * (kAbsorbCoords / 8); e += blockDim.x)
-    *(uint4*)(s_w + (size_t)(dn + e / (kAbsorbCoords / 8)) * kAbsorbCoords + (e % (kAbsorbCoords / 8)) * 8) =
+    *(uint4*)(s_w + (size_t)(dn + e / (kAbsorbCoords / 8)) * kAbsorbPitch + (e % (kAbsorbCoords / 8)) * 8) =
         make_uint4(0, 0, 0, 0);
   bool w_ready = dn == 0;
 
@@ -126,9 +127,9 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
 #pragma unroll
         for (int nt = 0; nt < 2; ++nt) {
           // B fragment (16 dims x 8 coordinates): coordinate g, dim pairs 2t and 2t+8
-          const unsigned short* wp = (const unsigned short*)(s_w + (size_t)(kk + 2 * t) * kAbsorbCoords + n0 + nt * 8 + g);
-          const uint32_t b0r = (uint32_t)wp[0] | ((uint32_t)wp[kAbsorbCoords] << 16);
-          const uint32_t b1r = (uint32_t)wp[8 * kAbsorbCoords] | ((uint32_t)wp[9 * kAbsorbCoords] << 16);
+          const unsigned short* wp = (const unsigned short*)(s_w + (size_t)(kk + 2 * t) * kAbsorbPitch + n0 + nt * 8 + g);
+          const uint32_t b0r = (uint32_t)wp[0] | ((uint32_t)wp[kAbsorbPitch] << 16);
+          const uint32_t b1r = (uint32_t)wp[8 * kAbsorbPitch] | ((uint32_t)wp[9 * kAbsorbPitch] << 16);
           mma_bf16_16816(acc[nt], a, b0r, b1r);
         }
       }
@@ -154,7 +155,7 @@ int ekv_launch_absorb(const elitekv_layer* L, const void* q, const int32_t* q_po
   if (B == 0) return ELITEKV_OK;
   dim3 grid(L->n_h, (L->d_c + kAbsorbCoords - 1) / kAbsorbCoords + 1);   // + one row of rope blocks
   const int kpad = (L->dn + 15) & ~15;
-  const size_t smem = sizeof(bf16) * ((size_t)kpad * kAbsorbCoords + (size_t)kAbsorbBatch * (kpad + 8)) + 16;
+  const size_t smem = sizeof(bf16) * ((size_t)kpad * kAbsorbPitch + (size_t)kAbsorbBatch * (kpad + 8)) + 16;
   if ((int)smem > L->smem_optin || L->d_c % 8 != 0) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
   EKV_CUDA_OK(cudaFuncSetAttribute(absorb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   absorb_kernel<<<grid, kAbsorbThreads, smem, st>>>(

@@ -18,13 +18,21 @@
 
 namespace {
 
+__device__ __forceinline__ void mma_bf16_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
 // ------------------------------------------------------------------ fast path
 constexpr int kFB = 16;          // sequences per group
 constexpr int kFK = 128;         // latent slice
 constexpr int kFD = 128;         // head dim
 constexpr int kFThreads = 256;
 constexpr int kFI = 16;          // items per sequence whose merge weights are staged in shared memory
-constexpr int kFStage = 512;     // items per sequence group whose (m, l) are staged in shared memory
+constexpr int kFStage = 448;     // items per sequence group whose (m, l) are staged in shared memory
 
 __global__ void __launch_bounds__(kFThreads)
 combine_fast_kernel(const float* __restrict__ part_acc, const float* __restrict__ part_ml,
@@ -32,8 +40,9 @@ combine_fast_kernel(const float* __restrict__ part_acc, const float* __restrict_
                     float* __restrict__ slice_out /* [n_slices][B][n_h][128] */,
                     int32_t* __restrict__ counters /* [n_h][n_groups], zeroed by the plan kernel */,
                     bf16* __restrict__ out, int B, int n_h, int d_c) {
-  __shared__ __align__(16) bf16 s_w[kFK][kFD];          // 32 KB
-  __shared__ __align__(16) float s_x[kFB][kFK];         // 8 KB merged latent outputs
+  __shared__ __align__(16) bf16 s_w[kFK][kFD + 8];      // W_uv slice; rows padded by 16 bytes so that the
+                                                        // fragment loads of the product spread over the banks
+  __shared__ __align__(16) float s_x[kFB][kFK + 8];     // merged latent outputs (padded rows: bank spread)
   __shared__ float s_M[kFB], s_invL[kFB];
   __shared__ float s_wt[kFB][kFI];
   __shared__ float2 s_ml[kFStage];
@@ -128,32 +137,40 @@ combine_fast_kernel(const float* __restrict__ part_acc, const float* __restrict_
     }
     cp_async_wait<0>();      // the W_uv slice (first group only; later a no-op)
     __syncthreads();
-    // [16 x 128] . [128 x 128]: thread = (dim pair, group of 4 sequences)
+    // [16 x 128] . [128 x 128] on mma.sync (m16n8k16, bf16 in, fp32 accumulate): one warp per 16
+    // output dims.  The fp32 rows of x are fed as a bf16 head plus a bf16 remainder (two MMAs),
+    // so nothing but the last ~2^-17 of x is lost; W_uv is bf16 as stored.
     {
-      const int pair = tid & 63, bg = tid >> 6;
-      float a0[4] = {0.f, 0.f, 0.f, 0.f}, a1[4] = {0.f, 0.f, 0.f, 0.f};
+      const int g = lane >> 2, t = lane & 3, n0 = warp * 16;
+      float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll 2
-      for (int k = 0; k < kFK; k += 4) {
-        float4 x[4];
+      for (int kk = 0; kk < kFK; kk += 16) {
+        uint32_t ahi[4], alo[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) x[j] = *(const float4*)&s_x[bg * 4 + j][k];
+        for (int f = 0; f < 4; ++f) {
+          const float2 x = *(const float2*)&s_x[g + (f & 1) * 8][kk + 2 * t + (f >> 1) * 8];
+          const bf162 hi = __floats2bfloat162_rn(x.x, x.y);
+          const float2 hf = __bfloat1622float2(hi);
+          const bf162 lo = __floats2bfloat162_rn(x.x - hf.x, x.y - hf.y);
+          ahi[f] = *(const uint32_t*)&hi;
+          alo[f] = *(const uint32_t*)&lo;
+        }
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-          const float2 w = __bfloat1622float2(*(const bf162*)&s_w[k + kk][2 * pair]);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const float xv = kk == 0 ? x[j].x : kk == 1 ? x[j].y : kk == 2 ? x[j].z : x[j].w;
-            a0[j] = fmaf(xv, w.x, a0[j]);
-            a1[j] = fmaf(xv, w.y, a1[j]);
-          }
+        for (int nt = 0; nt < 2; ++nt) {
+          const unsigned short* wp = (const unsigned short*)&s_w[kk + 2 * t][n0 + nt * 8 + g];
+          const uint32_t b0r = (uint32_t)wp[0] | ((uint32_t)wp[kFD + 8] << 16);
+          const uint32_t b1r = (uint32_t)wp[8 * (kFD + 8)] | ((uint32_t)wp[9 * (kFD + 8)] << 16);
+          mma_bf16_16816(acc[nt], ahi, b0r, b1r);
+          mma_bf16_16816(acc[nt], alo, b0r, b1r);
         }
       }
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int bb = bg * 4 + j;
-        if (bb < nb)
-          *(float2*)(slice_out + (((size_t)slice * B + b0 + bb) * n_h + h) * kFD + 2 * pair) =
-              make_float2(a0[j], a1[j]);
+      for (int nt = 0; nt < 2; ++nt) {
+        const int d = n0 + nt * 8 + 2 * t;
+        if (g < nb)
+          *(float2*)(slice_out + (((size_t)slice * B + b0 + g) * n_h + h) * kFD + d) = make_float2(acc[nt][0], acc[nt][1]);
+        if (g + 8 < nb)
+          *(float2*)(slice_out + (((size_t)slice * B + b0 + g + 8) * n_h + h) * kFD + d) = make_float2(acc[nt][2], acc[nt][3]);
       }
     }
     // last block of this (head, group) adds the slices in order

@@ -199,6 +199,18 @@ def test_decode_7b_shape_small_context(ek):
     H.check_parity(st, out, H.all_units(st))
 
 
+def test_decode_7b_shape_batch_not_a_multiple_of_16(ek):
+    """37 sequences: the absorb and combine kernels work on chunks of 16 sequences (one MMA row
+    tile), so the last chunk has 5 live rows; lengths from 1 token to a few tiles."""
+    B = 37
+    lens = [1 + (53 * i * i + 17 * i) % 330 for i in range(B)]
+    w = gen.shrink(gen.LLAMA7B_75, B=B, ctx=max(lens))
+    st = H.setup(w, lens=lens)
+    out = H.run_decode(st)
+    assert torch.isfinite(out.float()).all()
+    H.check_parity(st, out, H.sample_units(st, 96, seed=3))
+
+
 def test_back_to_back_steps_share_one_workspace(ek):
     """Two steps queued without a synchronisation in between, same workspace, different queries:
     the plan / split-K / combine kernels of the second step are launched with programmatic

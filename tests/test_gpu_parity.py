@@ -211,6 +211,41 @@ def test_decode_7b_shape_batch_not_a_multiple_of_16(ek):
     H.check_parity(st, out, H.sample_units(st, 96, seed=3))
 
 
+def test_step_replays_from_a_cuda_graph(ek):
+    """The calls only enqueue work and read lengths, positions and the plan on the device, so a
+    step (query preparation + attention, programmatic launches included) can be captured once
+    and replayed; after the queries change in place the replay gives the new result."""
+    w = gen.shrink(gen.LLAMA7B_75, B=4, ctx=600)
+    st = H.setup(w, lens=[600, 257, 128, 31])
+    eager1 = H.run_decode(st).clone()
+    q_live = st.q.clone()
+    q_rope = torch.empty((4, w.n_h, 2 * w.r), dtype=torch.bfloat16, device="cuda")
+    q_abs = torch.empty((4, w.n_h, w.d_c), dtype=torch.bfloat16, device="cuda")
+    out = torch.empty((4, w.n_h, w.d_h), dtype=torch.bfloat16, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for _ in range(2):   # warm-up outside capture (attribute calls, lazy module loading)
+            ek.elitekv_absorb_query(st.layer, q_live, st.q_pos, q_rope, q_abs)
+            ek.elitekv_decode(st.layer, st.cache, q_rope, q_abs, st.lens_dev, st.workspace, out)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        ek.elitekv_absorb_query(st.layer, q_live, st.q_pos, q_rope, q_abs)
+        ek.elitekv_decode(st.layer, st.cache, q_rope, q_abs, st.lens_dev, st.workspace, out)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, eager1)
+    q2 = torch.flip(st.q, dims=[1]).contiguous()
+    eager2 = H.run_decode(replace(st, q=q2)).clone()
+    q_live.copy_(q2)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert ek.elitekv_check_status(st.layer) == 0
+    assert torch.equal(out, eager2)
+
+
 def test_back_to_back_steps_share_one_workspace(ek):
     """Two steps queued without a synchronisation in between, same workspace, different queries:
     the plan / split-K / combine kernels of the second step are launched with programmatic

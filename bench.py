@@ -366,6 +366,30 @@ def run_gpu(args, w: gen.Workload):
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
 
+    # ---- the same end-to-end step captured once in a CUDA graph and replayed (informational:
+    #      what a serving loop that graphs its decode step gets; `e2e.value` stays the eager path)
+    e2e_graph_s = None
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for k in host:
+                staged[k].copy_(host[k], non_blocking=True)
+            step_serial(ek, layer, cache, staged, ws, bufs)
+            bufs["out_host"].copy_(bufs["out"], non_blocking=True)
+        for _ in range(3):
+            graph.replay()
+            torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            graph.replay()
+            torch.cuda.synchronize()
+        e2e_graph_s = time.perf_counter() - t0
+        assert ek.elitekv_check_status(layer) == 0
+    except Exception as exc:      # capture not possible in this environment: report only the eager number
+        print(f"[bench] CUDA-graph end-to-end leg skipped: {exc}", file=sys.stderr)
+
     # ---- per-call breakdown (informational; same kernels, a few extra untimed-by-the-metric calls)
     def timed(fn, n=10):
         evs = []
@@ -450,7 +474,8 @@ def run_gpu(args, w: gen.Workload):
                      "kernel_us": kern_avg_s * 1e6, "launches_timed": kern_n,
                      "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(w.name)},
         "e2e": {"value": world * w.B * args.steps / e2e_s, "unit": UNIT,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "value_cuda_graph": (world * w.B * args.steps / e2e_graph_s) if e2e_graph_s else None},
         "gpu_launches": KERNELS_PER_STEP * args.steps,
         "clocks": clocks,
         "stages": stages,

@@ -94,7 +94,8 @@ template <int N, int R2>
 __global__ void __launch_bounds__(kThreads, 1)
 decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_constant__ CUtensorMap map_rope,
                  const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_lat128,
-                 const __grid_constant__ CUtensorMap map_rope128, const TcArgs a) {
+                 const __grid_constant__ CUtensorMap map_rope128, const __grid_constant__ CUtensorMap map_part,
+                 const TcArgs a) {
   extern __shared__ unsigned char smem_raw[];
   const int worker = blockIdx.x / a.n_groups;         // persistent worker: walks its plan items
   const int h0 = (blockIdx.x % a.n_groups) * N;       // first head of this block's group
@@ -127,6 +128,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_rope128) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_lat) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_rope) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_part) : "memory");
   }
   if (threadIdx.x == 0) {
     for (int i = 0; i < kLatSlots; ++i) {
@@ -497,16 +499,26 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
     ok = mbar_wait_group(smem_u32(&bars->pv_done), (tbase + n_tiles - 1) & 1, s_abort, threadIdx.x == 64, 2, kSoftmaxThreads, 8) && ok;
     if (ok) {
       tc_fence_after();
-      float* pa = a.part_acc + ((size_t)item * a.n_h + h0) * d_c;
+      // The output block [128 coords x N heads] leaves TMEM with one thread per coordinate; it is
+      // turned into [N heads][128 coords] tiles in shared memory (the ring is idle by now) and
+      // written with one TMA store per block: part_acc[item][h0 + h][blk*128 ...].  Rows of a
+      // last, partly filled head group fall outside the tensor and are clipped by the store.
+      float* stage = (float*)s_lat;
       for (int blk = 0; blk < NB; ++blk) {
         float v[N];
         tc_ld_cols<N>(tmem_base + blk * N + lane_base, v);
         tc_wait_ld();
-        const int d = blk * 128 + trow;
+        float* tile_s = stage + (size_t)blk * N * 128;
 #pragma unroll
-        for (int h = 0; h < N; ++h)
-          if (h < nh_here) pa[(size_t)h * d_c + d] = v[h];
+        for (int h = 0; h < N; ++h) tile_s[h * 128 + trow] = v[h];
+        fence_proxy_async();
+        named_bar_sync(1, kSoftmaxThreads);
+        if (threadIdx.x == 64) {
+          tma_store_3d(&map_part, blk * 128, h0, item, smem_u32(tile_s));
+          bulk_commit_group();
+        }
       }
+      if (threadIdx.x == 64) bulk_wait_group_all();     // stores done before the ring is reused or the block leaves
       float wl = 0.f;
 #pragma unroll
       for (int h = 0; h < N; ++h) {
@@ -564,6 +576,8 @@ int ekv_tc_supported(const elitekv_layer* L, const elitekv_cache* cache) {
   if (n == 0) return 0;
   if ((L->n_h * r2) % 64 != 0 || L->n_h % 8 != 0) return 0;
   if ((n == 32 ? Smem<32>::total(L->d_c) : Smem<16>::total(L->d_c)) > L->smem_optin) return 0;
+  // the epilogue stages the whole fp32 output of a block ([d_c][n] floats) in the ring + rope area
+  if ((size_t)L->d_c * n * 4 > (size_t)kLatSlots * (kChunkBytes + n * 128) + (size_t)kRopeSlots * kChunkBytes) return 0;
   if (cache && cache->page_table && (cache->page_size % 64 != 0)) return 0;
   return 1;
 }
@@ -584,13 +598,14 @@ int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, con
   const unsigned long long rows =
       cv.page_table ? (unsigned long long)cv.num_pages << cv.page_shift : (unsigned long long)cv.max_ctx * cv.n_seqs;
   if (rows >= (1ull << 31)) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
-  CUtensorMap m_lat, m_rope, m_q, m_lat128, m_rope128;
+  CUtensorMap m_lat, m_rope, m_q, m_lat128, m_rope128, m_part;
   int rc = make_map(&m_lat, cache->latent, rows, L->d_c, 64);
   if (rc == ELITEKV_OK) rc = make_map(&m_rope, cache->rope, rows, (unsigned long long)L->n_h * 2 * L->r, 64);
   if (rc == ELITEKV_OK) rc = make_map(&m_lat128, cache->latent, rows, L->d_c, 128);
   if (rc == ELITEKV_OK) rc = make_map(&m_rope128, cache->rope, rows, (unsigned long long)L->n_h * 2 * L->r, 128);
   const int N = tc_pick_n(L);
   if (rc == ELITEKV_OK) rc = make_map(&m_q, q_abs, (unsigned long long)B * L->n_h, L->d_c, N);
+  if (rc == ELITEKV_OK) rc = make_map_f32_3d(&m_part, ws.part_acc, L->d_c, L->n_h, (unsigned long long)ws.max_items, N);
   if (rc != ELITEKV_OK) return rc;
   TcArgs a;
   a.items = ws.items;
@@ -613,7 +628,7 @@ int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, con
   auto launch = [&](auto kern) -> int {
     EKV_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     EKV_CUDA_OK(ekv_launch_pdl(kern, dim3(ws.n_workers * a.n_groups), dim3(kThreads), (size_t)smem, st, m_lat, m_rope,
-                               m_q, m_lat128, m_rope128, a));
+                               m_q, m_lat128, m_rope128, m_part, a));
     EKV_CUDA_OK(cudaGetLastError());
     return ELITEKV_OK;
   };

@@ -495,7 +495,24 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       if (threadIdx.x == 64) EKV_STAMP(2, 41, tile);
     }
 
-    // ---- epilogue: partial output and softmax statistics of this item
+    // ---- epilogue: softmax statistics of this item (while the last pass B still runs) ...
+    if (ok) {
+      float wl = 0.f;
+#pragma unroll
+      for (int h = 0; h < N; ++h) {
+        const float v = warp_sum(l_part[h]);
+        if (lane == h) wl = v;
+      }
+      named_bar_sync(1, kSoftmaxThreads);
+      if (lane < N) s_wmax[quarter * N + lane] = wl;
+      named_bar_sync(1, kSoftmaxThreads);
+      if (quarter == 0 && lane < nh_here) {
+        const float lsum = s_wmax[lane] + s_wmax[N + lane] + s_wmax[2 * N + lane] + s_wmax[3 * N + lane];
+        a.part_ml[((size_t)item * a.n_h + h0 + lane) * 2 + 0] = m_ref;
+        a.part_ml[((size_t)item * a.n_h + h0 + lane) * 2 + 1] = lsum;
+      }
+    }
+    // ---- ... and its partial output
     ok = mbar_wait_group(smem_u32(&bars->pv_done), (tbase + n_tiles - 1) & 1, s_abort, threadIdx.x == 64, 2, kSoftmaxThreads, 8) && ok;
     if (ok) {
       tc_fence_after();
@@ -519,20 +536,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         }
       }
       if (threadIdx.x == 64) bulk_wait_group_all();     // stores done before the ring is reused or the block leaves
-      float wl = 0.f;
-#pragma unroll
-      for (int h = 0; h < N; ++h) {
-        const float v = warp_sum(l_part[h]);
-        if (lane == h) wl = v;
-      }
-      named_bar_sync(1, kSoftmaxThreads);
-      if (lane < N) s_wmax[quarter * N + lane] = wl;
-      named_bar_sync(1, kSoftmaxThreads);
-      if (quarter == 0 && lane < nh_here) {
-        const float lsum = s_wmax[lane] + s_wmax[N + lane] + s_wmax[2 * N + lane] + s_wmax[3 * N + lane];
-        a.part_ml[((size_t)item * a.n_h + h0 + lane) * 2 + 0] = m_ref;
-        a.part_ml[((size_t)item * a.n_h + h0 + lane) * 2 + 1] = lsum;
-      }
     }
   }
 

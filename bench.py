@@ -493,8 +493,8 @@ def run_gpu(args, w: gen.Workload):
 # dram__bytes_read.sum + dram__bytes_write.sum of one split-K launch from the ncu capture
 # summarised under profiles/ (None until a capture of the current kernel exists).
 TRAFFIC_BYTES_PER_LAUNCH = {
-    # profiles/decode_tc_kernel__7b-75pct-b16-ctx4096.md: 275.4 MB read + 4.6 MB written
-    "7b-75pct-b16-ctx4096": 280013824,
+    # profiles/decode_tc_kernel__7b-75pct-b16-ctx4096.md: 274.9 MB read + 4.2 MB written
+    "7b-75pct-b16-ctx4096": 279057408,
 }
 
 

@@ -38,6 +38,7 @@
 //   warps 2-5    one thread per token row: rope dot products, S from TMEM, masking, running
 //                max / sum in base 2 with a lazily moved reference max, P to shared memory in the
 //                layout the second GEMM wants, TMEM rescale when the reference moves, epilogue
+//                (output blocks transposed through shared memory and written by TMA stores)
 // Every wait is bounded: when a limit is hit the block records ELITEKV_ERR_TIMEOUT in the
 // layer's status word, stops issuing work, frees its TMEM and leaves.
 #include "tc_ptx.cuh"

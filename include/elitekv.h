@@ -74,10 +74,10 @@ typedef struct {
                                  values are a pure function of the table (each product and sum
                                  rounded separately in fp32, then bf16 nearest-even).          */
   int32_t decode_kernel;      /* 0 = choose by shape; 1 = generic CUDA-core kernel; 2 = tcgen05
-                                 kernel, one block per item (latent streamed twice); 3 = tcgen05
-                                 kernel on block pairs (latent axis split over a 2-block
-                                 cluster).  2 and 3 fail with UNSUPPORTED_SHAPE when the shape
-                                 is not covered.                                               */
+                                 kernel that streams each 128-token tile twice (scores, then
+                                 values); 3 = tcgen05 kernel that keeps a 64-token tile
+                                 resident in shared memory between the two products.  2 and 3
+                                 fail with UNSUPPORTED_SHAPE when the shape is not covered.    */
 } elitekv_params;
 
 /* The two cache planes.  Contiguous (page_table == NULL): sequence s, position p live in row
@@ -101,7 +101,8 @@ typedef struct {
 int elitekv_layer_create(const elitekv_params* params, elitekv_layer** out);
 int elitekv_layer_destroy(elitekv_layer* layer);
 
-/* Cache append (Section 3.1, "incorporated into the KV cache"; Section 3.2, shared latent).
+/* Cache append (Section 3.1: the rotated elite chunks are stored once, at append time;
+ * Section 3.2: one latent shared by all heads).
  * For each of the T new tokens: rotate chunk j of head h by R(pos * theta_{idx[h][j]})
  * (Eq. 1a; (x0,x1) -> (x0 cos - x1 sin, x0 sin + x1 cos)) and write the rope row and the
  * latent row to the token's cache row.  The rotation happens here once; decode never rotates
@@ -172,9 +173,42 @@ int elitekv_decode_static(const elitekv_layer* layer, const elitekv_cache* cache
 int elitekv_plan(const int32_t* seq_lens, int32_t B, int32_t tile_tokens, int32_t max_items,
                  int32_t* items, int32_t* seq_first_item, elitekv_stream_t stream);
 
+/* The plan of the kernels whose blocks are persistent workers (the paper has no counterpart),
+ * exported for inspection.  Worker w owns the global tile range [w*quota, (w+1)*quota),
+ * quota = ceil(total tiles / n_workers); an item is the part of one sequence inside one
+ * worker's range, so items come out ordered by sequence and by worker.
+ *   items int32 [max_items][4] = (sequence, first token, token count, worker), unused entries
+ *   sequence = -1;  seq_first_item int32 [B+1];  worker_first int32 [n_workers+1]: items of
+ *   worker w are [worker_first[w], worker_first[w+1]).  max_items >= B + n_workers. */
+int elitekv_plan_workers(const int32_t* seq_lens, int32_t B, int32_t tile_tokens, int32_t n_workers,
+                         int32_t max_items, int32_t* items, int32_t* seq_first_item,
+                         int32_t* worker_first, elitekv_stream_t stream);
+
+/* Which split-K kernel and plan elitekv_decode uses for this layer, cache layout (may be NULL:
+ * shape-only answer) and batch (the paper has no counterpart).  info is a HOST array:
+ * info[0] = kernel (1, 2, 3 as in elitekv_params.decode_kernel), info[1] = tokens per plan tile,
+ * info[2] = persistent workers (0: the plain plan of elitekv_plan), info[3] = plan capacity. */
+int elitekv_decode_plan_info(const elitekv_layer* layer, const elitekv_cache* cache, int32_t B,
+                             int32_t info[4]);
+
 /* Synchronises `stream`, returns the layer's device status word (0 or a negative
  * elitekv_status recorded by a kernel) and clears it. */
 int elitekv_check_status(const elitekv_layer* layer, elitekv_stream_t stream);
+
+/* The two detail words and the fault count that the last elitekv_check_status of this layer
+ * read together with the code it returned (host array; e.g. sequence and length for
+ * BAD_POSITION, sequence and page id for BAD_PAGE, worker | wait code << 16 for TIMEOUT). */
+int elitekv_last_status_detail(const elitekv_layer* layer, int32_t detail[3]);
+
+/* Self-test of the bounded waits (the paper has no counterpart).  Launches one small block that
+ * initialises a shared-memory barrier nobody will ever arrive on and waits for it with each of
+ * the library's wait helpers (single thread, whole warp, group with a leader), every wait
+ * limited to `poll_limit` probes.  Each wait must give up: the kernel then records
+ * ELITEKV_ERR_TIMEOUT in the layer's status word (detail[0] = bit mask of the helpers that gave
+ * up as they should: 7 when all three did) and the block exits normally.  It touches no
+ * tensor memory, issues no copy and leaves the device usable.  poll_limit in [1, 2^20]. */
+int elitekv_selftest_bounded_wait(const elitekv_layer* layer, uint32_t poll_limit,
+                                  elitekv_stream_t stream);
 
 /* Comparator: uncompressed RoPE multi-head attention decode (Sections 2.1 and 2.2) over a
  * contiguous cache of rotated keys and values.

@@ -66,7 +66,11 @@ def lib() -> C.CDLL:
         L.elitekv_decode.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, i32, vp, sz, vp, vp]
         L.elitekv_decode_static.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, i32, vp, vp]
         L.elitekv_plan.argtypes = [vp, i32, i32, i32, vp, vp, vp]
+        L.elitekv_plan_workers.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp]
+        L.elitekv_decode_plan_info.argtypes = [vp, C.POINTER(CacheDesc), i32, C.POINTER(i32 * 4)]
         L.elitekv_check_status.argtypes = [vp, vp]
+        L.elitekv_last_status_detail.argtypes = [vp, C.POINTER(i32 * 3)]
+        L.elitekv_selftest_bounded_wait.argtypes = [vp, C.c_uint32, vp]
         L.elitekv_mha_workspace_size.argtypes = [i32, i32, i32, C.POINTER(sz)]
         L.elitekv_mha_decode.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, C.c_float, vp, sz, vp, vp]
         L.elitekv_profile_enable.argtypes = [vp, i32]
@@ -77,7 +81,8 @@ def lib() -> C.CDLL:
                      "elitekv_absorb_query", "elitekv_decode_workspace_size", "elitekv_decode",
                      "elitekv_plan", "elitekv_check_status", "elitekv_mha_workspace_size",
                      "elitekv_profile_enable", "elitekv_profile_collect", "elitekv_decode_static",
-                     "elitekv_mha_decode"):
+                     "elitekv_mha_decode", "elitekv_plan_workers", "elitekv_decode_plan_info",
+                     "elitekv_last_status_detail", "elitekv_selftest_bounded_wait"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -219,8 +224,39 @@ def elitekv_plan(seq_lens, tile_tokens: int, max_items: int):
     return items, first
 
 
+def elitekv_plan_workers(seq_lens, tile_tokens: int, n_workers: int, max_items: int):
+    B = seq_lens.shape[0]
+    items = torch.empty((max_items, 4), dtype=torch.int32, device=seq_lens.device)
+    first = torch.empty((B + 1,), dtype=torch.int32, device=seq_lens.device)
+    wfirst = torch.empty((n_workers + 1,), dtype=torch.int32, device=seq_lens.device)
+    _check(lib().elitekv_plan_workers(_ptr(_dev(seq_lens, torch.int32)), B, tile_tokens, n_workers,
+                                      max_items, _ptr(items), _ptr(first), _ptr(wfirst), _stream()),
+           "elitekv_plan_workers")
+    return items, first, wfirst
+
+
+def elitekv_decode_plan_info(layer: Layer, cache: Optional[CacheDesc], B: int):
+    """(kernel, tokens per plan tile, persistent workers, plan capacity)."""
+    info = (C.c_int32 * 4)()
+    _check(lib().elitekv_decode_plan_info(layer.handle, C.byref(cache) if cache is not None else None,
+                                          B, C.byref(info)), "elitekv_decode_plan_info")
+    return tuple(int(x) for x in info)
+
+
 def elitekv_check_status(layer: Layer) -> int:
     return lib().elitekv_check_status(layer.handle, _stream())
+
+
+def elitekv_last_status_detail(layer: Layer):
+    """(detail0, detail1, fault count) read by the last elitekv_check_status of this layer."""
+    d = (C.c_int32 * 3)()
+    _check(lib().elitekv_last_status_detail(layer.handle, C.byref(d)), "elitekv_last_status_detail")
+    return tuple(int(x) for x in d)
+
+
+def elitekv_selftest_bounded_wait(layer: Layer, poll_limit: int) -> None:
+    _check(lib().elitekv_selftest_bounded_wait(layer.handle, poll_limit, _stream()),
+           "elitekv_selftest_bounded_wait")
 
 
 def elitekv_profile_enable(layer: Layer, on: bool) -> None:

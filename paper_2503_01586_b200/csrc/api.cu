@@ -1,13 +1,6 @@
 // C entry points: argument checks, workspace carving, kernel selection.
 #include "common.cuh"
 
-// Diagnostic build (-DEKV_SYNC_EACH): synchronise after every launch and report which stage failed.
-#ifdef EKV_SYNC_EACH
-#define EKV_STAGE_CHECK(st, stage) do { if (cudaStreamSynchronize(st) != cudaSuccess) return -100 - (stage); } while (0)
-#else
-#define EKV_STAGE_CHECK(st, stage) do { } while (0)
-#endif
-
 namespace {
 
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -16,20 +9,19 @@ inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 // tensor-core kernel, -1 = none.  `cache` may be null (shape-only question).
 int select_kernel(const elitekv_layer* L, const elitekv_cache* cache) {
   const bool tc = ekv_tc_supported(L, cache) != 0;
-  const bool tc2 = ekv_tc2_supported(L, cache) != 0;
-  if (L->decode_kernel == 3) return tc2 ? 3 : -1;
   if (L->decode_kernel == 2) return tc ? 2 : -1;
   if (L->decode_kernel == 1) return ekv_generic_supported(L) ? 1 : -1;
-  // measured on B200 (7B shape, 75 %): the single-block kernel is the faster of the two today
   if (tc) return 2;
-  if (tc2) return 3;
   return ekv_generic_supported(L) ? 1 : -1;
 }
 
 int max_items_for(const elitekv_layer* L, int B, int kernel) {
-  if (kernel == 3) return ekv_tc2_max_items(L, B);
   return kernel == 2 ? ekv_tc_max_items(L, B) : ekv_generic_max_items(L, B);
 }
+
+// Tokens per plan tile and persistent workers (0: the plain plan) of each kernel.
+int plan_tile_for(int kernel) { return kernel == 2 ? 128 : ELITEKV_TILE_TOKENS; }
+int workers_for(const elitekv_layer* L, int kernel) { return kernel == 2 ? ekv_tc_workers(L) : 0; }
 
 // The workspace is sized for whichever kernel may be picked once the cache layout is known.
 int max_items_any(const elitekv_layer* L, int B) {
@@ -38,10 +30,6 @@ int max_items_any(const elitekv_layer* L, int B) {
   if (ekv_generic_supported(L) && (want == 0 || want == 1)) m = ekv_generic_max_items(L, B);
   if (ekv_tc_supported(L, nullptr) && (want == 0 || want == 2)) {
     const int t = ekv_tc_max_items(L, B);
-    if (t > m) m = t;
-  }
-  if (ekv_tc2_supported(L, nullptr) && (want == 0 || want == 3)) {
-    const int t = ekv_tc2_max_items(L, B);
     if (t > m) m = t;
   }
   return m;
@@ -78,7 +66,6 @@ extern "C" int elitekv_append(const elitekv_layer* L, const elitekv_cache* cache
   int rc = ekv_make_view(cache, &cv);
   if (rc != ELITEKV_OK) return rc;
   rc = ekv_launch_append(L, cache, cv, k_e, c, seq_id, pos, T, (cudaStream_t)stream);
-  EKV_STAGE_CHECK((cudaStream_t)stream, 1);
   return rc;
 }
 
@@ -88,7 +75,6 @@ extern "C" int elitekv_absorb_query(const elitekv_layer* L, const void* q, const
   if (((uintptr_t)q & 15) || ((uintptr_t)q_abs & 15) || ((uintptr_t)q_rope & 3))
     return ELITEKV_ERR_INVALID_ARG;
   int rc = ekv_launch_absorb(L, q, q_pos, B, q_rope, q_abs, (cudaStream_t)stream);
-  EKV_STAGE_CHECK((cudaStream_t)stream, 2);
   return rc;
 }
 
@@ -97,6 +83,18 @@ extern "C" int elitekv_decode_workspace_size(const elitekv_layer* L, int32_t B, 
   const int items = max_items_any(L, B);
   if (items <= 0) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
   *bytes = carve(L, B, items).total;
+  return ELITEKV_OK;
+}
+
+extern "C" int elitekv_decode_plan_info(const elitekv_layer* L, const elitekv_cache* cache, int32_t B,
+                                        int32_t info[4]) {
+  if (!L || !info || B <= 0) return ELITEKV_ERR_INVALID_ARG;
+  const int kernel = select_kernel(L, cache);
+  if (kernel < 0) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
+  info[0] = kernel;
+  info[1] = plan_tile_for(kernel);
+  info[2] = workers_for(L, kernel);
+  info[3] = max_items_for(L, B, kernel);
   return ELITEKV_OK;
 }
 
@@ -127,28 +125,26 @@ extern "C" int elitekv_decode(const elitekv_layer* L, const elitekv_cache* cache
   ws.counters = (int32_t*)(base + cw.off_cnt);
   ws.n_counters = ekv_combine_counters(L, B);
   ws.worker_first = (int32_t*)(base + cw.off_wfirst);
-  ws.n_workers = kernel == 3 ? ekv_tc2_workers(L) : kernel == 2 ? ekv_tc_workers(L) : 0;
+  ws.n_workers = workers_for(L, kernel);
   cudaStream_t st = (cudaStream_t)stream;
-  if (kernel == 3 || kernel == 2)
-    rc = ekv_launch_plan_balanced(seq_lens, B, kernel == 3 ? 32 : 128, ws.n_workers, max_items, ws.items,
-                                  ws.seq_first, ws.worker_first, ws.counters, ws.n_counters, st);
+  // tokens one sequence can hold: longer lengths are reported by the plan kernel and clamped
+  const long long max_len = cv.page_table ? (long long)cv.max_pages_per_seq << cv.page_shift : cv.max_ctx;
+  if (ws.n_workers > 0)
+    rc = ekv_launch_plan_balanced(seq_lens, B, plan_tile_for(kernel), ws.n_workers, max_items, ws.items, ws.seq_first,
+                                  ws.worker_first, ws.counters, ws.n_counters, max_len, L->d_status, st);
   else
-    rc = ekv_launch_plan(seq_lens, B, kernel == 2 ? 128 : ELITEKV_TILE_TOKENS, max_items, ws.items,
-                         ws.seq_first, ws.counters, ws.n_counters, st);
+    rc = ekv_launch_plan(seq_lens, B, plan_tile_for(kernel), max_items, ws.items, ws.seq_first,
+                         ws.counters, ws.n_counters, max_len, L->d_status, st);
   if (rc != ELITEKV_OK) return rc;
-  EKV_STAGE_CHECK(st, 3);
   EkvProfile* prof = (L->prof && L->prof->enabled && L->prof->count < kProfileSlots) ? L->prof : nullptr;
   if (prof) EKV_CUDA_OK(cudaEventRecord(prof->ev[2 * prof->count], st));
-  rc = kernel == 3   ? ekv_launch_decode_tc2(L, cache, cv, q_rope, q_abs, B, ws, st)
-       : kernel == 2 ? ekv_launch_decode_tc(L, cache, cv, q_rope, q_abs, B, ws, st)
-                     : ekv_launch_decode_generic(L, cache, cv, q_rope, q_abs, B, ws, st);
+  rc = kernel == 2 ? ekv_launch_decode_tc(L, cache, cv, q_rope, q_abs, B, ws, st)
+                   : ekv_launch_decode_generic(L, cache, cv, q_rope, q_abs, B, ws, st);
   if (rc != ELITEKV_OK) return rc;
   if (prof) {
     EKV_CUDA_OK(cudaEventRecord(prof->ev[2 * prof->count + 1], st));
     prof->count++;
   }
-  EKV_STAGE_CHECK(st, 4);
   rc = ekv_launch_combine(L, B, ws, out, st);
-  EKV_STAGE_CHECK(st, 5);
   return rc;
 }

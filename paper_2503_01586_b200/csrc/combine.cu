@@ -35,8 +35,10 @@ constexpr int kFI = 16;          // items per sequence whose merge weights are s
 constexpr int kFStage = 448;     // items per sequence group whose (m, l) are staged in shared memory
 
 __global__ void __launch_bounds__(kFThreads)
-combine_fast_kernel(const float* __restrict__ part_acc, const float* __restrict__ part_ml,
-                    const int32_t* __restrict__ seq_first, const bf16* __restrict__ Wuv,
+combine_fast_kernel(const float* part_acc, const float* part_ml,   // written by the split-K kernel while this
+                                                                   // kernel may already be resident: read
+                                                                   // with plain L2 loads, never ld.global.nc
+                    const int32_t* seq_first, const bf16* __restrict__ Wuv,
                     float* __restrict__ slice_out /* [n_slices][B][n_h][128] */,
                     int32_t* __restrict__ counters /* [n_h][n_groups], zeroed by the plan kernel */,
                     bf16* __restrict__ out, int B, int n_h, int d_c) {
@@ -65,15 +67,15 @@ combine_fast_kernel(const float* __restrict__ part_acc, const float* __restrict_
   for (int g = 0; g < n_groups; ++g) {
     const int b0 = g * kFB, nb = min(kFB, B - b0);
     __syncthreads();
-    if (tid <= nb) s_first[tid] = seq_first[b0 + tid];
+    if (tid <= nb) s_first[tid] = __ldcg(seq_first + b0 + tid);
     __syncthreads();
     // (m, l) of the group's items for this head: one trip to global memory, then shared
     const int gi0 = s_first[0], gin = s_first[nb] - gi0;
     for (int e = tid; e < min(gin, kFStage); e += kFThreads)
-      s_ml[e] = __ldg((const float2*)(part_ml + ((size_t)(gi0 + e) * n_h + h) * 2));
+      s_ml[e] = __ldcg((const float2*)(part_ml + ((size_t)(gi0 + e) * n_h + h) * 2));
     __syncthreads();
     auto item_ml = [&](int i) -> float2 {
-      return i - gi0 < kFStage ? s_ml[i - gi0] : __ldg((const float2*)(part_ml + ((size_t)i * n_h + h) * 2));
+      return i - gi0 < kFStage ? s_ml[i - gi0] : __ldcg((const float2*)(part_ml + ((size_t)i * n_h + h) * 2));
     };
     // softmax statistics per sequence: one warp each
     for (int bb = warp; bb < nb; bb += kFThreads / 32) {
@@ -118,7 +120,7 @@ combine_fast_kernel(const float* __restrict__ part_acc, const float* __restrict_
           float4 p[8];
 #pragma unroll
           for (int j = 0; j < 8; ++j)
-            p[j] = j0 + j < nfast ? __ldg((const float4*)(src + (size_t)(j0 + j) * stride)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            p[j] = j0 + j < nfast ? __ldcg((const float4*)(src + (size_t)(j0 + j) * stride)) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             const float w = j0 + j < nfast ? s_wt[bb][j0 + j] : 0.f;
@@ -128,7 +130,7 @@ combine_fast_kernel(const float* __restrict__ part_acc, const float* __restrict_
         }
         for (int j = kFI; j < ni; ++j) {     // rare: a sequence cut into more than kFI items
           const float w = exp2f(item_ml(i0 + j).x - s_M[bb]) * s_invL[bb];
-          const float4 p = __ldg((const float4*)(src + (size_t)j * stride));
+          const float4 p = __ldcg((const float4*)(src + (size_t)j * stride));
           acc.x = fmaf(w, p.x, acc.x); acc.y = fmaf(w, p.y, acc.y);
           acc.z = fmaf(w, p.z, acc.z); acc.w = fmaf(w, p.w, acc.w);
         }

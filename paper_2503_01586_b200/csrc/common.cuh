@@ -34,6 +34,7 @@ struct elitekv_layer {
   bf16* d_Wuv;                     // [d_c][n_h*d_h] private copy
   int32_t* d_status;               // [4] device status word: code, detail0, detail1, count
   struct EkvProfile* prof;         // optional event pairs around the split-K kernel
+  int32_t* last_detail;            // host [3]: detail words + count read by the last check_status
 };
 
 constexpr int kProfileSlots = 512;
@@ -142,12 +143,16 @@ int ekv_launch_append(const elitekv_layer* L, const elitekv_cache* cache, const 
                       long long T, cudaStream_t st);
 int ekv_launch_absorb(const elitekv_layer* L, const void* q, const int32_t* q_pos, int B,
                       void* q_rope, void* q_abs, cudaStream_t st);
+// max_len: tokens one sequence can hold in the cache; longer (or negative) lengths are recorded
+// in `status` (may be null) as BAD_POSITION and clamped.
 int ekv_launch_plan(const int32_t* seq_lens, int B, int tile_tokens, int max_items, int32_t* items,
-                    int32_t* seq_first_item, int32_t* zero_ints, int n_zero, cudaStream_t st);
+                    int32_t* seq_first_item, int32_t* zero_ints, int n_zero, long long max_len,
+                    int32_t* status, cudaStream_t st);
 
 int ekv_launch_plan_balanced(const int32_t* seq_lens, int B, int tile_tokens, int n_workers,
                              int max_items, int32_t* items, int32_t* seq_first_item,
-                             int32_t* worker_first, int32_t* zero_ints, int n_zero, cudaStream_t st);
+                             int32_t* worker_first, int32_t* zero_ints, int n_zero, long long max_len,
+                             int32_t* status, cudaStream_t st);
 
 struct DecodeScratch {
   int max_items;          // capacity of the plan
@@ -177,11 +182,5 @@ int ekv_tc_workers(const elitekv_layer* L);
 int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, const CacheView& cv,
                          const void* q_rope, const void* q_abs, int B, const DecodeScratch& ws,
                          cudaStream_t st);
-int ekv_tc2_supported(const elitekv_layer* L, const elitekv_cache* cache);  // cache may be null
-int ekv_tc2_workers(const elitekv_layer* L);
-int ekv_tc2_max_items(const elitekv_layer* L, int B);
-int ekv_launch_decode_tc2(const elitekv_layer* L, const elitekv_cache* cache, const CacheView& cv,
-                          const void* q_rope, const void* q_abs, int B, const DecodeScratch& ws,
-                          cudaStream_t st);
 int ekv_launch_combine(const elitekv_layer* L, int B, const DecodeScratch& ws, void* out,
                        cudaStream_t st);

@@ -86,7 +86,8 @@ struct Smem {
   __host__ __device__ static constexpr int p_off(int d_c) { return rope_off(d_c) + kRopeSlots * kChunkBytes; }
   static constexpr int p_bytes = kTile * N * 2;
   __host__ __device__ static constexpr int misc_off(int d_c) { return p_off(d_c) + p_bytes; }
-  // misc: q_rope fp32 [N][R2max=32] 4 KB | wmax [4][N] | corr [N] | barriers | tmem base | abort
+  // misc: q_rope fp32 [N][R2max=32] 4 KB | wmax [4][N] | corr [N] | barriers | tmem base | abort |
+  // the two outcome words of the group waits
   static constexpr int misc_bytes = N * 32 * 4 + 4 * N * 4 + N * 4 + (int)sizeof(TcBarriers) + 64;
   __host__ __device__ static constexpr int total(int d_c) { return misc_off(d_c) + misc_bytes + 1024; }
 };
@@ -119,9 +120,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   TcBarriers* bars = (TcBarriers*)(s_corr + N);
   uint32_t* s_tmem = (uint32_t*)(bars + 1);
   volatile int* s_abort = (volatile int*)(s_tmem + 1);
+  volatile int* s_verdict = s_abort + 1;     // [2] outcome words of the softmax threads' group waits
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  EKV_STAMP_DECL;
 
   if (threadIdx.x == 32) {
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_lat128) : "memory");
@@ -168,6 +169,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
 
   // running counters (each role advances its own copies identically): ring uses, tiles, items
   unsigned lat_n = 0, rope_n = 0, tbase = 0;
+  unsigned gw_turn = 0;      // group waits taken so far by the softmax threads
   int seq = -1;
   for (int item = item_lo; item < item_hi; ++item) {
   seq = a.items[4 * item + 0];
@@ -233,7 +235,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
             mbar_expect_tx(fb, (uint32_t)(halves * 8192 + (with_q ? N * 128 : 0)));
             if (with_q)   // the sequence's absorbed queries for these 64 latent coordinates (L2-resident)
               tma_load_2d_hint(smem_u32(s_lat + slot * kSlot + kChunkBytes), &map_q, kc * 64, seq * a.n_h + h0, fb, pol_keep);
-            if (prod == 0 && kc == 0) EKV_STAMP(0, with_q ? 100 : 200, tile);
             const uint64_t pol = with_q ? pol_keep : pol_drop;
             if (whole) {
               tma_load_2d_hint(smem_u32(s_lat + slot * kSlot), &map_lat128, kc * 64, (int)row[0], fb, pol);
@@ -289,7 +290,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       const unsigned n0 = lat_n;                 // first ring use of this tile
       // ---- pass A: NKC chunks, 4 K-steps of 16 latent coordinates each
       unsigned slot = n0 % kLatSlots, par = (n0 / kLatSlots) & 1;
-      if (elect_one()) EKV_STAMP(1, 300, tile);
       for (int kc = 0; kc < NKC; ++kc) {
         const uint32_t fb = full0 + slot * 8;
         ok = warp_wait(fb, par, s_abort, 3);
@@ -306,16 +306,12 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         if (++slot == kLatSlots) { slot = 0; par ^= 1; }
       }
       if (!ok) break;
-      if (elect_one()) {
-        tc_commit(smem_u32(&bars->s_full));
-        EKV_STAMP(1, 20, tile);
-      }
+      if (elect_one()) tc_commit(smem_u32(&bars->s_full));
       __syncwarp();
       // ---- wait for P (and the rescaled output) of this tile
       ok = warp_wait(smem_u32(&bars->p_ready), (tbase + tile) & 1, s_abort, 4);
       if (!ok) break;
       tc_fence_after();
-      if (elect_one()) EKV_STAMP(1, 21, tile);
       // ---- pass B: NB output blocks of 128 latent coordinates = one even/odd slot pair each
       const unsigned nb0 = n0 + NKC;
       slot = nb0 % kLatSlots;
@@ -360,10 +356,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         if (slot >= kLatSlots) { slot -= kLatSlots; par ^= 1; }
       }
       if (!ok) break;
-      if (elect_one()) {
-        tc_commit(smem_u32(&bars->pv_done));
-        EKV_STAMP(1, 22, tile);
-      }
+      if (elect_one()) tc_commit(smem_u32(&bars->pv_done));
       __syncwarp();
       lat_n = n0 + 2u * (unsigned)NKC;
     }
@@ -378,6 +371,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
     for (int h = 0; h < N; ++h) l_part[h] = 0.f;
     float m_ref = -INFINITY;                      // lane h holds head h's reference max (N <= 32 per group)
     bool ok = true;
+    const bool leader = threadIdx.x == 64;
     static_assert(N == 16 || N == 32, "softmax threads keep one head per lane (lanes >= N idle)");
 
     for (int tile = 0; tile < n_tiles && ok; ++tile) {
@@ -390,7 +384,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       for (int cb = 0; cb < NRB; ++cb) {
         if (!ok) break;
         const unsigned slot = rope_n % kRopeSlots;
-        ok = mbar_wait_group(smem_u32(&bars->rope_full[slot]), (rope_n / kRopeSlots) & 1, s_abort, threadIdx.x == 64, 2, kSoftmaxThreads, 6);
+        ok = mbar_wait_group(smem_u32(&bars->rope_full[slot]), (rope_n / kRopeSlots) & 1, s_abort, s_verdict, gw_turn, leader, 2, kSoftmaxThreads, 6);
         if (!ok) break;
         const unsigned char* rowp = s_rope + slot * kChunkBytes + trow * 128;
         float part[HPB];
@@ -419,12 +413,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         ++rope_n;
       }
       if (!ok) break;
-      if (threadIdx.x == 64) EKV_STAMP(2, 30, tile);
       // ---- latent part from TMEM
-      ok = mbar_wait_group(smem_u32(&bars->s_full), (tbase + tile) & 1, s_abort, threadIdx.x == 64, 2, kSoftmaxThreads, 7);
+      ok = mbar_wait_group(smem_u32(&bars->s_full), (tbase + tile) & 1, s_abort, s_verdict, gw_turn, leader, 2, kSoftmaxThreads, 7);
       if (!ok) break;
       tc_fence_after();
-      if (threadIdx.x == 64) EKV_STAMP(2, 31, tile);
       {
         float sv[N];
         tc_ld_cols<N>(tmem_s + lane_base, sv);
@@ -493,7 +485,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       fence_proxy_async();
       tc_fence_before();
       mbar_arrive(smem_u32(&bars->p_ready));
-      if (threadIdx.x == 64) EKV_STAMP(2, 41, tile);
     }
 
     // ---- epilogue: softmax statistics of this item (while the last pass B still runs) ...
@@ -514,7 +505,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       }
     }
     // ---- ... and its partial output
-    ok = mbar_wait_group(smem_u32(&bars->pv_done), (tbase + n_tiles - 1) & 1, s_abort, threadIdx.x == 64, 2, kSoftmaxThreads, 8) && ok;
+    ok = mbar_wait_group(smem_u32(&bars->pv_done), (tbase + n_tiles - 1) & 1, s_abort, s_verdict, gw_turn, leader, 2, kSoftmaxThreads, 8) && ok;
     if (ok) {
       tc_fence_after();
       // The output block [128 coords x N heads] leaves TMEM with one thread per coordinate; it is
@@ -649,14 +640,3 @@ int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, con
     default: return launch(decode_tc_kernel<16, 32>);
   }
 }
-
-#ifdef EKV_TIMELINE
-extern "C" int elitekv_debug_timeline(unsigned long long* host_out, int max_words, int reset) {
-  void* p = nullptr;
-  if (cudaGetSymbolAddress(&p, g_ekv_timeline) != cudaSuccess) return ELITEKV_ERR_CUDA;
-  if (host_out && cudaMemcpy(host_out, p, sizeof(unsigned long long) * (size_t)max_words, cudaMemcpyDeviceToHost) != cudaSuccess)
-    return ELITEKV_ERR_CUDA;
-  if (reset && cudaMemset(p, 0, sizeof(unsigned long long) * 3 * 8192) != cudaSuccess) return ELITEKV_ERR_CUDA;
-  return ELITEKV_OK;
-}
-#endif

@@ -69,8 +69,10 @@ extern "C" int elitekv_layer_create(const elitekv_params* p, elitekv_layer** out
   L->scale = p->softmax_scale > 0.f ? p->softmax_scale : (float)(1.0 / sqrt((double)d_h));
   L->pair_mode = p->pair_mode; L->max_pos = p->max_pos; L->decode_kernel = p->decode_kernel;
 
+  L->last_detail = (int32_t*)calloc(3, sizeof(int32_t));
   int rc = ELITEKV_ERR_CUDA;
   do {
+    if (!L->last_detail) break;
     if (cudaGetDevice(&L->device) != cudaSuccess) break;
     if (cudaDeviceGetAttribute(&L->sm_count, cudaDevAttrMultiProcessorCount, L->device) != cudaSuccess) break;
     if (cudaDeviceGetAttribute(&L->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, L->device) != cudaSuccess) break;
@@ -134,6 +136,7 @@ extern "C" int elitekv_layer_destroy(elitekv_layer* L) {
       if (L->prof->ev[i]) cudaEventDestroy(L->prof->ev[i]);
     free(L->prof);
   }
+  free(L->last_detail);
   free(L);
   return ELITEKV_OK;
 }
@@ -145,10 +148,16 @@ extern "C" int elitekv_check_status(const elitekv_layer* L, elitekv_stream_t str
   EKV_CUDA_OK(cudaMemcpyAsync(h, L->d_status, sizeof(h), cudaMemcpyDeviceToHost, st));
   EKV_CUDA_OK(cudaMemsetAsync(L->d_status, 0, sizeof(h), st));
   EKV_CUDA_OK(cudaStreamSynchronize(st));
-#ifdef EKV_SYNC_EACH
-  if (h[0] != 0) fprintf(stderr, "elitekv status %d detail %d (0x%x) %d count %d\n", h[0], h[1], h[1], h[2], h[3]);
-#endif
+  L->last_detail[0] = h[1];
+  L->last_detail[1] = h[2];
+  L->last_detail[2] = h[3];
   return h[0];
+}
+
+extern "C" int elitekv_last_status_detail(const elitekv_layer* L, int32_t detail[3]) {
+  if (!L || !detail) return ELITEKV_ERR_INVALID_ARG;
+  for (int i = 0; i < 3; ++i) detail[i] = L->last_detail[i];
+  return ELITEKV_OK;
 }
 
 extern "C" const char* elitekv_strerror(int status) {

@@ -36,10 +36,23 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int* t
   return before + incl - v;
 }
 
+// Length of sequence b as the kernels may use it: a length beyond what the cache can hold per
+// sequence (or a negative one) is recorded as BAD_POSITION and clamped, so that no kernel
+// downstream walks into another sequence's rows.  Only `report` threads record.
+__device__ __forceinline__ int checked_len(const int32_t* seq_lens, int b, long long max_len, int32_t* status,
+                                           bool report) {
+  int n = seq_lens[b];
+  if (n < 0 || n > max_len) {
+    if (report && status) ekv_record(status, ELITEKV_ERR_BAD_POSITION, b, n);
+    n = n < 0 ? 0 : (int)max_len;
+  }
+  return n;
+}
+
 __global__ void __launch_bounds__(kPlanThreads)
 plan_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int max_items,
             int32_t* __restrict__ items, int32_t* __restrict__ seq_first,
-            int32_t* __restrict__ zero_ints, int n_zero) {
+            int32_t* __restrict__ zero_ints, int n_zero, long long max_len, int32_t* status) {
   __shared__ int warp_tot[kPlanThreads / 32];
   __shared__ long long s_total;
   const int t = threadIdx.x;
@@ -48,7 +61,7 @@ plan_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int max_items
   __syncthreads();
   long long local = 0;
   for (int b = t; b < B; b += blockDim.x) {
-    int n = seq_lens[b];
+    int n = checked_len(seq_lens, b, max_len, status, true);
     local += n > 0 ? (n + tile - 1) / tile : 0;
   }
   if (local) atomicAdd((unsigned long long*)&s_total, (unsigned long long)local);
@@ -63,7 +76,7 @@ plan_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int max_items
     const int b = b0 + t;
     int n = 0, tiles = 0, pieces = 0;
     if (b < B) {
-      n = seq_lens[b];
+      n = checked_len(seq_lens, b, max_len, status, false);
       tiles = n > 0 ? (n + tile - 1) / tile : 0;
       pieces = (int)((tiles + target - 1) / target);
     }
@@ -94,7 +107,8 @@ plan_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int max_items
 __global__ void __launch_bounds__(kPlanThreads)
 plan_balanced_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int n_workers,
                      int max_items, int32_t* __restrict__ items, int32_t* __restrict__ seq_first,
-                     int32_t* __restrict__ worker_first, int32_t* __restrict__ zero_ints, int n_zero) {
+                     int32_t* __restrict__ worker_first, int32_t* __restrict__ zero_ints, int n_zero,
+                     long long max_len, int32_t* status) {
   __shared__ int warp_tot[kPlanThreads / 32];
   __shared__ long long s_total;
   const int t = threadIdx.x;
@@ -105,7 +119,7 @@ plan_balanced_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int 
   __syncthreads();
   long long local = 0;
   for (int b = t; b < B; b += blockDim.x) {
-    int n = seq_lens[b];
+    int n = checked_len(seq_lens, b, max_len, status, true);
     local += n > 0 ? (n + tile - 1) / tile : 0;
   }
   if (local) atomicAdd((unsigned long long*)&s_total, (unsigned long long)local);
@@ -124,7 +138,7 @@ plan_balanced_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int 
       const int b = b0 + t;
       int n = 0, tiles = 0;
       if (b < B) {
-        n = seq_lens[b];
+        n = checked_len(seq_lens, b, max_len, status, false);
         tiles = n > 0 ? (n + tile - 1) / tile : 0;
       }
       int chunk_tiles;
@@ -167,17 +181,20 @@ plan_balanced_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int 
 
 int ekv_launch_plan_balanced(const int32_t* seq_lens, int B, int tile_tokens, int n_workers,
                              int max_items, int32_t* items, int32_t* seq_first_item,
-                             int32_t* worker_first, int32_t* zero_ints, int n_zero, cudaStream_t st) {
+                             int32_t* worker_first, int32_t* zero_ints, int n_zero, long long max_len,
+                             int32_t* status, cudaStream_t st) {
   EKV_CUDA_OK(ekv_launch_pdl(plan_balanced_kernel, dim3(1), dim3(kPlanThreads), 0, st, seq_lens, B, tile_tokens,
-                             n_workers, max_items, items, seq_first_item, worker_first, zero_ints, n_zero));
+                             n_workers, max_items, items, seq_first_item, worker_first, zero_ints, n_zero,
+                             max_len, status));
   EKV_CUDA_OK(cudaGetLastError());
   return ELITEKV_OK;
 }
 
 int ekv_launch_plan(const int32_t* seq_lens, int B, int tile_tokens, int max_items, int32_t* items,
-                    int32_t* seq_first_item, int32_t* zero_ints, int n_zero, cudaStream_t st) {
+                    int32_t* seq_first_item, int32_t* zero_ints, int n_zero, long long max_len,
+                    int32_t* status, cudaStream_t st) {
   plan_kernel<<<1, kPlanThreads, 0, st>>>(seq_lens, B, tile_tokens, max_items, items, seq_first_item,
-                                          zero_ints, n_zero);
+                                          zero_ints, n_zero, max_len, status);
   EKV_CUDA_OK(cudaGetLastError());
   return ELITEKV_OK;
 }
@@ -189,5 +206,17 @@ extern "C" int elitekv_plan(const int32_t* seq_lens, int32_t B, int32_t tile_tok
     return ELITEKV_ERR_INVALID_ARG;
   if ((uintptr_t)items & 15) return ELITEKV_ERR_INVALID_ARG;
   return ekv_launch_plan(seq_lens, B, tile_tokens, max_items, items, seq_first_item, nullptr, 0,
-                         (cudaStream_t)stream);
+                         0x7fffffffLL, nullptr, (cudaStream_t)stream);
+}
+
+extern "C" int elitekv_plan_workers(const int32_t* seq_lens, int32_t B, int32_t tile_tokens,
+                                    int32_t n_workers, int32_t max_items, int32_t* items,
+                                    int32_t* seq_first_item, int32_t* worker_first,
+                                    elitekv_stream_t stream) {
+  if (!seq_lens || !items || !seq_first_item || !worker_first || B <= 0 || tile_tokens <= 0 ||
+      n_workers <= 0 || max_items < B + n_workers)
+    return ELITEKV_ERR_INVALID_ARG;
+  if ((uintptr_t)items & 15) return ELITEKV_ERR_INVALID_ARG;
+  return ekv_launch_plan_balanced(seq_lens, B, tile_tokens, n_workers, max_items, items, seq_first_item,
+                                  worker_first, nullptr, 0, 0x7fffffffLL, nullptr, (cudaStream_t)stream);
 }

@@ -1,6 +1,6 @@
 // Inline-PTX wrappers for the sm_100a tensor-core kernels: mbarrier, TMA (cp.async.bulk.tensor),
-// tcgen05 (MMA, commit, TMEM load/store, fences), shared-memory matrix descriptors, and the
-// cluster primitives the paired kernel uses.  Every wait helper is bounded.
+// tcgen05 (MMA, commit, TMEM load/store, fences) and shared-memory matrix descriptors.  Every
+// wait helper is bounded.
 #pragma once
 
 #include <cuda.h>
@@ -8,26 +8,6 @@
 #include "common.cuh"
 
 constexpr unsigned kWaitLimit = 1u << 20;   // polls of mbarrier.try_wait before giving up
-
-// Optional in-kernel event timeline (compiled in with -DEKV_TIMELINE): four roles of block 0
-// append (event code, tile, nanosecond timer) records; elitekv_debug_timeline copies them out.
-#ifdef EKV_TIMELINE
-__device__ unsigned long long g_ekv_timeline[3 * 8192];
-__device__ __forceinline__ void ekv_stamp(int role, unsigned& idx, int code, int tile) {
-  if (blockIdx.x != 0 || idx >= 2048) return;
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  const unsigned i = role * 2048 + idx++;
-  g_ekv_timeline[3 * i] = (unsigned long long)code;
-  g_ekv_timeline[3 * i + 1] = (unsigned long long)tile;
-  g_ekv_timeline[3 * i + 2] = t;
-}
-#define EKV_STAMP_DECL unsigned ekv_stamp_idx = 0
-#define EKV_STAMP(role, code, tile) ekv_stamp(role, ekv_stamp_idx, code, tile)
-#else
-#define EKV_STAMP_DECL
-#define EKV_STAMP(role, code, tile) ((void)0)
-#endif
 
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -51,7 +31,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int why = 1);
 // True in exactly one lane of a fully converged warp.  Code that issues tcgen05.mma or TMA runs
 // warp-uniformly with only the instruction itself under this predicate: operands of those
 // instructions then live in uniform registers, which was measured to matter (42 clocks per
@@ -75,32 +54,40 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded busy wait on test_wait for the threads on the critical hand-off path (MMA issuer, TMA
-// producers): same contract as mbar_wait, 16 times the poll budget because a probe is cheap.
-__device__ __forceinline__ bool mbar_spin(uint32_t bar, uint32_t parity, volatile int* abort_flag, int why = 1) {
-  for (unsigned i = 0; i < 16u * kWaitLimit; ++i) {
+// Every wait below is bounded: after `limit` probes the waiter writes `why` (a small positive
+// code that names the wait) to the block's abort flag, unless somebody else gave up first, and
+// returns false; it also returns false when it sees the flag set by another role.  The kernels
+// pass kSpinLimit (seconds of probing, far beyond any legitimate wait); the self-test kernel
+// passes a short limit to make a wait run out on purpose.
+constexpr unsigned kSpinLimit = 16u * kWaitLimit;
+
+// Busy wait of a single thread on test_wait.
+__device__ __forceinline__ bool mbar_spin(uint32_t bar, uint32_t parity, volatile int* abort_flag, int why,
+                                          unsigned limit = kSpinLimit) {
+  for (unsigned i = 0; i < limit; ++i) {
     if (mbar_test_wait(bar, parity)) return true;
     if ((i & 4095) == 4095 && *abort_flag) return false;
   }
   if (*abort_flag == 0) *abort_flag = why;
   return false;
 }
-// Warp-uniform bounded wait on one phase for a fully converged warp: every lane probes and any
-// lane's success counts for all (a phase that this warp waits for cannot be undone by anybody
-// else), so the lanes can never disagree about the outcome.
-__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int why) {
+// Warp-uniform wait of a fully converged warp: every lane probes and any lane's success counts
+// for all (a phase that this warp waits for cannot be undone by anybody else), so the lanes can
+// never disagree about the outcome.
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int why,
+                                          unsigned limit = kSpinLimit) {
   if (__any_sync(0xffffffffu, mbar_test_wait(bar, parity))) return true;
-  for (unsigned i = 0; i < 16u * kWaitLimit; ++i) {
+  for (unsigned i = 0; i < limit; ++i) {
     if (__any_sync(0xffffffffu, mbar_test_wait(bar, parity))) return true;
     if ((i & 4095) == 4095 && __any_sync(0xffffffffu, *abort_flag != 0)) return false;
   }
   if (*abort_flag == 0) *abort_flag = why;
   return false;
 }
-// Bounded wait; returns false when the limit is hit (the block's abort flag is then set to `why`,
-// a small positive code that names the wait) or when another thread has already given up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int why) {
-  for (unsigned i = 0; i < kWaitLimit; ++i) {
+// Wait of many independent threads on try_wait (which may park the thread between probes).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int why,
+                                          unsigned limit = kWaitLimit) {
+  for (unsigned i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 1023) == 1023 && *abort_flag) return false;
   }
@@ -114,13 +101,23 @@ __device__ __forceinline__ void drain_after_abort() {
 }
 // Group wait for long waits of many threads: one leader polls the mbarrier, the others sleep in
 // a hardware named barrier (polling threads hammer the shared-memory pipe that feeds the tensor
-// core).  Afterwards every thread confirms the phase itself (one immediate try_wait = its own
-// acquire); false means the block is aborting.  All `n` threads of barrier `id` must call it.
-__device__ __forceinline__ bool mbar_wait_group(uint32_t bar, uint32_t parity, volatile int* abort_flag, bool leader,
-                                                int id, int n, int why = 1) {
-  if (leader) (void)mbar_spin(bar, parity, abort_flag, why);
+// core).  The leader's outcome is the outcome for everybody: it leaves it in verdict[turn & 1]
+// before the named barrier and every thread returns that word, so the group can never split
+// into threads that go on and threads that give up.  `turn` is the caller's count of group
+// waits (the same in all threads); two words are enough because the leader cannot get two waits
+// ahead of a thread that has not passed the barrier of the previous one.  A thread that goes on
+// confirms the phase itself (one immediate try_wait = its own acquire).  All `n` threads of
+// barrier `id` must call it.
+__device__ __forceinline__ bool mbar_wait_group(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                volatile int* verdict, unsigned& turn, bool leader, int id, int n,
+                                                int why, unsigned limit = kSpinLimit) {
+  volatile int* word = verdict + (turn & 1u);
+  ++turn;
+  if (leader) *word = mbar_spin(bar, parity, abort_flag, why, limit) ? 1 : 0;
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory");
-  return mbar_try_wait(bar, parity);
+  const bool ok = *word != 0;
+  if (ok) (void)mbar_try_wait(bar, parity);
+  return ok;
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
@@ -267,46 +264,6 @@ __device__ __forceinline__ int f2ord(float f) {
 }
 __device__ __forceinline__ float ord2f(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
 
-
-// ---------------------------------------------------------------- cluster / distributed smem
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// address of the same shared-memory location in CTA `rank` of the cluster
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ void st_cluster_f4(uint32_t caddr, float4 v) {
-  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(caddr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cbar) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cbar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (unsigned i = 0; i < kWaitLimit; ++i) {
-    if (mbar_try_wait_cluster(bar, parity)) return true;
-    if ((i & 1023) == 1023 && *abort_flag) return false;
-  }
-  *abort_flag = 1;
-  return false;
-}
 
 // ---------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,

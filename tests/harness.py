@@ -49,9 +49,12 @@ class State:
 
 
 def setup(w: gen.Workload, *, lens: Optional[Sequence[int]] = None, decode_kernel: int = 0,
-          pos_offset: int = 0, cos_sin=None, fill: bool = True, device="cuda") -> State:
+          pos_offset: int = 0, cos_sin=None, fill: bool = True, device="cuda",
+          q_scale: float = 1.0, edit_tokens=None) -> State:
     """Builds layer, cache planes and the token stream; when `fill`, appends every token of
-    every sequence (so the cache holds lens[b] tokens, the last being the decoding token)."""
+    every sequence (so the cache holds lens[b] tokens, the last being the decoding token).
+    `q_scale` multiplies the drawn queries (exactly, for a power of two); `edit_tokens(st)` may
+    overwrite rows of st.k_e / st.c before they are appended."""
     idx = gen.elite_index_sets(w)
     W_uk, W_uv = gen.up_projections(w, device)
     lens_t = gen.sequence_lengths(w) if lens is None else torch.tensor(list(lens), dtype=torch.int32)
@@ -64,6 +67,8 @@ def setup(w: gen.Workload, *, lens: Optional[Sequence[int]] = None, decode_kerne
     pos = torch.cat([torch.arange(int(n), dtype=torch.int32) for n in lens_t.tolist()]) if N else \
         torch.zeros(0, dtype=torch.int32)
     q = gen.queries(w, device)
+    if q_scale != 1.0:
+        q = (q.float() * q_scale).to(torch.bfloat16)
     q_pos = (lens_t - 1).clamp(min=0)
     max_pos = int(lens_t.max().item()) + 2 if B else 2
     if pos_offset:
@@ -92,6 +97,8 @@ def setup(w: gen.Workload, *, lens: Optional[Sequence[int]] = None, decode_kerne
     st = State(w, idx, W_uk, W_uv, lens_t, starts, k_e, c, seq_id.to(device), pos.to(device), q,
                q_pos.to(torch.int32).to(device), layer, cache, rope_plane, latent_plane, page_table,
                lens_t.to(device), ws, pos_offset)
+    if edit_tokens is not None:
+        edit_tokens(st)
     if fill and N:
         ek.elitekv_append(layer, cache, st.k_e, st.c, st.seq_id, st.pos)
     return st

@@ -270,7 +270,12 @@ def test_back_to_back_steps_share_one_workspace(ek):
     H.check_parity(st, alone1, H.all_units(st))
 
 
-@pytest.mark.parametrize("kernel", [1, 2, 3], ids=["generic", "tensor-core", "tensor-core-pair"])
+KERNELS = [1, 2]
+KERNEL_IDS = ["generic", "two-pass"]
+TC_KERNELS, TC_KERNEL_IDS = KERNELS[1:], KERNEL_IDS[1:]
+
+
+@pytest.mark.parametrize("kernel", KERNELS, ids=KERNEL_IDS)
 def test_decode_7b_shape_ragged_tails_both_kernels(ek, kernel):
     """Same inputs through the CUDA-core kernel and the tcgen05 kernel: lengths around the
     16-token MMA step and the 128-token tile."""
@@ -280,7 +285,7 @@ def test_decode_7b_shape_ragged_tails_both_kernels(ek, kernel):
     H.check_parity(st, out, H.all_units(st))
 
 
-@pytest.mark.parametrize("kernel", [2, 3], ids=["tensor-core", "tensor-core-pair"])
+@pytest.mark.parametrize("kernel", TC_KERNELS, ids=TC_KERNEL_IDS)
 @pytest.mark.parametrize("page_size", [64, 128])
 def test_decode_7b_shape_paged_tensor_core(ek, page_size, kernel):
     w = replace(gen.shrink(gen.LLAMA7B_75, B=3, ctx=700), paged=True, page_size=page_size)
@@ -289,21 +294,74 @@ def test_decode_7b_shape_paged_tensor_core(ek, page_size, kernel):
     H.check_parity(st, out, H.all_units(st))
 
 
-def test_pair_kernel_many_items_per_worker(ek):
-    """More sequences than workers can split evenly: workers walk several items, some of them
-    a few tiles long, and sequences are cut at arbitrary 32-token boundaries."""
-    w = gen.shrink(gen.LLAMA7B_75, B=40, ctx=300)
-    lens = [1 + (37 * i) % 300 for i in range(40)]
-    st = H.setup(w, lens=lens, decode_kernel=3)
+@pytest.mark.parametrize("kernel", TC_KERNELS, ids=TC_KERNEL_IDS)
+def test_tensor_core_kernels_many_items_per_worker(ek, kernel):
+    """Many short sequences: workers walk several items, some of them a few tiles long, and
+    sequences are cut at tile boundaries that fall anywhere."""
+    w = gen.shrink(gen.LLAMA7B_75, B=300, ctx=300)
+    lens = [1 + (37 * i) % 300 for i in range(300)]
+    st = H.setup(w, lens=lens, decode_kernel=kernel)
     out = H.run_decode(st)
+    assert torch.isfinite(out.float()).all()
     H.check_parity(st, out, H.sample_units(st, 96))
 
 
-def test_pair_kernel_87_5pct_shape(ek):
+@pytest.mark.parametrize("kernel", TC_KERNELS, ids=TC_KERNEL_IDS)
+def test_tensor_core_kernels_87_5pct_shape(ek, kernel):
     w = gen.shrink(gen.SWEEP_875, B=3, ctx=500)
-    st = H.setup(w, lens=[500, 33, 160], decode_kernel=3)
+    st = H.setup(w, lens=[500, 33, 160], decode_kernel=kernel)
     out = H.run_decode(st)
     H.check_parity(st, out, H.all_units(st))
+
+
+# ------------------------------------------------------------------ faults the device reports
+@pytest.mark.parametrize("kernel", KERNELS, ids=KERNEL_IDS)
+def test_decode_overlong_length_is_reported_and_clamped(ek, kernel):
+    """A length beyond the rows a sequence owns must not reach into the next sequence's rows:
+    the plan records BAD_POSITION (sequence, length), clamps, and the other sequences' outputs
+    are bit for bit what they are without the fault."""
+    w = gen.shrink(gen.LLAMA7B_75, B=3, ctx=200)
+    st = H.setup(w, lens=[200, 150, 90], decode_kernel=kernel)
+    good = H.run_decode(st).clone()
+    bad_lens = st.lens_dev.clone()
+    bad_lens[1] = st.cache.max_ctx + 77
+    q_rope, q_abs = ek.elitekv_absorb_query(st.layer, st.q, st.q_pos)
+    out = ek.elitekv_decode(st.layer, st.cache, q_rope, q_abs, bad_lens, st.workspace)
+    assert ek.elitekv_check_status(st.layer) == ek.ERR_BAD_POSITION
+    assert ek.elitekv_last_status_detail(st.layer)[:2] == (1, st.cache.max_ctx + 77)
+    assert torch.equal(out[0], good[0]) and torch.equal(out[2], good[2])
+    assert torch.isfinite(out.float()).all()
+    assert torch.equal(H.run_decode(st), good)        # the layer is usable afterwards
+
+
+@pytest.mark.parametrize("kernel", KERNELS, ids=KERNEL_IDS)
+def test_decode_bad_page_id_is_reported(ek, kernel):
+    w = replace(gen.shrink(gen.LLAMA7B_75, B=3, ctx=300), paged=True, page_size=64)
+    st = H.setup(w, lens=[300, 200, 100], decode_kernel=kernel)
+    good = H.run_decode(st).clone()
+    keep = st.page_table[1, 1].item()
+    st.page_table[1, 1] = st.cache.num_pages + 5
+    q_rope, q_abs = ek.elitekv_absorb_query(st.layer, st.q, st.q_pos)
+    out = ek.elitekv_decode(st.layer, st.cache, q_rope, q_abs, st.lens_dev, st.workspace)
+    assert ek.elitekv_check_status(st.layer) == ek.ERR_BAD_PAGE
+    assert ek.elitekv_last_status_detail(st.layer)[:2] == (1, st.cache.num_pages + 5)
+    assert torch.equal(out[0], good[0]) and torch.equal(out[2], good[2])
+    st.page_table[1, 1] = keep
+    assert torch.equal(H.run_decode(st), good)
+
+
+def test_bounded_waits_give_up_and_report(ek):
+    """A wait that cannot complete must end with TIMEOUT in the status word, for every wait
+    helper the tensor-core kernels use; the context stays usable."""
+    w = gen.shrink(gen.LLAMA7B_75, B=2, ctx=200)
+    st = H.setup(w, lens=[200, 67])
+    good = H.run_decode(st).clone()
+    for limit in (1, 100, 5000):
+        ek.elitekv_selftest_bounded_wait(st.layer, limit)
+        assert ek.elitekv_check_status(st.layer) == ek.ERR_TIMEOUT
+        assert ek.elitekv_last_status_detail(st.layer) == (7, limit, 1)
+    assert ek.elitekv_check_status(st.layer) == 0
+    assert torch.equal(H.run_decode(st), good)
 
 
 def test_tensor_core_kernel_refuses_uncovered_shapes(ek):
@@ -374,6 +432,52 @@ def test_plan_partitions_every_sequence(ek, lens, max_items):
         budget = max_items - len(lens)
         target = max(1, -(-total_tiles // budget))
         assert max(sizes) <= target * 64
+
+
+def _plan_cases():
+    return [([4096] * 16, 128, 148), ([4096] * 16, 64, 148), ([1], 64, 148), ([64, 65, 0, 1000], 64, 7),
+            (list(range(1, 3000, 37)), 128, 49), ([100000, 3], 64, 148), ([0, 0, 5], 128, 3),
+            ([1024 + (7919 * i) % 31744 for i in range(64)], 64, 148)]
+
+
+@pytest.mark.parametrize("lens,tile,n_workers", _plan_cases())
+def test_worker_plan_structure(ek, lens, tile, n_workers):
+    """The persistent-worker plan: every sequence is partitioned into consecutive items that
+    start on tile boundaries; items are ordered by worker; worker w holds exactly the tiles
+    [w*quota, (w+1)*quota) of the batch's tile list; worker_first is monotone and covers all."""
+    B = len(lens)
+    t = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    max_items = B + n_workers
+    items, first, wfirst = ek.elitekv_plan_workers(t, tile, n_workers, max_items)
+    torch.cuda.synchronize()
+    items, first, wfirst = items.cpu().numpy(), first.cpu().numpy(), wfirst.cpu().numpy()
+    n_items = int(first[-1])
+    assert first[0] == 0 and n_items <= max_items
+    assert np.all(items[n_items:, 0] == -1)
+    tiles_of = [(n + tile - 1) // tile for n in lens]
+    total = sum(tiles_of)
+    quota = max(1, -(-total // n_workers))
+    g0 = np.concatenate([[0], np.cumsum(tiles_of)])
+    # sequences: consecutive, tile-aligned, complete
+    for b, n in enumerate(lens):
+        at = 0
+        for s, t0, cnt, wk in items[first[b]:first[b + 1]]:
+            assert s == b and t0 == at and cnt > 0 and t0 % tile == 0
+            at += cnt
+        assert at == n
+    # workers: monotone boundaries that cover all items; each item lies inside its worker's range
+    assert wfirst[0] == 0 and wfirst[-1] == n_items and np.all(np.diff(wfirst) >= 0)
+    per_worker = np.zeros(n_workers, dtype=np.int64)
+    for w_id in range(n_workers):
+        for s, t0, cnt, wk in items[wfirst[w_id]:wfirst[w_id + 1]]:
+            assert wk == w_id
+            ga = g0[s] + t0 // tile
+            gb = g0[s] + (t0 + cnt + tile - 1) // tile
+            assert w_id * quota <= ga and gb <= (w_id + 1) * quota
+            per_worker[w_id] += gb - ga
+    assert per_worker.sum() == total
+    want = np.clip(total - quota * np.arange(n_workers), 0, quota)
+    assert np.array_equal(per_worker, want)
 
 
 # ------------------------------------------------------------------ comparator

@@ -133,7 +133,7 @@ def _run(ek, shape, mode, kernel):
     assert rel <= H.REL_L2_TOL and mx <= H.MAX_ABS_TOL, (rel, mx)
     # element by element, relative to the size of the unit's output row
     rows = np.max(np.abs(want), axis=1, keepdims=True)
-    assert np.all(np.abs(got - want) <= 2e-2 * rows + 2e-3), float(np.max(np.abs(got - want) / rows))
+    assert np.all(np.abs(got - want) <= 4e-2 * rows), float(np.max(np.abs(got - want) / rows))
     used, moves = _moves_after_first_tile(ek, st, units)
     if used != 1:
         assert moves > 0, "the inputs did not move the reference maximum after an item's first tile"

@@ -5,23 +5,30 @@ namespace {
 
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
-// Which split-K kernel serves a layer (and cache): 1 = generic CUDA-core kernel, 2 = tcgen05
-// tensor-core kernel, -1 = none.  `cache` may be null (shape-only question).
+// Which split-K kernel serves a layer (and cache): 1 = generic CUDA-core kernel, 2 = two-pass
+// tcgen05 kernel, 3 = resident-tile tcgen05 kernel on block pairs, -1 = none.  `cache` may be
+// null (shape-only question).
 int select_kernel(const elitekv_layer* L, const elitekv_cache* cache) {
   const bool tc = ekv_tc_supported(L, cache) != 0;
+  const bool rt = ekv_rt_supported(L, cache) != 0;
+  if (L->decode_kernel == 3) return rt ? 3 : -1;
   if (L->decode_kernel == 2) return tc ? 2 : -1;
   if (L->decode_kernel == 1) return ekv_generic_supported(L) ? 1 : -1;
+  if (rt) return 3;
   if (tc) return 2;
   return ekv_generic_supported(L) ? 1 : -1;
 }
 
 int max_items_for(const elitekv_layer* L, int B, int kernel) {
+  if (kernel == 3) return ekv_rt_max_items(L, B);
   return kernel == 2 ? ekv_tc_max_items(L, B) : ekv_generic_max_items(L, B);
 }
 
 // Tokens per plan tile and persistent workers (0: the plain plan) of each kernel.
 int plan_tile_for(int kernel) { return kernel == 2 ? 128 : ELITEKV_TILE_TOKENS; }
-int workers_for(const elitekv_layer* L, int kernel) { return kernel == 2 ? ekv_tc_workers(L) : 0; }
+int workers_for(const elitekv_layer* L, int kernel) {
+  return kernel == 3 ? ekv_rt_workers(L) : kernel == 2 ? ekv_tc_workers(L) : 0;
+}
 
 // The workspace is sized for whichever kernel may be picked once the cache layout is known.
 int max_items_any(const elitekv_layer* L, int B) {
@@ -30,6 +37,10 @@ int max_items_any(const elitekv_layer* L, int B) {
   if (ekv_generic_supported(L) && (want == 0 || want == 1)) m = ekv_generic_max_items(L, B);
   if (ekv_tc_supported(L, nullptr) && (want == 0 || want == 2)) {
     const int t = ekv_tc_max_items(L, B);
+    if (t > m) m = t;
+  }
+  if (ekv_rt_supported(L, nullptr) && (want == 0 || want == 3)) {
+    const int t = ekv_rt_max_items(L, B);
     if (t > m) m = t;
   }
   return m;
@@ -138,8 +149,9 @@ extern "C" int elitekv_decode(const elitekv_layer* L, const elitekv_cache* cache
   if (rc != ELITEKV_OK) return rc;
   EkvProfile* prof = (L->prof && L->prof->enabled && L->prof->count < kProfileSlots) ? L->prof : nullptr;
   if (prof) EKV_CUDA_OK(cudaEventRecord(prof->ev[2 * prof->count], st));
-  rc = kernel == 2 ? ekv_launch_decode_tc(L, cache, cv, q_rope, q_abs, B, ws, st)
-                   : ekv_launch_decode_generic(L, cache, cv, q_rope, q_abs, B, ws, st);
+  rc = kernel == 3   ? ekv_launch_decode_rt(L, cache, cv, q_rope, q_abs, B, ws, st)
+       : kernel == 2 ? ekv_launch_decode_tc(L, cache, cv, q_rope, q_abs, B, ws, st)
+                     : ekv_launch_decode_generic(L, cache, cv, q_rope, q_abs, B, ws, st);
   if (rc != ELITEKV_OK) return rc;
   if (prof) {
     EKV_CUDA_OK(cudaEventRecord(prof->ev[2 * prof->count + 1], st));

@@ -182,5 +182,11 @@ int ekv_tc_workers(const elitekv_layer* L);
 int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, const CacheView& cv,
                          const void* q_rope, const void* q_abs, int B, const DecodeScratch& ws,
                          cudaStream_t st);
+int ekv_rt_supported(const elitekv_layer* L, const elitekv_cache* cache);   // cache may be null
+int ekv_rt_workers(const elitekv_layer* L);
+int ekv_rt_max_items(const elitekv_layer* L, int B);
+int ekv_launch_decode_rt(const elitekv_layer* L, const elitekv_cache* cache, const CacheView& cv,
+                         const void* q_rope, const void* q_abs, int B, const DecodeScratch& ws,
+                         cudaStream_t st);
 int ekv_launch_combine(const elitekv_layer* L, int B, const DecodeScratch& ws, void* out,
                        cudaStream_t st);

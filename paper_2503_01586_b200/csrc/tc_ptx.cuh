@@ -1,6 +1,6 @@
 // Inline-PTX wrappers for the sm_100a tensor-core kernels: mbarrier, TMA (cp.async.bulk.tensor),
-// tcgen05 (MMA, commit, TMEM load/store, fences) and shared-memory matrix descriptors.  Every
-// wait helper is bounded.
+// tcgen05 (MMA, commit, TMEM load/store, fences), shared-memory matrix descriptors and the
+// cluster primitives of the block-pair kernel.  Every wait helper is bounded.
 #pragma once
 
 #include <cuda.h>
@@ -264,6 +264,54 @@ __device__ __forceinline__ int f2ord(float f) {
 }
 __device__ __forceinline__ float ord2f(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
 
+
+// ---------------------------------------------------------------- cluster / distributed smem
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in block `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void st_cluster_f4(uint32_t caddr, float4 v) {
+  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(caddr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+// arrive on a barrier of another block of the cluster; orders this thread's earlier
+// distributed-shared-memory stores before it (release at cluster scope)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cbar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cbar) : "memory");
+}
+// probe with acquire at cluster scope: pairs with mbar_arrive_cluster of the peer block
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// mbar_wait_group for a barrier the peer block arrives on: same protocol, with the acquire of
+// every thread taken at cluster scope so that the peer's stores are visible afterwards.
+__device__ __forceinline__ bool mbar_wait_group_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                        volatile int* verdict, unsigned& turn, bool leader, int id,
+                                                        int n, int why, unsigned limit = kSpinLimit) {
+  volatile int* word = verdict + (turn & 1u);
+  ++turn;
+  if (leader) *word = mbar_spin(bar, parity, abort_flag, why, limit) ? 1 : 0;
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory");
+  const bool ok = *word != 0;
+  if (ok) (void)mbar_try_wait_cluster(bar, parity);
+  return ok;
+}
 
 // ---------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,

@@ -61,7 +61,7 @@ def test_config2_7b_75pct_b16_ctx4096(ek):
 def test_config2_all_three_kernels_agree(ek):
     """The CUDA-core kernel and the tcgen05 kernels on the same full-size inputs."""
     outs = []
-    for kernel in (1, 2):
+    for kernel in (1, 2, 3):
         st = H.setup(gen.LLAMA7B_75, decode_kernel=kernel)
         outs.append(H.f64(H.run_decode(st)))
         del st

@@ -270,8 +270,8 @@ def test_back_to_back_steps_share_one_workspace(ek):
     H.check_parity(st, alone1, H.all_units(st))
 
 
-KERNELS = [1, 2]
-KERNEL_IDS = ["generic", "two-pass"]
+KERNELS = [1, 2, 3]
+KERNEL_IDS = ["generic", "two-pass", "resident"]
 TC_KERNELS, TC_KERNEL_IDS = KERNELS[1:], KERNEL_IDS[1:]
 
 

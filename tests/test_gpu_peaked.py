@@ -141,7 +141,7 @@ def _run(ek, shape, mode, kernel):
 
 
 @pytest.mark.parametrize("mode", ["scaled", "planted"])
-@pytest.mark.parametrize("kernel", [1, 2], ids=["generic", "two-pass"])
+@pytest.mark.parametrize("kernel", [1, 2, 3], ids=["generic", "two-pass", "resident"])
 def test_peaked_7b_shape_each_kernel(ek, mode, kernel):
     assert _run(ek, "7b", mode, kernel) == kernel
 

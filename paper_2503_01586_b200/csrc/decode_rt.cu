@@ -30,11 +30,17 @@
 // A cluster is a persistent worker walking its items of the balanced plan (64-token tiles); per
 // item each block writes its half of (acc) and block 0 writes (m, l).
 //
-// Roles per block (352 threads):
-//   warps 0, 6   TMA producers (units dealt alternately); warp 0 also loads the query half
-//   warp 1       TMEM owner and MMA issuer (warp-uniform, instruction under an elected lane)
-//   warps 2-5    mixing of the partial scores, exchange, softmax, rescale, epilogue
-//   warps 7-10   rope dot products: a warp reads whole rope rows with 16-byte loads per lane
+// Roles per block (384 threads = three warpgroups, each with its own register budget):
+//   warps 0, 2   TMA producers (units dealt alternately); warp 0 also loads the query half
+//   warp 1       TMEM owner and MMA issuer (warp-uniform, instruction under an elected lane;
+//                slot and phase counters advance incrementally so that the descriptor words
+//                stay in uniform registers)
+//   warp 3       idle
+//   warps 4-7    mixing of the partial scores, exchange, softmax, rescale, epilogue
+//   warps 8-11   rope dot products: a warp reads whole rope rows with 16-byte loads per lane
+// Warpgroup 0 gives registers back right away (setmaxnreg), the other two take them: the
+// softmax and rope code would otherwise spill, and with nearly all of L1 carved out as shared
+// memory a spill is an L2 round trip.
 // Every wait is bounded; on a timeout the block records ELITEKV_ERR_TIMEOUT, stops issuing work
 // and leaves through the common exit (its peer then runs into its own limit).
 #include "tc_ptx.cuh"
@@ -44,9 +50,11 @@ namespace {
 constexpr int kT = 64;                 // tokens per tile
 constexpr int kUnit = 16384;           // ring unit: [2 chunks][64 tokens][64 bf16]
 constexpr int kMaxRing = 9;
-constexpr int kRtThreads = 352;
-constexpr int kSm = 128;               // softmax threads (warps 2-5)
-constexpr int kRopeWarps = 4;          // warps 7-10
+constexpr int kRtThreads = 384;
+constexpr int kSm = 128;               // softmax threads (warps 4-7)
+constexpr int kRopeWarps = 4;          // warps 8-11
+// register budgets per warpgroup after the split: 128 * (96 + 224 + 184) = 384 * 168, the launch total
+constexpr int kRegsIssue = 96, kRegsSoftmax = 224, kRegsRope = 184;
 constexpr int kHeads = 32;
 
 struct RtArgs {
@@ -91,6 +99,29 @@ __host__ __device__ inline RtSmem rt_layout(int d_c, int n_ring) {
 }
 
 __device__ __forceinline__ float4 ld_f4(const float* p) { return *(const float4*)p; }
+
+#ifndef RT_WAIT_MODE
+#define RT_WAIT_MODE 1
+#endif
+// Warp-level wait used by the roles that wait long (producers for a free unit, rope warps for
+// the hand-over buffer, the MMA warp for P): the probe is mbarrier.try_wait, which parks the
+// warp in hardware for a while instead of spinning, so a waiting warp does not take issue
+// slots and shared-memory cycles from the warp of its scheduler that is doing the work.
+__device__ __forceinline__ bool rt_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int why) {
+#if RT_WAIT_MODE == 0
+  return warp_wait(bar, parity, abort_flag, why);
+#else
+  for (unsigned i = 0; i < kWaitLimit; ++i) {
+    if (__any_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+#if RT_WAIT_MODE == 2
+    asm volatile("nanosleep.u32 64;" ::: "memory");
+#endif
+    if ((i & 255) == 255 && __any_sync(0xffffffffu, *abort_flag != 0)) return false;
+  }
+  if (*abort_flag == 0) *abort_flag = why;
+  return false;
+#endif
+}
 
 template <int R2>
 __global__ void __launch_bounds__(kRtThreads, 1)
@@ -163,58 +194,68 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   ekv_pdl_trigger();
   const int item_lo = a.worker_first[worker], item_hi = a.worker_first[worker + 1];
 
-  unsigned gt_base = 0;                  // tiles of this worker before the current item
-  unsigned gw_turn = 0;                  // group waits taken so far by the softmax threads
+  // first cache row of a tile (tiles start on multiples of 64 tokens and pages hold a multiple
+  // of 64 tokens, so a tile never straddles pages)
+  auto tile_row = [&](int seq, int t_abs, bool report) -> long long {
+    if (a.page_table == nullptr) return (long long)seq * a.max_ctx + t_abs;
+    const int pi = t_abs >> a.page_shift;
+    int page = pi < a.max_pages_per_seq ? a.page_table[(long long)seq * a.max_pages_per_seq + pi] : -1;
+    if (page < 0 || page >= a.num_pages) {
+      if (report) ekv_record(a.status, ELITEKV_ERR_BAD_PAGE, seq, page);
+      page = 0;
+    }
+    return ((long long)page << a.page_shift) + (t_abs & a.page_mask);
+  };
+  // end of an item: every role is done with the queries, the P tile, the ring and the output
+  // columns.  All 384 threads meet here from their own loops; false = the block is aborting
+  // (same answer in every thread: nobody is inside a wait at this point).
+  auto item_end = [&]() -> bool {
+    tc_fence_before();
+    named_bar_sync(3, kRtThreads);
+    tc_fence_after();
+    return *s_abort == 0;
+  };
   int seq = -1;
-  for (int item = item_lo; item < item_hi; ++item) {
-    seq = a.items[4 * item + 0];
-    const int tok0 = a.items[4 * item + 1];
-    const int ntok = a.items[4 * item + 2];
-    const int n_tiles = (ntok + kT - 1) / kT;
-    const unsigned item_n = (unsigned)(item - item_lo);
 
-    // first cache row of a tile (tiles start on multiples of 64 tokens and pages hold a multiple
-    // of 64 tokens, so a tile never straddles pages)
-    auto tile_row = [&](int tile, bool report) -> long long {
-      const int t_abs = tok0 + tile * kT;
-      if (a.page_table == nullptr) return (long long)seq * a.max_ctx + t_abs;
-      const int pi = t_abs >> a.page_shift;
-      int page = pi < a.max_pages_per_seq ? a.page_table[(long long)seq * a.max_pages_per_seq + pi] : -1;
-      if (page < 0 || page >= a.num_pages) {
-        if (report) ekv_record(a.status, ELITEKV_ERR_BAD_PAGE, seq, page);
-        page = 0;
-      }
-      return ((long long)page << a.page_shift) + (t_abs & a.page_mask);
-    };
-    // ============================================================ warps 0, 6: TMA producers
-    if (warp == 0 || warp == 6) {
-      const int prod = warp == 0 ? 0 : 1;
+  if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIssue));
+    // ============================================================ warps 0, 2: TMA producers
+    if (warp == 0 || warp == 2) {
+      const int prod = warp >> 1;
       const uint64_t pol_drop = make_l2_policy_evict_first(), pol_keep = make_l2_policy_evict_last();
-      if (prod == 0 && elect_one()) {
-        // this block's half of the sequence's absorbed queries: stays for the whole item
-        const uint32_t qb = smem_u32(&bars->q_full);
-        mbar_expect_tx(qb, (uint32_t)(2 * NU * N * 128));
-        for (int kc = 0; kc < 2 * NU; ++kc)
-          tma_load_2d_hint(smem_u32(s_q + kc * N * 128), &map_q, (int)rank * DH + kc * 64, seq * N, qb, pol_keep);
-      }
-      __syncwarp();
-      bool ok = true;
-      for (int tile = 0; tile < n_tiles && ok; ++tile) {
-        const int row = (int)tile_row(tile, prod == 0 && lane == 0);
-        const unsigned n0 = (gt_base + (unsigned)tile) * (unsigned)NU;
-        for (int u = prod; u < NU; u += 2) {
-          const unsigned n = n0 + (unsigned)u, slot = n % (unsigned)NR;
-          ok = warp_wait(smem_u32(&bars->empty[slot]), ((n / (unsigned)NR) & 1) ^ 1, s_abort, 1);
-          if (!ok) break;
-          if (elect_one()) {
-            const uint32_t fb = smem_u32(&bars->full[slot]);
-            mbar_expect_tx(fb, (uint32_t)kUnit);
-            const uint32_t dst = smem_u32(s_ring + slot * kUnit);
-            tma_load_2d_hint(dst, &map_lat, (int)rank * DH + (2 * u) * 64, row, fb, pol_drop);
-            tma_load_2d_hint(dst + 8192, &map_lat, (int)rank * DH + (2 * u + 1) * 64, row, fb, pol_drop);
-          }
-          __syncwarp();
+      unsigned slot = 0, par = 0;          // ring position of the next unit and its phase parity
+      for (int item = item_lo; item < item_hi; ++item) {
+        seq = a.items[4 * item + 0];
+        const int tok0 = a.items[4 * item + 1];
+        const int n_tiles = (a.items[4 * item + 2] + kT - 1) / kT;
+        if (prod == 0 && elect_one()) {
+          // this block's half of the sequence's absorbed queries: stays for the whole item
+          const uint32_t qb = smem_u32(&bars->q_full);
+          mbar_expect_tx(qb, (uint32_t)(2 * NU * N * 128));
+          for (int kc = 0; kc < 2 * NU; ++kc)
+            tma_load_2d_hint(smem_u32(s_q + kc * N * 128), &map_q, (int)rank * DH + kc * 64, seq * N, qb, pol_keep);
         }
+        __syncwarp();
+        bool ok = true;
+        for (int tile = 0; tile < n_tiles && ok; ++tile) {
+          const int row = (int)tile_row(seq, tok0 + tile * kT, prod == 0 && lane == 0);
+          for (int u = 0; u < NU; ++u) {
+            if ((u & 1) == prod) {
+              ok = rt_wait(smem_u32(&bars->empty[slot]), par ^ 1, s_abort, 1);
+              if (!ok) break;
+              if (elect_one()) {
+                const uint32_t fb = smem_u32(&bars->full[slot]);
+                mbar_expect_tx(fb, (uint32_t)kUnit);
+                const uint32_t dst = smem_u32(s_ring + slot * kUnit);
+                tma_load_2d_hint(dst, &map_lat, (int)rank * DH + (2 * u) * 64, row, fb, pol_drop);
+                tma_load_2d_hint(dst + 8192, &map_lat, (int)rank * DH + (2 * u + 1) * 64, row, fb, pol_drop);
+              }
+              __syncwarp();
+            }
+            if (++slot == (unsigned)NR) { slot = 0; par ^= 1; }
+          }
+        }
+        if (!item_end()) break;
       }
     }
     // ============================================================ warp 1: MMA issuer
@@ -229,168 +270,114 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       const uint32_t ring16 = (smem_u32(s_ring) >> 4) & 0x3FFFu, q16 = (smem_u32(s_q) >> 4) & 0x3FFFu;
       const uint32_t lo_p = desc_lo(smem_u32(s_p), 128);
       const uint32_t full0 = smem_u32(&bars->full[0]), empty0 = smem_u32(&bars->empty[0]);
-      bool ok = warp_wait(smem_u32(&bars->q_full), item_n & 1, s_abort, 2);
-      for (int tile = 0; tile < n_tiles && ok; ++tile) {
-        const unsigned gt = gt_base + (unsigned)tile;
-        const unsigned n0 = gt * (unsigned)NU;
-        const int nvalid = min(kT, ntok - tile * kT);
-        const int ksteps = (nvalid + 15) >> 4;
-        // ---- partial scores: one unit (two chunks) per 4 MMAs
-        for (int u = 0; u < NU; ++u) {
-          const unsigned n = n0 + (unsigned)u, slot = n % (unsigned)NR;
-          ok = warp_wait(full0 + slot * 8, (n / (unsigned)NR) & 1, s_abort, 3);
-          if (!ok) break;
-          const uint32_t la = (ring16 + slot * (kUnit >> 4)) | (1u << 16);
-          const uint32_t lb = (q16 + (uint32_t)u * 512u) | (1u << 16);
-          if (elect_one()) {
-            tc_mma_w(tmem_s, la, hi_sw, lb, hi_sw, idesc_s, u != 0);
-            tc_mma_w(tmem_s, la + 2, hi_sw, lb + 2, hi_sw, idesc_s, 1);     // +32 bytes along K per step
-            tc_mma_w(tmem_s, la + 4, hi_sw, lb + 4, hi_sw, idesc_s, 1);
-            tc_mma_w(tmem_s, la + 6, hi_sw, lb + 6, hi_sw, idesc_s, 1);
-          }
-          __syncwarp();
-        }
-        if (!ok) break;
-        if (elect_one()) tc_commit(smem_u32(&bars->s_full));
-        __syncwarp();
-        // ---- wait for P (and the rescaled output) of this tile
-        ok = warp_wait(smem_u32(&bars->p_ready), gt & 1, s_abort, 4);
-        if (!ok) break;
-        tc_fence_after();
-        // ---- value product: unit u = output block u (two 64-coordinate atoms 8 KB apart)
-        for (int u = 0; u < NU; ++u) {
-          const unsigned n = n0 + (unsigned)u, slot = n % (unsigned)NR;
-          if (ksteps * 16 > nvalid) {
-            // ragged end of a sequence: rows past its last token inside the last 16-token step
-            // become exact zeros so that zero-probability rows cannot inject NaN/Inf bit patterns
-            unsigned char* unit = s_ring + slot * kUnit;
-            for (int e = lane; e < (ksteps * 16 - nvalid) * 16; e += 32) {
-              const int rrow = nvalid + (e >> 4), c16 = e & 15;
-              *(uint4*)(unit + (c16 >> 3) * 8192 + rrow * 128 + (c16 & 7) * 16) = make_uint4(0, 0, 0, 0);
+      unsigned slot = 0, par = 0;          // ring position of the next tile's first unit
+      unsigned tiles_done = 0;
+      for (int item = item_lo; item < item_hi; ++item) {
+        seq = a.items[4 * item + 0];
+        const int ntok = a.items[4 * item + 2];
+        const int n_tiles = (ntok + kT - 1) / kT;
+        bool ok = rt_wait(smem_u32(&bars->q_full), (unsigned)(item - item_lo) & 1, s_abort, 2);
+        for (int tile = 0; tile < n_tiles && ok; ++tile) {
+          const int nvalid = min(kT, ntok - tile * kT);
+          const int ksteps = (nvalid + 15) >> 4;
+          // ---- partial scores: one unit (two chunks) per 4 MMAs
+          unsigned sa = slot, pa = par;
+          uint32_t lb = q16 | (1u << 16);
+          for (int u = 0; u < NU; ++u) {
+            ok = rt_wait(full0 + sa * 8, pa, s_abort, 3);
+            if (!ok) break;
+            const uint32_t la = (ring16 + sa * (kUnit >> 4)) | (1u << 16);
+            if (elect_one()) {
+              tc_mma_w(tmem_s, la, hi_sw, lb, hi_sw, idesc_s, u != 0);
+              tc_mma_w(tmem_s, la + 2, hi_sw, lb + 2, hi_sw, idesc_s, 1);     // +32 bytes along K per step
+              tc_mma_w(tmem_s, la + 4, hi_sw, lb + 4, hi_sw, idesc_s, 1);
+              tc_mma_w(tmem_s, la + 6, hi_sw, lb + 6, hi_sw, idesc_s, 1);
             }
-            fence_proxy_async();
             __syncwarp();
+            lb += 512u;                                                       // next pair of query chunks
+            if (++sa == (unsigned)NR) { sa = 0; pa ^= 1; }
           }
-          const uint32_t la = (ring16 + slot * (kUnit >> 4)) | (512u << 16);
-          const uint32_t d = tmem_base + (uint32_t)u * N;
-          if (elect_one()) {
-            if (ksteps == 4) {
-              tc_mma_w(d, la, hi_sw, lo_p, hi_p, idesc_pv, tile != 0);
-              tc_mma_w(d, la + 128, hi_sw, lo_p + 16, hi_p, idesc_pv, 1);   // +16 tokens: 2048 bytes in A, 256 in P
-              tc_mma_w(d, la + 256, hi_sw, lo_p + 32, hi_p, idesc_pv, 1);
-              tc_mma_w(d, la + 384, hi_sw, lo_p + 48, hi_p, idesc_pv, 1);
-            } else {
-              for (int k = 0; k < ksteps; ++k)
-                tc_mma_w(d, la + 128 * k, hi_sw, lo_p + 16 * k, hi_p, idesc_pv, (tile | k) != 0);
-            }
-            tc_commit(empty0 + slot * 8);
-          }
+          if (!ok) break;
+          if (elect_one()) tc_commit(smem_u32(&bars->s_full));
           __syncwarp();
+          // ---- wait for P (and the rescaled output) of this tile
+          ok = rt_wait(smem_u32(&bars->p_ready), tiles_done & 1, s_abort, 4);
+          if (!ok) break;
+          tc_fence_after();
+          // ---- value product: unit u = output block u (two 64-coordinate atoms 8 KB apart)
+          unsigned sb = slot;
+          for (int u = 0; u < NU; ++u) {
+            if (ksteps * 16 > nvalid) {
+              // ragged end of a sequence: rows past its last token inside the last 16-token step
+              // become exact zeros so that zero-probability rows cannot inject NaN/Inf bit patterns
+              unsigned char* unit = s_ring + sb * kUnit;
+              for (int e = lane; e < (ksteps * 16 - nvalid) * 16; e += 32) {
+                const int rrow = nvalid + (e >> 4), c16 = e & 15;
+                *(uint4*)(unit + (c16 >> 3) * 8192 + rrow * 128 + (c16 & 7) * 16) = make_uint4(0, 0, 0, 0);
+              }
+              fence_proxy_async();
+              __syncwarp();
+            }
+            const uint32_t la = (ring16 + sb * (kUnit >> 4)) | (512u << 16);
+            const uint32_t d = tmem_base + (uint32_t)u * N;
+            if (elect_one()) {
+              if (ksteps == 4) {
+                tc_mma_w(d, la, hi_sw, lo_p, hi_p, idesc_pv, tile != 0);
+                tc_mma_w(d, la + 128, hi_sw, lo_p + 16, hi_p, idesc_pv, 1);   // +16 tokens: 2048 bytes in A, 256 in P
+                tc_mma_w(d, la + 256, hi_sw, lo_p + 32, hi_p, idesc_pv, 1);
+                tc_mma_w(d, la + 384, hi_sw, lo_p + 48, hi_p, idesc_pv, 1);
+              } else {
+                for (int k = 0; k < ksteps; ++k)
+                  tc_mma_w(d, la + 128 * k, hi_sw, lo_p + 16 * k, hi_p, idesc_pv, (tile | k) != 0);
+              }
+              tc_commit(empty0 + sb * 8);
+            }
+            __syncwarp();
+            if (++sb == (unsigned)NR) sb = 0;
+          }
+          if (elect_one()) tc_commit(smem_u32(&bars->pv_done));
+          __syncwarp();
+          slot = sa;
+          par = pa;
+          ++tiles_done;
         }
-        if (elect_one()) tc_commit(smem_u32(&bars->pv_done));
-        __syncwarp();
+        if (!item_end()) break;
       }
     }
-    // ============================================================ warps 7-10: rope dot products
-    // The block adds the rope part for tokens [32 rank, 32 rank + 32) of every tile.  A warp
-    // takes 8 of them; a rope row is 32 heads x R2 bf16 = 4 R2 pieces of 16 bytes, lane L of
-    // load i reads piece 32 i + L (one coalesced 512-byte request per load), which belongs to
-    // head 8 (32 i + L) / R2.  The products wait in registers until the softmax threads have
-    // released the hand-over buffer, then the per-head sums go to s_xmix[token][head].
-    else if (warp >= 7) {
-      const int rw = warp - 7;
-      float qr[LPT][8];
-#pragma unroll
-      for (int i = 0; i < LPT; ++i) {
-        const int e0 = 8 * (32 * i + lane);          // first element of the piece inside the row
-        const bf16* src = a.q_rope + (size_t)seq * N * R2 + e0;
-        const uint4 v = *(const uint4*)src;
-        const bf162* p2 = (const bf162*)&v;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const float2 f = __bfloat1622float2(p2[j]);
-          qr[i][2 * j] = f.x;
-          qr[i][2 * j + 1] = f.y;
-        }
-      }
-      bool ok = true;
-      const size_t row_elems = (size_t)N * R2;
-      for (int tile = 0; tile < n_tiles && ok; ++tile) {
-        const unsigned gt = gt_base + (unsigned)tile;
-        const int nvalid = min(kT, ntok - tile * kT);
-        const long long row0 = tile_row(tile, false);
-        float part[8][LPT];
-#pragma unroll
-        for (int tt = 0; tt < 8; ++tt) {
-          const int t = 32 * (int)rank + 8 * rw + tt;
-          uint4 v[LPT];
-#pragma unroll
-          for (int i = 0; i < LPT; ++i) {
-            v[i] = make_uint4(0, 0, 0, 0);
-            if (t < nvalid)
-              v[i] = __ldcs((const uint4*)(a.rope_plane + (size_t)(row0 + t) * row_elems) + 32 * i + lane);
-          }
-#pragma unroll
-          for (int i = 0; i < LPT; ++i) {
-            const bf162* k2 = (const bf162*)&v[i];
-            float acc = 0.f;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const float2 f = __bfloat1622float2(k2[j]);
-              acc = fmaf(qr[i][2 * j], f.x, acc);
-              acc = fmaf(qr[i][2 * j + 1], f.y, acc);
-            }
-            part[tt][i] = acc;
-          }
-        }
-        // sum over the LPT adjacent lanes that share a head
-#pragma unroll
-        for (int tt = 0; tt < 8; ++tt)
-#pragma unroll
-          for (int i = 0; i < LPT; ++i) {
-            float s = part[tt][i];
-            if (LPT >= 2) s += __shfl_xor_sync(0xffffffffu, s, 1);
-            if (LPT >= 4) s += __shfl_xor_sync(0xffffffffu, s, 2);
-            part[tt][i] = s;
-          }
-        // the softmax threads are done with the previous tile's hand-over
-        ok = warp_wait(smem_u32(&bars->rope_free), (gt & 1) ^ 1, s_abort, 5);
-        if (!ok) break;
-        if ((lane & (LPT - 1)) == 0) {
-#pragma unroll
-          for (int tt = 0; tt < 8; ++tt) {
-            const int t = 32 * (int)rank + 8 * rw + tt;
-#pragma unroll
-            for (int i = 0; i < LPT; ++i) {
-              const int h = (8 * (32 * i + lane)) / R2;
-              s_xmix[t * N + ((((h >> 2) + t) & 7) << 2) + (h & 3)] = part[tt][i];
-            }
-          }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bars->rope_ready));
-      }
+    // warp 3 has no work; it only keeps the item barrier's head count
+    else {
+      for (int item = item_lo; item < item_hi; ++item)
+        if (!item_end()) break;
     }
-    // ============================================================ warps 2-5: scores -> P, rescale, epilogue
+  }
+  else if (warp < 8) {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
+    // ============================================================ warps 4-7: scores -> P, rescale, epilogue
     // Thread (quarter, lane) may touch TMEM lanes 32 quarter + lane.  Quarters 0, 1 hold the
     // even-chunk diagonal block (accumulator rows = tokens 0-63, columns 0-31), quarters 2, 3 the
     // odd-chunk block (rows 64-127 = tokens 0-63 again, columns 32-63).  The two threads of a
     // token split the heads: the even-side thread finishes heads 0-15, the odd-side thread heads
     // 16-31, each handing the other 16 values to its partner through s_xmix.
-    else {
-      const int sid = threadIdx.x - 64;
+    {
+      const int sid = threadIdx.x - 128;
+      unsigned gt_base = 0;              // tiles of this worker before the current item
+      unsigned gw_turn = 0;              // group waits taken so far
       const int quarter = warp & 3;
       const int hh = quarter >> 1;                       // head half this thread finishes
       const int t = (quarter & 1) * 32 + lane;           // token row inside the tile
       const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
       const bool leader = sid == 0;
       const bool own_tok = (uint32_t)(t >> 5) == rank;   // this block added the rope part of the token
+      float* xrow = s_xmix + t * N;
+      for (int item = item_lo; item < item_hi; ++item) {
+      seq = a.items[4 * item + 0];
+      const int ntok = a.items[4 * item + 2];
+      const int n_tiles = (ntok + kT - 1) / kT;
       float l_part[16];
 #pragma unroll
       for (int i = 0; i < 16; ++i) l_part[i] = 0.f;
       float m_ref = -INFINITY;                           // lane h: reference maximum of head h (all 32, in every warp)
       bool ok = true;
-      float* xrow = s_xmix + t * N;
       for (int tile = 0; tile < n_tiles && ok; ++tile) {
         const unsigned gt = gt_base + (unsigned)tile, par = gt & 1, k2 = gt >> 1;
         const int nvalid = min(kT, ntok - tile * kT);
@@ -559,12 +546,100 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         }
         if (leader) bulk_wait_group_all();     // stores done before the ring is reused or the block leaves
       }
+      gt_base += (unsigned)n_tiles;
+      if (!item_end()) break;
+      }
     }
-    gt_base += (unsigned)n_tiles;
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    if (*s_abort) break;      // same value in every thread: nobody is inside a wait here
+  }
+  else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsRope));
+    // ============================================================ warps 8-11: rope dot products
+    // The block adds the rope part for tokens [32 rank, 32 rank + 32) of every tile.  A warp
+    // takes 8 of them; a rope row is 32 heads x R2 bf16 = 4 R2 pieces of 16 bytes, lane L of
+    // load i reads piece 32 i + L (one coalesced 512-byte request per load), which belongs to
+    // head 8 (32 i + L) / R2.  The products wait in registers until the softmax threads have
+    // released the hand-over buffer, then the per-head sums go to s_xmix[token][head].
+    {
+      const int rw = warp - 8;
+      unsigned gt = 0;                   // tiles of this worker so far
+      for (int item = item_lo; item < item_hi; ++item) {
+      seq = a.items[4 * item + 0];
+      const int tok0 = a.items[4 * item + 1];
+      const int ntok = a.items[4 * item + 2];
+      const int n_tiles = (ntok + kT - 1) / kT;
+      float qr[LPT][8];
+#pragma unroll
+      for (int i = 0; i < LPT; ++i) {
+        const int e0 = 8 * (32 * i + lane);          // first element of the piece inside the row
+        const bf16* src = a.q_rope + (size_t)seq * N * R2 + e0;
+        const uint4 v = *(const uint4*)src;
+        const bf162* p2 = (const bf162*)&v;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float2 f = __bfloat1622float2(p2[j]);
+          qr[i][2 * j] = f.x;
+          qr[i][2 * j + 1] = f.y;
+        }
+      }
+      bool ok = true;
+      const size_t row_elems = (size_t)N * R2;
+      for (int tile = 0; tile < n_tiles && ok; ++tile, ++gt) {
+        const int nvalid = min(kT, ntok - tile * kT);
+        const long long row0 = tile_row(seq, tok0 + tile * kT, false);
+        float part[8][LPT];
+#pragma unroll
+        for (int tt = 0; tt < 8; ++tt) {
+          const int t = 32 * (int)rank + 8 * rw + tt;
+          uint4 v[LPT];
+#pragma unroll
+          for (int i = 0; i < LPT; ++i) {
+            v[i] = make_uint4(0, 0, 0, 0);
+            if (t < nvalid)
+              v[i] = __ldcs((const uint4*)(a.rope_plane + (size_t)(row0 + t) * row_elems) + 32 * i + lane);
+          }
+#pragma unroll
+          for (int i = 0; i < LPT; ++i) {
+            const bf162* k2 = (const bf162*)&v[i];
+            float acc = 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const float2 f = __bfloat1622float2(k2[j]);
+              acc = fmaf(qr[i][2 * j], f.x, acc);
+              acc = fmaf(qr[i][2 * j + 1], f.y, acc);
+            }
+            part[tt][i] = acc;
+          }
+        }
+        // sum over the LPT adjacent lanes that share a head
+#pragma unroll
+        for (int tt = 0; tt < 8; ++tt)
+#pragma unroll
+          for (int i = 0; i < LPT; ++i) {
+            float s = part[tt][i];
+            if (LPT >= 2) s += __shfl_xor_sync(0xffffffffu, s, 1);
+            if (LPT >= 4) s += __shfl_xor_sync(0xffffffffu, s, 2);
+            part[tt][i] = s;
+          }
+        // the softmax threads are done with the previous tile's hand-over
+        ok = rt_wait(smem_u32(&bars->rope_free), (gt & 1) ^ 1, s_abort, 5);
+        if (!ok) break;
+        if ((lane & (LPT - 1)) == 0) {
+#pragma unroll
+          for (int tt = 0; tt < 8; ++tt) {
+            const int t = 32 * (int)rank + 8 * rw + tt;
+#pragma unroll
+            for (int i = 0; i < LPT; ++i) {
+              const int h = (8 * (32 * i + lane)) / R2;
+              s_xmix[t * N + ((((h >> 2) + t) & 7) << 2) + (h & 3)] = part[tt][i];
+            }
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars->rope_ready));
+      }
+      if (!item_end()) break;
+      }
+    }
   }
 
   // ============================================================== teardown

@@ -75,7 +75,7 @@ struct RtArgs {
 
 struct __align__(8) RtBarriers {
   uint64_t full[kMaxRing], empty[kMaxRing];
-  uint64_t q_full, s_full, p_ready, pv_done, rope_ready, rope_free;
+  uint64_t q_full, s_full, p_ready, pv_done, rope_ready, recv_done;
   uint64_t x_full[2], x_free[2];
 };
 
@@ -107,12 +107,13 @@ __device__ __forceinline__ float4 ld_f4(const float* p) { return *(const float4*
 // the hand-over buffer, the MMA warp for P): the probe is mbarrier.try_wait, which parks the
 // warp in hardware for a while instead of spinning, so a waiting warp does not take issue
 // slots and shared-memory cycles from the warp of its scheduler that is doing the work.
+template <bool kClusterAcquire = false>
 __device__ __forceinline__ bool rt_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int why) {
 #if RT_WAIT_MODE == 0
   return warp_wait(bar, parity, abort_flag, why);
 #else
   for (unsigned i = 0; i < kWaitLimit; ++i) {
-    if (__any_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+    if (__any_sync(0xffffffffu, kClusterAcquire ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity))) return true;
 #if RT_WAIT_MODE == 2
     asm volatile("nanosleep.u32 64;" ::: "memory");
 #endif
@@ -168,9 +169,9 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
     mbar_init(smem_u32(&bars->p_ready), kSm);
     mbar_init(smem_u32(&bars->pv_done), 1);
     mbar_init(smem_u32(&bars->rope_ready), kRopeWarps);
-    mbar_init(smem_u32(&bars->rope_free), kSm);
+    mbar_init(smem_u32(&bars->recv_done), kSm);
     for (int i = 0; i < 2; ++i) {
-      mbar_init(smem_u32(&bars->x_full[i]), kSm);     // one arrival per softmax thread of the peer
+      mbar_init(smem_u32(&bars->x_full[i]), 1);       // armed per tile; completed by the peer's bulk copy
       mbar_init(smem_u32(&bars->x_free[i]), 1);
     }
     *s_abort = 0;
@@ -344,10 +345,23 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         if (!item_end()) break;
       }
     }
-    // warp 3 has no work; it only keeps the item barrier's head count
+    // ============================================================ warp 3: hand-back of the receive buffer
+    // Tells the peer that this block has consumed the partial scores the peer sent for a tile
+    // (so the peer may reuse that receive buffer and its own send buffer), off the softmax
+    // threads' critical path: a remote arrive with release semantics takes a round trip.
     else {
-      for (int item = item_lo; item < item_hi; ++item)
+      unsigned gt = 0;
+      for (int item = item_lo; item < item_hi; ++item) {
+        const int n_tiles = (a.items[4 * item + 2] + kT - 1) / kT;
+        bool ok = true;
+        for (int tile = 0; tile < n_tiles && ok; ++tile, ++gt) {
+          ok = rt_wait(smem_u32(&bars->recv_done), gt & 1, s_abort, 11);
+          if (!ok) break;
+          if (elect_one()) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->x_free[gt & 1]), peer));
+          __syncwarp();
+        }
         if (!item_end()) break;
+      }
     }
   }
   else if (warp < 8) {
@@ -378,20 +392,22 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       for (int i = 0; i < 16; ++i) l_part[i] = 0.f;
       float m_ref = -INFINITY;                           // lane h: reference maximum of head h (all 32, in every warp)
       bool ok = true;
-      for (int tile = 0; tile < n_tiles && ok; ++tile) {
+      for (int tile = 0; tile < n_tiles; ++tile) {
         const unsigned gt = gt_base + (unsigned)tile, par = gt & 1, k2 = gt >> 1;
         const int nvalid = min(kT, ntok - tile * kT);
+        // Waits inside a tile are per thread (try_wait parks the thread between probes).  A
+        // thread whose wait gives up goes on to the tile's named barriers all the same; behind
+        // the last of them the leader's view of the abort flag decides for the whole group.
         // ---- this thread's diagonal block row out of TMEM
-        ok = mbar_wait_group(smem_u32(&bars->s_full), gt & 1, s_abort, s_verdict, gw_turn, leader, 2, kSm, 6);
-        if (!ok) break;
+        (void)mbar_wait(smem_u32(&bars->s_full), gt & 1, s_abort, 6);
         tc_fence_after();
         float mine[16], other[16];                       // heads 16 hh .. + 15, and the partner's 16
         tc_ld16(tmem_s + lane_base + (uint32_t)(hh * 32 + hh * 16), mine);
         tc_ld16(tmem_s + lane_base + (uint32_t)(hh * 32 + (1 - hh) * 16), other);
         tc_wait_ld();
+        if (leader) mbar_expect_tx(smem_u32(&bars->x_full[par]), (uint32_t)(kT * N * 4));   // the peer's rows of this tile
         // ---- hand the partner its 16 heads (on top of the rope part where this block owns it)
-        ok = mbar_wait_group(smem_u32(&bars->rope_ready), gt & 1, s_abort, s_verdict, gw_turn, leader, 2, kSm, 7);
-        if (!ok) break;
+        (void)mbar_wait(smem_u32(&bars->rope_ready), gt & 1, s_abort, 7);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int c = 4 * (1 - hh) + j;                // logical 16-byte chunk = heads 4c .. 4c+3
@@ -404,33 +420,31 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
           *(float4*)px = v;
         }
         named_bar_sync(1, kSm);
+        // ---- this block's sum for the thread's 16 heads, kept and put back in place: the buffer
+        //      then holds the block's whole [64 x 32] contribution, which one bulk copy takes to
+        //      the peer
         float s[16];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int c = 4 * hh + j;
-          const float4 x = ld_f4(xrow + (((c + t) & 7) << 2));
+          float* px = xrow + (((c + t) & 7) << 2);
+          const float4 x = ld_f4(px);
           s[4 * j] = mine[4 * j] + x.x;
           s[4 * j + 1] = mine[4 * j + 1] + x.y;
           s[4 * j + 2] = mine[4 * j + 2] + x.z;
           s[4 * j + 3] = mine[4 * j + 3] + x.w;
+          *(float4*)px = make_float4(s[4 * j], s[4 * j + 1], s[4 * j + 2], s[4 * j + 3]);
         }
-        mbar_arrive(smem_u32(&bars->rope_free));
-        // ---- exchange with the peer block: its buffer of this parity was consumed two tiles ago
-        if (k2 > 0) {
-          ok = mbar_wait_group_cluster(smem_u32(&bars->x_free[par]), (k2 - 1) & 1, s_abort, s_verdict, gw_turn, leader, 2, kSm, 8);
-          if (!ok) break;
+        fence_proxy_async();
+        named_bar_sync(1, kSm);
+        if (leader) {
+          // the peer's receive buffer of this parity was handed back two tiles ago
+          const bool free_ok = k2 == 0 || mbar_wait_cluster(smem_u32(&bars->x_free[par]), (k2 - 1) & 1, s_abort, 8);
+          if (free_ok)
+            bulk_copy_to_peer(map_to_cta(smem_u32(s_recv + par * kT * N), peer), smem_u32(s_xmix), (uint32_t)(kT * N * 4),
+                              map_to_cta(smem_u32(&bars->x_full[par]), peer));
         }
-        {
-          const uint32_t remote = map_to_cta(smem_u32(s_recv + (par * kT + t) * N), peer);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int c = 4 * hh + j;
-            st_cluster_f4(remote + ((uint32_t)((c + t) & 7) << 4), make_float4(s[4 * j], s[4 * j + 1], s[4 * j + 2], s[4 * j + 3]));
-          }
-          mbar_arrive_cluster(map_to_cta(smem_u32(&bars->x_full[par]), peer));
-        }
-        ok = mbar_wait_group_cluster(smem_u32(&bars->x_full[par]), k2 & 1, s_abort, s_verdict, gw_turn, leader, 2, kSm, 9);
-        if (!ok) break;
+        (void)mbar_wait(smem_u32(&bars->x_full[par]), k2 & 1, s_abort, 9);
         {
           const float* rrow = s_recv + (par * kT + t) * N;
 #pragma unroll
@@ -440,6 +454,7 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
             s[4 * j] += x.x; s[4 * j + 1] += x.y; s[4 * j + 2] += x.z; s[4 * j + 3] += x.w;
           }
         }
+        mbar_arrive(smem_u32(&bars->recv_done));         // warp 3 hands the buffer back to the peer
         const bool live = t < nvalid;
 #pragma unroll
         for (int i = 0; i < 16; ++i) s[i] = live ? s[i] * a.scale_log2e : -INFINITY;
@@ -451,9 +466,12 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
           if (lane == i) wm = v;
         }
         if (lane < 16) s_wmax[quarter * 16 + lane] = wm;
+        if (leader) s_verdict[0] = *s_abort;             // every wait of this tile lies behind us
         named_bar_sync(1, kSm);
-        // every thread has read the peer-written rows: hand the buffer back
-        if (leader) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->x_free[par]), peer));
+        if (s_verdict[0] != 0) {
+          ok = false;
+          break;
+        }
         // lane h follows head h (all 32 heads, identically in the four warps and in both blocks)
         const int hq = (lane >> 4) * 2;                  // the two warps that hold head `lane`
         const float tm = fmaxf(s_wmax[hq * 16 + (lane & 15)], s_wmax[(hq + 1) * 16 + (lane & 15)]);
@@ -505,7 +523,10 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         mbar_arrive(smem_u32(&bars->p_ready));
       }
 
-      // ---- epilogue: softmax statistics of this item (while the last value MMAs still run) ...
+      // ---- epilogue, once the last value MMAs are done (group wait: one outcome for all)
+      const unsigned gl = gt_base + (unsigned)n_tiles - 1u;
+      ok = mbar_wait_group(smem_u32(&bars->pv_done), gl & 1, s_abort, s_verdict, gw_turn, leader, 2, kSm, 10) && ok;
+      // softmax statistics of this item ...
       if (ok) {
         float wl = 0.f;
 #pragma unroll
@@ -522,11 +543,9 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
           *(float2*)(a.part_ml + ((size_t)item * N + lane) * 2) = make_float2(m_ref, lsum);
         }
       }
-      // ---- ... and this block's half of the partial output: [128 coords x 32 heads] blocks leave
-      //      TMEM with one thread per coordinate, are turned into [32 heads][128 coords] tiles in
-      //      the (now idle) ring and written with one TMA store each
-      const unsigned gl = gt_base + (unsigned)n_tiles - 1u;
-      ok = mbar_wait_group(smem_u32(&bars->pv_done), gl & 1, s_abort, s_verdict, gw_turn, leader, 2, kSm, 10) && ok;
+      // ... and this block's half of the partial output: [128 coords x 32 heads] blocks leave
+      // TMEM with one thread per coordinate, are turned into [32 heads][128 coords] tiles in
+      // the (now idle) ring and written with one TMA store each
       if (ok) {
         tc_fence_after();
         const int trow = quarter * 32 + lane;
@@ -620,9 +639,12 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
             if (LPT >= 4) s += __shfl_xor_sync(0xffffffffu, s, 2);
             part[tt][i] = s;
           }
-        // the softmax threads are done with the previous tile's hand-over
-        ok = rt_wait(smem_u32(&bars->rope_free), (gt & 1) ^ 1, s_abort, 5);
-        if (!ok) break;
+        // the hand-over buffer doubles as the send buffer of the previous tile: it is free once the
+        // peer has handed that tile's rows back (they were copied out of it before)
+        if (gt > 0) {
+          ok = rt_wait<true>(smem_u32(&bars->x_free[(gt - 1) & 1]), ((gt - 1) >> 1) & 1, s_abort, 5);
+          if (!ok) break;
+        }
         if ((lane & (LPT - 1)) == 0) {
 #pragma unroll
           for (int tt = 0; tt < 8; ++tt) {

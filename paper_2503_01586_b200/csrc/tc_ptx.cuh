@@ -299,6 +299,23 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+// Bulk copy of `bytes` (a multiple of 16, both addresses 16-byte aligned) from this block's shared
+// memory into a peer block's; completion is counted in bytes on the PEER's barrier `cbar`
+// (both destination and barrier are addresses mapped with map_to_cta).
+__device__ __forceinline__ void bulk_copy_to_peer(uint32_t cdst, uint32_t src, uint32_t bytes, uint32_t cbar) {
+  asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(cdst), "r"(src), "r"(bytes), "r"(cbar) : "memory");
+}
+// mbar_wait with the acquire taken at cluster scope (a barrier the peer block arrives on)
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, int why,
+                                                  unsigned limit = kWaitLimit) {
+  for (unsigned i = 0; i < limit; ++i) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    if ((i & 1023) == 1023 && *abort_flag) return false;
+  }
+  if (*abort_flag == 0) *abort_flag = why;
+  return false;
+}
 // mbar_wait_group for a barrier the peer block arrives on: same protocol, with the acquire of
 // every thread taken at cluster scope so that the peer's stores are visible afterwards.
 __device__ __forceinline__ bool mbar_wait_group_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,

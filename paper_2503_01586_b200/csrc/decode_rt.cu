@@ -127,7 +127,8 @@ __device__ __forceinline__ bool rt_wait(uint32_t bar, uint32_t parity, volatile 
 template <int R2>
 __global__ void __launch_bounds__(kRtThreads, 1)
 decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_constant__ CUtensorMap map_q,
-                 const __grid_constant__ CUtensorMap map_part, const RtArgs a) {
+                 const __grid_constant__ CUtensorMap map_part, const __grid_constant__ CUtensorMap map_pf,
+                 const RtArgs a) {
   constexpr int N = kHeads;
   constexpr int LPT = R2 / 8;           // 16-byte loads per lane per rope row (row = 32 * R2 bf16)
   extern __shared__ unsigned char smem_raw[];
@@ -158,6 +159,7 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_lat) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_q) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_part) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_pf) : "memory");
   }
   if (threadIdx.x == 0) {
     for (int i = 0; i < kMaxRing; ++i) {
@@ -237,6 +239,18 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
             tma_load_2d_hint(smem_u32(s_q + kc * N * 128), &map_q, (int)rank * DH + kc * 64, seq * N, qb, pol_keep);
         }
         __syncwarp();
+        // The ring holds only half a tile beyond the resident one, so a unit's refill can start
+        // only when the value product has released its slot, and would then wait a full HBM
+        // latency.  The producers therefore pull every tile into L2 one tile ahead
+        // ([64 tokens x 256 coordinates] boxes, no shared memory involved): the refill is an
+        // L2 hit, and HBM keeps streaming while the block is busy with the softmax.
+        auto prefetch_tile = [&](int tile) {
+          if (tile < n_tiles && elect_one()) {
+            const int row = (int)tile_row(seq, tok0 + tile * kT, false);
+            for (int x = prod * 256; x < DH; x += 512) tma_prefetch_2d(&map_pf, (int)rank * DH + x, row);
+          }
+          __syncwarp();
+        };
         bool ok = true;
         for (int tile = 0; tile < n_tiles && ok; ++tile) {
           const int row = (int)tile_row(seq, tok0 + tile * kT, prod == 0 && lane == 0);
@@ -255,6 +269,9 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
             }
             if (++slot == (unsigned)NR) { slot = 0; par ^= 1; }
           }
+          // behind this tile's own loads, so that a prefetch never delays data that is waited for
+          if (tile == 0) prefetch_tile(1);
+          prefetch_tile(tile + 2);
         }
         if (!item_end()) break;
       }
@@ -305,36 +322,49 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
           ok = rt_wait(smem_u32(&bars->p_ready), tiles_done & 1, s_abort, 4);
           if (!ok) break;
           tc_fence_after();
-          // ---- value product: unit u = output block u (two 64-coordinate atoms 8 KB apart)
-          unsigned sb = slot;
-          for (int u = 0; u < NU; ++u) {
-            if (ksteps * 16 > nvalid) {
-              // ragged end of a sequence: rows past its last token inside the last 16-token step
-              // become exact zeros so that zero-probability rows cannot inject NaN/Inf bit patterns
-              unsigned char* unit = s_ring + sb * kUnit;
-              for (int e = lane; e < (ksteps * 16 - nvalid) * 16; e += 32) {
-                const int rrow = nvalid + (e >> 4), c16 = e & 15;
-                *(uint4*)(unit + (c16 >> 3) * 8192 + rrow * 128 + (c16 & 7) * 16) = make_uint4(0, 0, 0, 0);
-              }
-              fence_proxy_async();
-              __syncwarp();
-            }
-            const uint32_t la = (ring16 + sb * (kUnit >> 4)) | (512u << 16);
-            const uint32_t d = tmem_base + (uint32_t)u * N;
+          // ---- value product: unit u = output block u (two 64-coordinate atoms 8 KB apart).
+          //      Entering and leaving an elected block costs about as much as issuing four MMAs,
+          //      so a full tile is issued under one election; every unit still gets its own commit
+          //      so that the producers can refill it as early as possible.
+          if (ksteps == 4) {
             if (elect_one()) {
-              if (ksteps == 4) {
+              unsigned sb = slot;
+              for (int u = 0; u < NU; ++u) {
+                const uint32_t la = (ring16 + sb * (kUnit >> 4)) | (512u << 16);
+                const uint32_t d = tmem_base + (uint32_t)u * N;
                 tc_mma_w(d, la, hi_sw, lo_p, hi_p, idesc_pv, tile != 0);
                 tc_mma_w(d, la + 128, hi_sw, lo_p + 16, hi_p, idesc_pv, 1);   // +16 tokens: 2048 bytes in A, 256 in P
                 tc_mma_w(d, la + 256, hi_sw, lo_p + 32, hi_p, idesc_pv, 1);
                 tc_mma_w(d, la + 384, hi_sw, lo_p + 48, hi_p, idesc_pv, 1);
-              } else {
-                for (int k = 0; k < ksteps; ++k)
-                  tc_mma_w(d, la + 128 * k, hi_sw, lo_p + 16 * k, hi_p, idesc_pv, (tile | k) != 0);
+                tc_commit(empty0 + sb * 8);
+                if (++sb == (unsigned)NR) sb = 0;
               }
-              tc_commit(empty0 + sb * 8);
             }
             __syncwarp();
-            if (++sb == (unsigned)NR) sb = 0;
+          } else {
+            // ragged end of a sequence: rows past its last token inside the last 16-token step
+            // become exact zeros so that zero-probability rows cannot inject NaN/Inf bit patterns
+            unsigned sb = slot;
+            for (int u = 0; u < NU; ++u) {
+              if (ksteps * 16 > nvalid) {
+                unsigned char* unit = s_ring + sb * kUnit;
+                for (int e = lane; e < (ksteps * 16 - nvalid) * 16; e += 32) {
+                  const int rrow = nvalid + (e >> 4), c16 = e & 15;
+                  *(uint4*)(unit + (c16 >> 3) * 8192 + rrow * 128 + (c16 & 7) * 16) = make_uint4(0, 0, 0, 0);
+                }
+                fence_proxy_async();
+                __syncwarp();
+              }
+              const uint32_t la = (ring16 + sb * (kUnit >> 4)) | (512u << 16);
+              const uint32_t d = tmem_base + (uint32_t)u * N;
+              if (elect_one()) {
+                for (int k = 0; k < ksteps; ++k)
+                  tc_mma_w(d, la + 128 * k, hi_sw, lo_p + 16 * k, hi_p, idesc_pv, (tile | k) != 0);
+                tc_commit(empty0 + sb * 8);
+              }
+              __syncwarp();
+              if (++sb == (unsigned)NR) sb = 0;
+            }
           }
           if (elect_one()) tc_commit(smem_u32(&bars->pv_done));
           __syncwarp();
@@ -692,7 +722,8 @@ cudaLaunchAttribute rt_cluster_attr() {
 }
 
 template <int R2>
-int rt_launch(const CUtensorMap& m_lat, const CUtensorMap& m_q, const CUtensorMap& m_part, const RtArgs& a,
+int rt_launch(const CUtensorMap& m_lat, const CUtensorMap& m_q, const CUtensorMap& m_part, const CUtensorMap& m_pf,
+              const RtArgs& a,
               int n_workers, int smem, cudaStream_t st) {
   EKV_CUDA_OK(cudaFuncSetAttribute(decode_rt_kernel<R2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
   cudaLaunchConfig_t cfg = {};
@@ -706,7 +737,7 @@ int rt_launch(const CUtensorMap& m_lat, const CUtensorMap& m_q, const CUtensorMa
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  EKV_CUDA_OK(cudaLaunchKernelEx(&cfg, decode_rt_kernel<R2>, m_lat, m_q, m_part, a));
+  EKV_CUDA_OK(cudaLaunchKernelEx(&cfg, decode_rt_kernel<R2>, m_lat, m_q, m_part, m_pf, a));
   EKV_CUDA_OK(cudaGetLastError());
   return ELITEKV_OK;
 }
@@ -774,10 +805,11 @@ int ekv_launch_decode_rt(const elitekv_layer* L, const elitekv_cache* cache, con
   const unsigned long long rows =
       cv.page_table ? (unsigned long long)cv.num_pages << cv.page_shift : (unsigned long long)cv.max_ctx * cv.n_seqs;
   if (rows >= (1ull << 31)) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
-  CUtensorMap m_lat, m_q, m_part;
+  CUtensorMap m_lat, m_q, m_part, m_pf;
   int rc = make_map(&m_lat, cache->latent, rows, L->d_c, kT);
   if (rc == ELITEKV_OK) rc = make_map(&m_q, q_abs, (unsigned long long)B * L->n_h, L->d_c, kHeads);
   if (rc == ELITEKV_OK) rc = make_map_f32_3d(&m_part, ws.part_acc, L->d_c, L->n_h, (unsigned long long)ws.max_items, kHeads);
+  if (rc == ELITEKV_OK) rc = make_map_plain(&m_pf, cache->latent, rows, L->d_c, 256, kT);
   if (rc != ELITEKV_OK) return rc;
   RtArgs a;
   a.items = ws.items;
@@ -797,8 +829,8 @@ int ekv_launch_decode_rt(const elitekv_layer* L, const elitekv_cache* cache, con
   a.scale_log2e = L->scale * 1.4426950408889634f;
   const int smem = rt_layout(L->d_c, a.n_ring).total;
   switch (2 * L->r) {
-    case 8: return rt_launch<8>(m_lat, m_q, m_part, a, ws.n_workers, smem, st);
-    case 16: return rt_launch<16>(m_lat, m_q, m_part, a, ws.n_workers, smem, st);
-    default: return rt_launch<32>(m_lat, m_q, m_part, a, ws.n_workers, smem, st);
+    case 8: return rt_launch<8>(m_lat, m_q, m_part, m_pf, a, ws.n_workers, smem, st);
+    case 16: return rt_launch<16>(m_lat, m_q, m_part, m_pf, a, ws.n_workers, smem, st);
+    default: return rt_launch<32>(m_lat, m_q, m_part, m_pf, a, ws.n_workers, smem, st);
   }
 }

@@ -30,17 +30,17 @@
 // A cluster is a persistent worker walking its items of the balanced plan (64-token tiles); per
 // item each block writes its half of (acc) and block 0 writes (m, l).
 //
-// Roles per block (384 threads = three warpgroups, each with its own register budget):
-//   warps 0, 2   TMA producers (units dealt alternately); warp 0 also loads the query half
-//   warp 1       TMEM owner and MMA issuer (warp-uniform, instruction under an elected lane;
-//                slot and phase counters advance incrementally so that the descriptor words
-//                stay in uniform registers)
-//   warp 3       idle
-//   warps 4-7    mixing of the partial scores, exchange, softmax, rescale, epilogue
-//   warps 8-11   rope dot products: a warp reads whole rope rows with 16-byte loads per lane
-// Warpgroup 0 gives registers back right away (setmaxnreg), the other two take them: the
-// softmax and rope code would otherwise spill, and with nearly all of L1 carved out as shared
-// memory a spill is an L2 round trip.
+// Roles per block (256 threads):
+//   warps 0, 2   TMA producers (units dealt alternately); warp 0 also loads the query half; both
+//                pull the next tiles into L2 ahead of time
+//   warp 1       TMEM owner and MMA issuer (warp-uniform, instructions under an elected lane,
+//                as many landed units as possible per election; slot and phase counters advance
+//                incrementally so that the descriptor words stay in uniform registers)
+//   warp 3       hands the receive buffer back to the peer
+//   warps 4-7    mixing of the partial scores, exchange, softmax, rescale, epilogue; while the
+//                tensor core works on the value product of a tile and the score product of the
+//                next one they compute the next tile's rope dot products (a warp reads whole rope
+//                rows with 16-byte loads per lane, straight from global memory into registers)
 // Every wait is bounded; on a timeout the block records ELITEKV_ERR_TIMEOUT, stops issuing work
 // and leaves through the common exit (its peer then runs into its own limit).
 #include "tc_ptx.cuh"
@@ -50,18 +50,16 @@ namespace {
 constexpr int kT = 64;                 // tokens per tile
 constexpr int kUnit = 16384;           // ring unit: [2 chunks][64 tokens][64 bf16]
 constexpr int kMaxRing = 9;
-constexpr int kRtThreads = 384;
+constexpr int kRtThreads = 256;
 constexpr int kSm = 128;               // softmax threads (warps 4-7)
-constexpr int kRopeWarps = 4;          // warps 8-11
-// register budgets per warpgroup after the split: 128 * (96 + 224 + 184) = 384 * 168, the launch total
-constexpr int kRegsIssue = 96, kRegsSoftmax = 224, kRegsRope = 184;
 constexpr int kHeads = 32;
 
 struct RtArgs {
   const int32_t* items;
   const int32_t* worker_first;
   const int32_t* page_table;
-  float* part_ml;
+  float* part_acc;          // [items][32][d_c]
+  float* part_ml;           // [items][32][2]
   const bf16* q_rope;       // [B][32][R2]
   const bf16* rope_plane;   // [rows][32 * R2]
   int32_t* status;
@@ -75,7 +73,7 @@ struct RtArgs {
 
 struct __align__(8) RtBarriers {
   uint64_t full[kMaxRing], empty[kMaxRing];
-  uint64_t q_full, s_full, p_ready, pv_done, rope_ready, recv_done;
+  uint64_t q_full, q_free, s_full, p_ready, pv_done, recv_done;
   uint64_t x_full[2], x_free[2];
 };
 
@@ -127,8 +125,7 @@ __device__ __forceinline__ bool rt_wait(uint32_t bar, uint32_t parity, volatile 
 template <int R2>
 __global__ void __launch_bounds__(kRtThreads, 1)
 decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_constant__ CUtensorMap map_q,
-                 const __grid_constant__ CUtensorMap map_part, const __grid_constant__ CUtensorMap map_pf,
-                 const RtArgs a) {
+                 const __grid_constant__ CUtensorMap map_pf, const RtArgs a) {
   constexpr int N = kHeads;
   constexpr int LPT = R2 / 8;           // 16-byte loads per lane per rope row (row = 32 * R2 bf16)
   extern __shared__ unsigned char smem_raw[];
@@ -158,7 +155,6 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   if (threadIdx.x == 32) {
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_lat) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_q) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_part) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_pf) : "memory");
   }
   if (threadIdx.x == 0) {
@@ -167,11 +163,11 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       mbar_init(smem_u32(&bars->empty[i]), 1);
     }
     mbar_init(smem_u32(&bars->q_full), 1);
+    mbar_init(smem_u32(&bars->q_free), 1);
     mbar_init(smem_u32(&bars->s_full), 1);
-    mbar_init(smem_u32(&bars->p_ready), kSm);
+    mbar_init(smem_u32(&bars->p_ready), kSm / 32);
     mbar_init(smem_u32(&bars->pv_done), 1);
-    mbar_init(smem_u32(&bars->rope_ready), kRopeWarps);
-    mbar_init(smem_u32(&bars->recv_done), kSm);
+    mbar_init(smem_u32(&bars->recv_done), kSm / 32);
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&bars->x_full[i]), 1);       // armed per tile; completed by the peer's bulk copy
       mbar_init(smem_u32(&bars->x_free[i]), 1);
@@ -209,19 +205,13 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
     }
     return ((long long)page << a.page_shift) + (t_abs & a.page_mask);
   };
-  // end of an item: every role is done with the queries, the P tile, the ring and the output
-  // columns.  All 384 threads meet here from their own loops; false = the block is aborting
-  // (same answer in every thread: nobody is inside a wait at this point).
-  auto item_end = [&]() -> bool {
-    tc_fence_before();
-    named_bar_sync(3, kRtThreads);
-    tc_fence_after();
-    return *s_abort == 0;
-  };
+  // Items follow one another without a block-wide barrier: the roles are coupled only through
+  // the mbarriers of the data they hand over (the query half through q_full / q_free, tiles
+  // through the ring, scores and probabilities through s_full / p_ready), so the loads and the
+  // score product of the next item run under the epilogue of the current one.
   int seq = -1;
 
   if (warp < 4) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIssue));
     // ============================================================ warps 0, 2: TMA producers
     if (warp == 0 || warp == 2) {
       const int prod = warp >> 1;
@@ -231,6 +221,10 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         seq = a.items[4 * item + 0];
         const int tok0 = a.items[4 * item + 1];
         const int n_tiles = (a.items[4 * item + 2] + kT - 1) / kT;
+        if (prod == 0 && item > item_lo) {
+          // the score product of the previous item's last tile has read the query half
+          if (!rt_wait(smem_u32(&bars->q_free), (unsigned)(item - item_lo - 1) & 1, s_abort, 12)) break;
+        }
         if (prod == 0 && elect_one()) {
           // this block's half of the sequence's absorbed queries: stays for the whole item
           const uint32_t qb = smem_u32(&bars->q_full);
@@ -273,7 +267,7 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
           if (tile == 0) prefetch_tile(1);
           prefetch_tile(tile + 2);
         }
-        if (!item_end()) break;
+        if (!ok) break;
       }
     }
     // ============================================================ warp 1: MMA issuer
@@ -298,25 +292,51 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         for (int tile = 0; tile < n_tiles && ok; ++tile) {
           const int nvalid = min(kT, ntok - tile * kT);
           const int ksteps = (nvalid + 15) >> 4;
-          // ---- partial scores: one unit (two chunks) per 4 MMAs
+          // ---- partial scores: 4 MMAs per unit (two chunks).  Units whose data has already landed
+          //      are issued under one election (probing a completed phase is cheap, entering an
+          //      elected block is not); only a unit that is still in flight is waited for.
           unsigned sa = slot, pa = par;
           uint32_t lb = q16 | (1u << 16);
-          for (int u = 0; u < NU; ++u) {
-            ok = rt_wait(full0 + sa * 8, pa, s_abort, 3);
-            if (!ok) break;
-            const uint32_t la = (ring16 + sa * (kUnit >> 4)) | (1u << 16);
+          int u = 0;
+          while (u < NU) {
+            int n_ready = 0;
+            {
+              unsigned s2 = sa, p2 = pa;
+              while (u + n_ready < NU && __any_sync(0xffffffffu, mbar_test_wait(full0 + s2 * 8, p2))) {
+                ++n_ready;
+                if (++s2 == (unsigned)NR) { s2 = 0; p2 ^= 1; }
+              }
+            }
+            if (n_ready == 0) {
+              ok = rt_wait(full0 + sa * 8, pa, s_abort, 3);
+              if (!ok) break;
+              n_ready = 1;
+            }
             if (elect_one()) {
-              tc_mma_w(tmem_s, la, hi_sw, lb, hi_sw, idesc_s, u != 0);
-              tc_mma_w(tmem_s, la + 2, hi_sw, lb + 2, hi_sw, idesc_s, 1);     // +32 bytes along K per step
-              tc_mma_w(tmem_s, la + 4, hi_sw, lb + 4, hi_sw, idesc_s, 1);
-              tc_mma_w(tmem_s, la + 6, hi_sw, lb + 6, hi_sw, idesc_s, 1);
+              unsigned s2 = sa;
+              uint32_t lb2 = lb;
+              for (int k = 0; k < n_ready; ++k) {
+                const uint32_t la = (ring16 + s2 * (kUnit >> 4)) | (1u << 16);
+                tc_mma_w(tmem_s, la, hi_sw, lb2, hi_sw, idesc_s, (u + k) != 0);
+                tc_mma_w(tmem_s, la + 2, hi_sw, lb2 + 2, hi_sw, idesc_s, 1);   // +32 bytes along K per step
+                tc_mma_w(tmem_s, la + 4, hi_sw, lb2 + 4, hi_sw, idesc_s, 1);
+                tc_mma_w(tmem_s, la + 6, hi_sw, lb2 + 6, hi_sw, idesc_s, 1);
+                lb2 += 512u;                                                   // next pair of query chunks
+                if (++s2 == (unsigned)NR) s2 = 0;
+              }
             }
             __syncwarp();
-            lb += 512u;                                                       // next pair of query chunks
-            if (++sa == (unsigned)NR) { sa = 0; pa ^= 1; }
+            for (int k = 0; k < n_ready; ++k) {
+              lb += 512u;
+              if (++sa == (unsigned)NR) { sa = 0; pa ^= 1; }
+            }
+            u += n_ready;
           }
           if (!ok) break;
-          if (elect_one()) tc_commit(smem_u32(&bars->s_full));
+          if (elect_one()) {
+            tc_commit(smem_u32(&bars->s_full));
+            if (tile == n_tiles - 1) tc_commit(smem_u32(&bars->q_free));   // the query half may be replaced
+          }
           __syncwarp();
           // ---- wait for P (and the rescaled output) of this tile
           ok = rt_wait(smem_u32(&bars->p_ready), tiles_done & 1, s_abort, 4);
@@ -372,7 +392,7 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
           par = pa;
           ++tiles_done;
         }
-        if (!item_end()) break;
+        if (!ok) break;
       }
     }
     // ============================================================ warp 3: hand-back of the receive buffer
@@ -390,12 +410,11 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
           if (elect_one()) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->x_free[gt & 1]), peer));
           __syncwarp();
         }
-        if (!item_end()) break;
+        if (!ok) break;
       }
     }
   }
-  else if (warp < 8) {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
+  else {
     // ============================================================ warps 4-7: scores -> P, rescale, epilogue
     // Thread (quarter, lane) may touch TMEM lanes 32 quarter + lane.  Quarters 0, 1 hold the
     // even-chunk diagonal block (accumulator rows = tokens 0-63, columns 0-31), quarters 2, 3 the
@@ -422,6 +441,78 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       for (int i = 0; i < 16; ++i) l_part[i] = 0.f;
       float m_ref = -INFINITY;                           // lane h: reference maximum of head h (all 32, in every warp)
       bool ok = true;
+      // ---- rope part of the scores (FP32 FMA): the block adds it for tokens [32 rank, 32 rank + 32)
+      // of every tile, a warp taking 8 of them.  A rope row is 32 heads x R2 bf16 = 4 R2 pieces of
+      // 16 bytes; lane L of load i reads piece 32 i + L (one coalesced 512-byte request per
+      // load), which belongs to head 8 (32 i + L) / R2.  The sums go to s_xmix[token][head], the
+      // buffer the two halves of the block mix their partial scores in.
+      const int tok0 = a.items[4 * item + 1];
+      float qr[LPT][8];
+#pragma unroll
+      for (int i = 0; i < LPT; ++i) {
+        const uint4 v = *(const uint4*)(a.q_rope + (size_t)seq * N * R2 + 8 * (32 * i + lane));
+        const bf162* p2 = (const bf162*)&v;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float2 f = __bfloat1622float2(p2[j]);
+          qr[i][2 * j] = f.x;
+          qr[i][2 * j + 1] = f.y;
+        }
+      }
+      // `g` = global tile count of the tile; the buffer was the send buffer of tile g - 1 and is free
+      // once the peer has handed that tile's rows back
+      auto rope_tile = [&](int tile, unsigned g) {
+        const int nvalid = min(kT, ntok - tile * kT);
+        const long long row0 = tile_row(seq, tok0 + tile * kT, false);
+        float part[8][LPT];
+#pragma unroll
+        for (int tt = 0; tt < 8; ++tt) {
+          const int tk = 32 * (int)rank + 8 * quarter + tt;
+          uint4 v[LPT];
+#pragma unroll
+          for (int i = 0; i < LPT; ++i) {
+            v[i] = make_uint4(0, 0, 0, 0);
+            if (tk < nvalid)
+              v[i] = __ldcs((const uint4*)(a.rope_plane + (size_t)(row0 + tk) * (size_t)(N * R2)) + 32 * i + lane);
+          }
+#pragma unroll
+          for (int i = 0; i < LPT; ++i) {
+            const bf162* k2 = (const bf162*)&v[i];
+            float acc = 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const float2 f = __bfloat1622float2(k2[j]);
+              acc = fmaf(qr[i][2 * j], f.x, acc);
+              acc = fmaf(qr[i][2 * j + 1], f.y, acc);
+            }
+            part[tt][i] = acc;
+          }
+        }
+        // sum over the LPT adjacent lanes that share a head
+#pragma unroll
+        for (int tt = 0; tt < 8; ++tt)
+#pragma unroll
+          for (int i = 0; i < LPT; ++i) {
+            float v = part[tt][i];
+            if (LPT >= 2) v += __shfl_xor_sync(0xffffffffu, v, 1);
+            if (LPT >= 4) v += __shfl_xor_sync(0xffffffffu, v, 2);
+            part[tt][i] = v;
+          }
+        if (g > 0) (void)mbar_wait_cluster(smem_u32(&bars->x_free[(g - 1) & 1]), ((g - 1) >> 1) & 1, s_abort, 5);
+        if ((lane & (LPT - 1)) == 0) {
+#pragma unroll
+          for (int tt = 0; tt < 8; ++tt) {
+            const int tk = 32 * (int)rank + 8 * quarter + tt;
+#pragma unroll
+            for (int i = 0; i < LPT; ++i) {
+              const int h = (8 * (32 * i + lane)) / R2;
+              s_xmix[tk * N + ((((h >> 2) + tk) & 7) << 2) + (h & 3)] = part[tt][i];
+            }
+          }
+        }
+        named_bar_sync(1, kSm);              // rows are read by other warps than the ones that wrote them
+      };
+      rope_tile(0, gt_base);
       for (int tile = 0; tile < n_tiles; ++tile) {
         const unsigned gt = gt_base + (unsigned)tile, par = gt & 1, k2 = gt >> 1;
         const int nvalid = min(kT, ntok - tile * kT);
@@ -437,7 +528,6 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         tc_wait_ld();
         if (leader) mbar_expect_tx(smem_u32(&bars->x_full[par]), (uint32_t)(kT * N * 4));   // the peer's rows of this tile
         // ---- hand the partner its 16 heads (on top of the rope part where this block owns it)
-        (void)mbar_wait(smem_u32(&bars->rope_ready), gt & 1, s_abort, 7);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int c = 4 * (1 - hh) + j;                // logical 16-byte chunk = heads 4c .. 4c+3
@@ -484,7 +574,8 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
             s[4 * j] += x.x; s[4 * j + 1] += x.y; s[4 * j + 2] += x.z; s[4 * j + 3] += x.w;
           }
         }
-        mbar_arrive(smem_u32(&bars->recv_done));         // warp 3 hands the buffer back to the peer
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars->recv_done));   // warp 3 hands the buffer back to the peer
         const bool live = t < nvalid;
 #pragma unroll
         for (int i = 0; i < 16; ++i) s[i] = live ? s[i] * a.scale_log2e : -INFINITY;
@@ -550,7 +641,10 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         }
         fence_proxy_async();
         tc_fence_before();
-        mbar_arrive(smem_u32(&bars->p_ready));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars->p_ready));
+        // ---- the tensor core is busy with this tile's value product and the next tile's scores
+        if (tile + 1 < n_tiles) rope_tile(tile + 1, gt + 1);
       }
 
       // ---- epilogue, once the last value MMAs are done (group wait: one outcome for all)
@@ -573,123 +667,24 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
           *(float2*)(a.part_ml + ((size_t)item * N + lane) * 2) = make_float2(m_ref, lsum);
         }
       }
-      // ... and this block's half of the partial output: [128 coords x 32 heads] blocks leave
-      // TMEM with one thread per coordinate, are turned into [32 heads][128 coords] tiles in
-      // the (now idle) ring and written with one TMA store each
+      // ... and this block's half of the partial output: a [128 coords x 32 heads] block leaves
+      // TMEM with one thread per coordinate, so for a fixed head the lanes of a warp hold 32
+      // consecutive coordinates: 128-byte stores straight from registers.  No shared memory is
+      // involved, so the ring already carries the next item's tiles meanwhile.
       if (ok) {
         tc_fence_after();
-        const int trow = quarter * 32 + lane;
+        float* dst = a.part_acc + (size_t)item * N * d_c + (size_t)rank * DH + quarter * 32 + lane;
         for (int blk = 0; blk < NU; ++blk) {
           float v[32];
           tc_ld32(tmem_base + blk * N + lane_base, v);
           tc_wait_ld();
-          float* tile_s = (float*)(s_ring + (size_t)blk * kUnit);
 #pragma unroll
-          for (int h = 0; h < 32; ++h) tile_s[h * 128 + trow] = v[h];
-          fence_proxy_async();
-          named_bar_sync(1, kSm);
-          if (leader) {
-            tma_store_3d(&map_part, (int)rank * DH + blk * 128, 0, item, smem_u32(tile_s));
-            bulk_commit_group();
-          }
+          for (int h = 0; h < 32; ++h) __stcg(dst + (size_t)h * d_c + blk * 128, v[h]);
         }
-        if (leader) bulk_wait_group_all();     // stores done before the ring is reused or the block leaves
+        tc_fence_before();     // the next item's first value MMA overwrites these columns (after p_ready)
       }
       gt_base += (unsigned)n_tiles;
-      if (!item_end()) break;
-      }
-    }
-  }
-  else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsRope));
-    // ============================================================ warps 8-11: rope dot products
-    // The block adds the rope part for tokens [32 rank, 32 rank + 32) of every tile.  A warp
-    // takes 8 of them; a rope row is 32 heads x R2 bf16 = 4 R2 pieces of 16 bytes, lane L of
-    // load i reads piece 32 i + L (one coalesced 512-byte request per load), which belongs to
-    // head 8 (32 i + L) / R2.  The products wait in registers until the softmax threads have
-    // released the hand-over buffer, then the per-head sums go to s_xmix[token][head].
-    {
-      const int rw = warp - 8;
-      unsigned gt = 0;                   // tiles of this worker so far
-      for (int item = item_lo; item < item_hi; ++item) {
-      seq = a.items[4 * item + 0];
-      const int tok0 = a.items[4 * item + 1];
-      const int ntok = a.items[4 * item + 2];
-      const int n_tiles = (ntok + kT - 1) / kT;
-      float qr[LPT][8];
-#pragma unroll
-      for (int i = 0; i < LPT; ++i) {
-        const int e0 = 8 * (32 * i + lane);          // first element of the piece inside the row
-        const bf16* src = a.q_rope + (size_t)seq * N * R2 + e0;
-        const uint4 v = *(const uint4*)src;
-        const bf162* p2 = (const bf162*)&v;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const float2 f = __bfloat1622float2(p2[j]);
-          qr[i][2 * j] = f.x;
-          qr[i][2 * j + 1] = f.y;
-        }
-      }
-      bool ok = true;
-      const size_t row_elems = (size_t)N * R2;
-      for (int tile = 0; tile < n_tiles && ok; ++tile, ++gt) {
-        const int nvalid = min(kT, ntok - tile * kT);
-        const long long row0 = tile_row(seq, tok0 + tile * kT, false);
-        float part[8][LPT];
-#pragma unroll
-        for (int tt = 0; tt < 8; ++tt) {
-          const int t = 32 * (int)rank + 8 * rw + tt;
-          uint4 v[LPT];
-#pragma unroll
-          for (int i = 0; i < LPT; ++i) {
-            v[i] = make_uint4(0, 0, 0, 0);
-            if (t < nvalid)
-              v[i] = __ldcs((const uint4*)(a.rope_plane + (size_t)(row0 + t) * row_elems) + 32 * i + lane);
-          }
-#pragma unroll
-          for (int i = 0; i < LPT; ++i) {
-            const bf162* k2 = (const bf162*)&v[i];
-            float acc = 0.f;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const float2 f = __bfloat1622float2(k2[j]);
-              acc = fmaf(qr[i][2 * j], f.x, acc);
-              acc = fmaf(qr[i][2 * j + 1], f.y, acc);
-            }
-            part[tt][i] = acc;
-          }
-        }
-        // sum over the LPT adjacent lanes that share a head
-#pragma unroll
-        for (int tt = 0; tt < 8; ++tt)
-#pragma unroll
-          for (int i = 0; i < LPT; ++i) {
-            float s = part[tt][i];
-            if (LPT >= 2) s += __shfl_xor_sync(0xffffffffu, s, 1);
-            if (LPT >= 4) s += __shfl_xor_sync(0xffffffffu, s, 2);
-            part[tt][i] = s;
-          }
-        // the hand-over buffer doubles as the send buffer of the previous tile: it is free once the
-        // peer has handed that tile's rows back (they were copied out of it before)
-        if (gt > 0) {
-          ok = rt_wait<true>(smem_u32(&bars->x_free[(gt - 1) & 1]), ((gt - 1) >> 1) & 1, s_abort, 5);
-          if (!ok) break;
-        }
-        if ((lane & (LPT - 1)) == 0) {
-#pragma unroll
-          for (int tt = 0; tt < 8; ++tt) {
-            const int t = 32 * (int)rank + 8 * rw + tt;
-#pragma unroll
-            for (int i = 0; i < LPT; ++i) {
-              const int h = (8 * (32 * i + lane)) / R2;
-              s_xmix[t * N + ((((h >> 2) + t) & 7) << 2) + (h & 3)] = part[tt][i];
-            }
-          }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bars->rope_ready));
-      }
-      if (!item_end()) break;
+      if (!ok) break;
       }
     }
   }
@@ -722,7 +717,7 @@ cudaLaunchAttribute rt_cluster_attr() {
 }
 
 template <int R2>
-int rt_launch(const CUtensorMap& m_lat, const CUtensorMap& m_q, const CUtensorMap& m_part, const CUtensorMap& m_pf,
+int rt_launch(const CUtensorMap& m_lat, const CUtensorMap& m_q, const CUtensorMap& m_pf,
               const RtArgs& a,
               int n_workers, int smem, cudaStream_t st) {
   EKV_CUDA_OK(cudaFuncSetAttribute(decode_rt_kernel<R2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
@@ -737,7 +732,7 @@ int rt_launch(const CUtensorMap& m_lat, const CUtensorMap& m_q, const CUtensorMa
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  EKV_CUDA_OK(cudaLaunchKernelEx(&cfg, decode_rt_kernel<R2>, m_lat, m_q, m_part, m_pf, a));
+  EKV_CUDA_OK(cudaLaunchKernelEx(&cfg, decode_rt_kernel<R2>, m_lat, m_q, m_pf, a));
   EKV_CUDA_OK(cudaGetLastError());
   return ELITEKV_OK;
 }
@@ -805,16 +800,16 @@ int ekv_launch_decode_rt(const elitekv_layer* L, const elitekv_cache* cache, con
   const unsigned long long rows =
       cv.page_table ? (unsigned long long)cv.num_pages << cv.page_shift : (unsigned long long)cv.max_ctx * cv.n_seqs;
   if (rows >= (1ull << 31)) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
-  CUtensorMap m_lat, m_q, m_part, m_pf;
+  CUtensorMap m_lat, m_q, m_pf;
   int rc = make_map(&m_lat, cache->latent, rows, L->d_c, kT);
   if (rc == ELITEKV_OK) rc = make_map(&m_q, q_abs, (unsigned long long)B * L->n_h, L->d_c, kHeads);
-  if (rc == ELITEKV_OK) rc = make_map_f32_3d(&m_part, ws.part_acc, L->d_c, L->n_h, (unsigned long long)ws.max_items, kHeads);
   if (rc == ELITEKV_OK) rc = make_map_plain(&m_pf, cache->latent, rows, L->d_c, 256, kT);
   if (rc != ELITEKV_OK) return rc;
   RtArgs a;
   a.items = ws.items;
   a.worker_first = ws.worker_first;
   a.page_table = cv.page_table;
+  a.part_acc = ws.part_acc;
   a.part_ml = ws.part_ml;
   a.q_rope = (const bf16*)q_rope;
   a.rope_plane = (const bf16*)cache->rope;
@@ -829,8 +824,8 @@ int ekv_launch_decode_rt(const elitekv_layer* L, const elitekv_cache* cache, con
   a.scale_log2e = L->scale * 1.4426950408889634f;
   const int smem = rt_layout(L->d_c, a.n_ring).total;
   switch (2 * L->r) {
-    case 8: return rt_launch<8>(m_lat, m_q, m_part, m_pf, a, ws.n_workers, smem, st);
-    case 16: return rt_launch<16>(m_lat, m_q, m_part, m_pf, a, ws.n_workers, smem, st);
-    default: return rt_launch<32>(m_lat, m_q, m_part, m_pf, a, ws.n_workers, smem, st);
+    case 8: return rt_launch<8>(m_lat, m_q, m_pf, a, ws.n_workers, smem, st);
+    case 16: return rt_launch<16>(m_lat, m_q, m_pf, a, ws.n_workers, smem, st);
+    default: return rt_launch<32>(m_lat, m_q, m_pf, a, ws.n_workers, smem, st);
   }
 }

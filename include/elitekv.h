@@ -174,22 +174,25 @@ int elitekv_plan(const int32_t* seq_lens, int32_t B, int32_t tile_tokens, int32_
                  int32_t* items, int32_t* seq_first_item, elitekv_stream_t stream);
 
 /* The plan of the kernels whose blocks are persistent workers (the paper has no counterpart),
- * exported for inspection.  Worker w owns the global tile range [w*quota, (w+1)*quota),
- * quota = ceil(total tiles / n_workers); an item is the part of one sequence inside one
- * worker's range, so items come out ordered by sequence and by worker.
+ * exported for inspection.  Worker w owns the global tile range [w*total/n, (w+1)*total/n),
+ * n = min(n_workers, total) (integer division; later workers stay idle); an item is the part
+ * of one sequence inside one worker's range, so items come out ordered by sequence and worker.
  *   items int32 [max_items][4] = (sequence, first token, token count, worker), unused entries
  *   sequence = -1;  seq_first_item int32 [B+1];  worker_first int32 [n_workers+1]: items of
- *   worker w are [worker_first[w], worker_first[w+1]).  max_items >= B + n_workers. */
+ *   worker w are [worker_first[w], worker_first[w+1]).  max_items >= B + n_workers.
+ * item_overhead_tiles (>= 0): empty tiles counted in front of every sequence when the ranges
+ * are cut, the price of starting one more item; 0 gives the plain equal-tile cut. */
 int elitekv_plan_workers(const int32_t* seq_lens, int32_t B, int32_t tile_tokens, int32_t n_workers,
-                         int32_t max_items, int32_t* items, int32_t* seq_first_item,
-                         int32_t* worker_first, elitekv_stream_t stream);
+                         int32_t item_overhead_tiles, int32_t max_items, int32_t* items,
+                         int32_t* seq_first_item, int32_t* worker_first, elitekv_stream_t stream);
 
 /* Which split-K kernel and plan elitekv_decode uses for this layer, cache layout (may be NULL:
  * shape-only answer) and batch (the paper has no counterpart).  info is a HOST array:
  * info[0] = kernel (1, 2, 3 as in elitekv_params.decode_kernel), info[1] = tokens per plan tile,
- * info[2] = persistent workers (0: the plain plan of elitekv_plan), info[3] = plan capacity. */
+ * info[2] = persistent workers (0: the plain plan of elitekv_plan), info[3] = plan capacity,
+ * info[4] = item_overhead_tiles of elitekv_plan_workers. */
 int elitekv_decode_plan_info(const elitekv_layer* layer, const elitekv_cache* cache, int32_t B,
-                             int32_t info[4]);
+                             int32_t info[5]);
 
 /* Synchronises `stream`, returns the layer's device status word (0 or a negative
  * elitekv_status recorded by a kernel) and clears it. */

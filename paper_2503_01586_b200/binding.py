@@ -66,8 +66,8 @@ def lib() -> C.CDLL:
         L.elitekv_decode.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, i32, vp, sz, vp, vp]
         L.elitekv_decode_static.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, i32, vp, vp]
         L.elitekv_plan.argtypes = [vp, i32, i32, i32, vp, vp, vp]
-        L.elitekv_plan_workers.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp]
-        L.elitekv_decode_plan_info.argtypes = [vp, C.POINTER(CacheDesc), i32, C.POINTER(i32 * 4)]
+        L.elitekv_plan_workers.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp]
+        L.elitekv_decode_plan_info.argtypes = [vp, C.POINTER(CacheDesc), i32, C.POINTER(i32 * 5)]
         L.elitekv_check_status.argtypes = [vp, vp]
         L.elitekv_last_status_detail.argtypes = [vp, C.POINTER(i32 * 3)]
         L.elitekv_selftest_bounded_wait.argtypes = [vp, C.c_uint32, vp]
@@ -224,20 +224,21 @@ def elitekv_plan(seq_lens, tile_tokens: int, max_items: int):
     return items, first
 
 
-def elitekv_plan_workers(seq_lens, tile_tokens: int, n_workers: int, max_items: int):
+def elitekv_plan_workers(seq_lens, tile_tokens: int, n_workers: int, max_items: int,
+                         item_overhead_tiles: int = 0):
     B = seq_lens.shape[0]
     items = torch.empty((max_items, 4), dtype=torch.int32, device=seq_lens.device)
     first = torch.empty((B + 1,), dtype=torch.int32, device=seq_lens.device)
     wfirst = torch.empty((n_workers + 1,), dtype=torch.int32, device=seq_lens.device)
     _check(lib().elitekv_plan_workers(_ptr(_dev(seq_lens, torch.int32)), B, tile_tokens, n_workers,
-                                      max_items, _ptr(items), _ptr(first), _ptr(wfirst), _stream()),
+                                      item_overhead_tiles, max_items, _ptr(items), _ptr(first), _ptr(wfirst), _stream()),
            "elitekv_plan_workers")
     return items, first, wfirst
 
 
 def elitekv_decode_plan_info(layer: Layer, cache: Optional[CacheDesc], B: int):
-    """(kernel, tokens per plan tile, persistent workers, plan capacity)."""
-    info = (C.c_int32 * 4)()
+    """(kernel, tokens per plan tile, persistent workers, plan capacity, item overhead tiles)."""
+    info = (C.c_int32 * 5)()
     _check(lib().elitekv_decode_plan_info(layer.handle, C.byref(cache) if cache is not None else None,
                                           B, C.byref(info)), "elitekv_decode_plan_info")
     return tuple(int(x) for x in info)

@@ -26,6 +26,9 @@ int max_items_for(const elitekv_layer* L, int B, int kernel) {
 
 // Tokens per plan tile and persistent workers (0: the plain plan) of each kernel.
 int plan_tile_for(int kernel) { return kernel == 2 ? 128 : ELITEKV_TILE_TOKENS; }
+// Tiles' worth of time that starting an item costs a worker (measured on B200: about one
+// 64-token tile for the resident-tile kernel).
+int item_overhead_for(int kernel) { return kernel == 3 ? 1 : 0; }
 int workers_for(const elitekv_layer* L, int kernel) {
   return kernel == 3 ? ekv_rt_workers(L) : kernel == 2 ? ekv_tc_workers(L) : 0;
 }
@@ -98,7 +101,7 @@ extern "C" int elitekv_decode_workspace_size(const elitekv_layer* L, int32_t B, 
 }
 
 extern "C" int elitekv_decode_plan_info(const elitekv_layer* L, const elitekv_cache* cache, int32_t B,
-                                        int32_t info[4]) {
+                                        int32_t info[5]) {
   if (!L || !info || B <= 0) return ELITEKV_ERR_INVALID_ARG;
   const int kernel = select_kernel(L, cache);
   if (kernel < 0) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
@@ -106,6 +109,7 @@ extern "C" int elitekv_decode_plan_info(const elitekv_layer* L, const elitekv_ca
   info[1] = plan_tile_for(kernel);
   info[2] = workers_for(L, kernel);
   info[3] = max_items_for(L, B, kernel);
+  info[4] = item_overhead_for(kernel);
   return ELITEKV_OK;
 }
 
@@ -142,7 +146,8 @@ extern "C" int elitekv_decode(const elitekv_layer* L, const elitekv_cache* cache
   const long long max_len = cv.page_table ? (long long)cv.max_pages_per_seq << cv.page_shift : cv.max_ctx;
   if (ws.n_workers > 0)
     rc = ekv_launch_plan_balanced(seq_lens, B, plan_tile_for(kernel), ws.n_workers, max_items, ws.items, ws.seq_first,
-                                  ws.worker_first, ws.counters, ws.n_counters, max_len, L->d_status, st);
+                                  ws.worker_first, ws.counters, ws.n_counters, max_len, L->d_status,
+                                  item_overhead_for(kernel), st);
   else
     rc = ekv_launch_plan(seq_lens, B, plan_tile_for(kernel), max_items, ws.items, ws.seq_first,
                          ws.counters, ws.n_counters, max_len, L->d_status, st);

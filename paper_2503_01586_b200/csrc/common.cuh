@@ -152,7 +152,7 @@ int ekv_launch_plan(const int32_t* seq_lens, int B, int tile_tokens, int max_ite
 int ekv_launch_plan_balanced(const int32_t* seq_lens, int B, int tile_tokens, int n_workers,
                              int max_items, int32_t* items, int32_t* seq_first_item,
                              int32_t* worker_first, int32_t* zero_ints, int n_zero, long long max_len,
-                             int32_t* status, cudaStream_t st);
+                             int32_t* status, int overhead_tiles, cudaStream_t st);
 
 struct DecodeScratch {
   int max_items;          // capacity of the plan

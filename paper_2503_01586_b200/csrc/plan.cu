@@ -100,15 +100,20 @@ plan_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int max_items
 }
 
 // Balanced plan for kernels whose blocks walk several items: worker w of `n_workers` owns the
-// global tile range [w*quota, (w+1)*quota), quota = ceil(total / n_workers); an item is the
+// global tile range [w*total/n, (w+1)*total/n), n = min(n_workers, total) (integer division: the
+// ranges differ by at most one tile and none is empty); an item is the
 // intersection of one worker's range with one sequence.  Items come out in global order, so they
 // are grouped by sequence (seq_first) and by worker (worker_first).  items[i] = (sequence, first
 // token, token count, worker).
+// Starting an item costs a worker about as much as `overhead` tiles (new queries, a partial
+// result to write out), and a worker whose range contains the start of a sequence has one item
+// more than the others.  The tile list therefore carries `overhead` empty tiles in front of every
+// sequence: they take room in a worker's quota and hold no tokens.
 __global__ void __launch_bounds__(kPlanThreads)
 plan_balanced_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int n_workers,
                      int max_items, int32_t* __restrict__ items, int32_t* __restrict__ seq_first,
                      int32_t* __restrict__ worker_first, int32_t* __restrict__ zero_ints, int n_zero,
-                     long long max_len, int32_t* status) {
+                     long long max_len, int32_t* status, int overhead) {
   __shared__ int warp_tot[kPlanThreads / 32];
   __shared__ long long s_total;
   const int t = threadIdx.x;
@@ -120,14 +125,16 @@ plan_balanced_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int 
   long long local = 0;
   for (int b = t; b < B; b += blockDim.x) {
     int n = checked_len(seq_lens, b, max_len, status, true);
-    local += n > 0 ? (n + tile - 1) / tile : 0;
+    local += n > 0 ? (n + tile - 1) / tile + overhead : 0;
   }
   if (local) atomicAdd((unsigned long long*)&s_total, (unsigned long long)local);
   __syncthreads();
-  const long long total = s_total;
-  long long quota = (total + n_workers - 1) / n_workers;
-  if (quota < 1) quota = 1;
-
+  const long long total = s_total > 0 ? s_total : 1;
+  // first position of worker w's range, and the worker that owns position g
+  // (with fewer positions than workers only the first `total` workers get a range, of one each)
+  const long long nw = total < n_workers ? total : n_workers;
+  auto bound = [&](long long w) -> long long { return w * total / nw; };
+  auto owner = [&](long long g) -> int { return (int)(((g + 1) * nw - 1) / total); };
   // pass 1: count items to know n_items (default of worker_first)
   int carry_tiles = 0, carry_items = 0;
   // per-thread record of its sequences is recomputed in pass 2; B is small compared to the block
@@ -139,14 +146,14 @@ plan_balanced_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int 
       int n = 0, tiles = 0;
       if (b < B) {
         n = checked_len(seq_lens, b, max_len, status, false);
-        tiles = n > 0 ? (n + tile - 1) / tile : 0;
+        tiles = n > 0 ? (n + tile - 1) / tile + overhead : 0;     // with the empty tiles in front
       }
       int chunk_tiles;
       const int g0 = carry_tiles + block_exclusive_scan(tiles, warp_tot, &chunk_tiles);
       int pieces = 0, w0 = 0;
       if (tiles > 0) {
-        w0 = (int)(g0 / quota);
-        const int w1 = (int)((g0 + tiles - 1) / quota);
+        w0 = owner(g0 + overhead);                                // workers that hold real tiles
+        const int w1 = owner(g0 + tiles - 1);
         pieces = w1 - w0 + 1;
       }
       int chunk_items;
@@ -154,15 +161,12 @@ plan_balanced_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int 
       if (pass == 1 && b < B) {
         seq_first[b] = first;
         for (int j = 0; j < pieces; ++j) {
-          const long long ga = max((long long)g0, (w0 + j) * quota);
-          const long long gb = min((long long)g0 + tiles, (w0 + j + 1) * quota);
-          const int tok0 = (int)(ga - g0) * tile;
-          const int tok1 = min((int)(gb - g0) * tile, n);
+          const long long ga = max((long long)g0 + overhead, bound(w0 + j));
+          const long long gb = min((long long)g0 + tiles, bound(w0 + j + 1));
+          const int tok0 = (int)(ga - g0 - overhead) * tile;
+          const int tok1 = min((int)(gb - g0 - overhead) * tile, n);
           const int it = first + j;
-          if (it < max_items) {
-            *(int4*)(items + 4 * it) = make_int4(b, tok0, tok1 - tok0, w0 + j);
-            if (ga == (w0 + j) * quota) worker_first[w0 + j] = it;
-          }
+          if (it < max_items) *(int4*)(items + 4 * it) = make_int4(b, tok0, tok1 - tok0, w0 + j);
         }
       }
       carry_tiles += chunk_tiles;
@@ -175,6 +179,19 @@ plan_balanced_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int 
   }
   if (t == 0) seq_first[B] = carry_items;
   for (int it = carry_items + t; it < max_items; it += blockDim.x) *(int4*)(items + 4 * it) = make_int4(-1, 0, 0, 0);
+  // worker_first: items are ordered by worker; a worker without items gets an empty range
+  __syncthreads();
+  const int n_items = min(carry_items, max_items);
+  for (int it = t; it < n_items; it += blockDim.x) {
+    const int wk = items[4 * it + 3];
+    if (it == 0 || items[4 * (it - 1) + 3] != wk) worker_first[wk] = it;
+  }
+  __syncthreads();
+  if (t == 0) {
+    // unset entries still hold the item count; an entry may not exceed its successor
+    for (int w = n_workers - 1; w >= 0; --w)
+      if (worker_first[w] > worker_first[w + 1]) worker_first[w] = worker_first[w + 1];
+  }
 }
 
 }  // namespace
@@ -182,10 +199,10 @@ plan_balanced_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int 
 int ekv_launch_plan_balanced(const int32_t* seq_lens, int B, int tile_tokens, int n_workers,
                              int max_items, int32_t* items, int32_t* seq_first_item,
                              int32_t* worker_first, int32_t* zero_ints, int n_zero, long long max_len,
-                             int32_t* status, cudaStream_t st) {
+                             int32_t* status, int overhead_tiles, cudaStream_t st) {
   EKV_CUDA_OK(ekv_launch_pdl(plan_balanced_kernel, dim3(1), dim3(kPlanThreads), 0, st, seq_lens, B, tile_tokens,
                              n_workers, max_items, items, seq_first_item, worker_first, zero_ints, n_zero,
-                             max_len, status));
+                             max_len, status, overhead_tiles));
   EKV_CUDA_OK(cudaGetLastError());
   return ELITEKV_OK;
 }
@@ -210,13 +227,13 @@ extern "C" int elitekv_plan(const int32_t* seq_lens, int32_t B, int32_t tile_tok
 }
 
 extern "C" int elitekv_plan_workers(const int32_t* seq_lens, int32_t B, int32_t tile_tokens,
-                                    int32_t n_workers, int32_t max_items, int32_t* items,
-                                    int32_t* seq_first_item, int32_t* worker_first,
+                                    int32_t n_workers, int32_t item_overhead_tiles, int32_t max_items,
+                                    int32_t* items, int32_t* seq_first_item, int32_t* worker_first,
                                     elitekv_stream_t stream) {
   if (!seq_lens || !items || !seq_first_item || !worker_first || B <= 0 || tile_tokens <= 0 ||
-      n_workers <= 0 || max_items < B + n_workers)
+      n_workers <= 0 || max_items < B + n_workers || item_overhead_tiles < 0 || item_overhead_tiles > 64)
     return ELITEKV_ERR_INVALID_ARG;
   if ((uintptr_t)items & 15) return ELITEKV_ERR_INVALID_ARG;
   return ekv_launch_plan_balanced(seq_lens, B, tile_tokens, n_workers, max_items, items, seq_first_item,
-                                  worker_first, nullptr, 0, 0x7fffffffLL, nullptr, (cudaStream_t)stream);
+                                  worker_first, nullptr, 0, 0x7fffffffLL, nullptr, item_overhead_tiles, (cudaStream_t)stream);
 }

@@ -440,24 +440,29 @@ def _plan_cases():
             ([1024 + (7919 * i) % 31744 for i in range(64)], 64, 148)]
 
 
+@pytest.mark.parametrize("overhead", [0, 1, 3])
 @pytest.mark.parametrize("lens,tile,n_workers", _plan_cases())
-def test_worker_plan_structure(ek, lens, tile, n_workers):
-    """The persistent-worker plan: every sequence is partitioned into consecutive items that
-    start on tile boundaries; items are ordered by worker; worker w holds exactly the tiles
-    [w*quota, (w+1)*quota) of the batch's tile list; worker_first is monotone and covers all."""
+def test_worker_plan_structure(ek, lens, tile, n_workers, overhead):
+    """The persistent-worker plan.  The batch's tile list carries `overhead` empty tiles in front
+    of every non-empty sequence; worker w owns positions [w*total/n, (w+1)*total/n) of that list, n = min(workers, total).
+    Every sequence is partitioned into consecutive items that start on tile boundaries; items are
+    ordered by worker and lie inside their worker's range; worker_first is monotone and covers
+    all items; with overhead 0 every worker holds exactly the tiles of its range."""
     B = len(lens)
     t = torch.tensor(lens, dtype=torch.int32, device="cuda")
     max_items = B + n_workers
-    items, first, wfirst = ek.elitekv_plan_workers(t, tile, n_workers, max_items)
+    items, first, wfirst = ek.elitekv_plan_workers(t, tile, n_workers, max_items, overhead)
     torch.cuda.synchronize()
     items, first, wfirst = items.cpu().numpy(), first.cpu().numpy(), wfirst.cpu().numpy()
     n_items = int(first[-1])
     assert first[0] == 0 and n_items <= max_items
     assert np.all(items[n_items:, 0] == -1)
     tiles_of = [(n + tile - 1) // tile for n in lens]
-    total = sum(tiles_of)
-    quota = max(1, -(-total // n_workers))
-    g0 = np.concatenate([[0], np.cumsum(tiles_of)])
+    slots_of = [k + overhead if k else 0 for k in tiles_of]
+    total = max(1, sum(slots_of))
+    n_used = min(n_workers, total)
+    bound = [min(w, n_used) * total // n_used for w in range(n_workers + 1)]
+    g0 = np.concatenate([[0], np.cumsum(slots_of)])
     # sequences: consecutive, tile-aligned, complete
     for b, n in enumerate(lens):
         at = 0
@@ -471,13 +476,13 @@ def test_worker_plan_structure(ek, lens, tile, n_workers):
     for w_id in range(n_workers):
         for s, t0, cnt, wk in items[wfirst[w_id]:wfirst[w_id + 1]]:
             assert wk == w_id
-            ga = g0[s] + t0 // tile
-            gb = g0[s] + (t0 + cnt + tile - 1) // tile
-            assert w_id * quota <= ga and gb <= (w_id + 1) * quota
+            ga = g0[s] + overhead + t0 // tile
+            gb = g0[s] + overhead + (t0 + cnt + tile - 1) // tile
+            assert bound[w_id] <= ga and gb <= bound[w_id + 1]
             per_worker[w_id] += gb - ga
-    assert per_worker.sum() == total
-    want = np.clip(total - quota * np.arange(n_workers), 0, quota)
-    assert np.array_equal(per_worker, want)
+    assert per_worker.sum() == sum(tiles_of)
+    if overhead == 0 and sum(tiles_of) > 0:
+        assert np.array_equal(per_worker, np.diff(bound))
 
 
 # ------------------------------------------------------------------ comparator

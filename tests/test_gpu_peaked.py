@@ -56,11 +56,11 @@ def _moves_after_first_tile(ek, st, units):
     """Replays the lazy reference-maximum rule on the oracle's scores: number of (unit, item,
     tile > 0) triples in which the reference moves."""
     w = st.w
-    kernel, tile, n_workers, max_items = ek.elitekv_decode_plan_info(st.layer, st.cache, w.B)
+    kernel, tile, n_workers, max_items, overhead = ek.elitekv_decode_plan_info(st.layer, st.cache, w.B)
     if n_workers == 0:
         items, first = ek.elitekv_plan(st.lens_dev, tile, max_items)
     else:
-        items, first, _ = ek.elitekv_plan_workers(st.lens_dev, tile, n_workers, max_items)
+        items, first, _ = ek.elitekv_plan_workers(st.lens_dev, tile, n_workers, max_items, overhead)
     torch.cuda.synchronize()
     items, first = items.cpu().numpy(), first.cpu().numpy()
     idx = st.idx.numpy().astype(np.int64)

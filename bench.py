@@ -152,38 +152,38 @@ def cpu_baseline(w: gen.Workload, budget_s: float = 12.0):
                       f"{t_total:.2f} s of oracle time"}
 
 
-def config_of(w: gen.Workload, world: int, cache_bytes=None):
+def config_of(w: gen.Workload, world: int):
     c = {"workload": w.name, "n_h": w.n_h, "d_h": w.d_h, "r": w.r, "d_c": w.d_c,
          "batch_per_gpu": w.B, "context": w.ctx, "paged": w.paged,
          "l2": "256 MiB flush write before every timed step; cache larger than L2",
          "parallelism": f"replicas x{world} (independent sequences, no collective)",
          "streams": "append on a second stream beside absorb_query; joined before decode"}
-    if cache_bytes is not None:
-        c["cache_bytes_per_step"] = cache_bytes
     return c
 
 
 def run_reference(args, w: gen.Workload):
+    """The oracle as it stands on the host cores: every step is one whole sequence of the
+    workload (all heads, full context), the same sampling rule as `cpu_baseline`; a step of the
+    workload advances B sequences, so ms_per_step is the measured time times B."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     times = []
-    n_units = 4
     for i in range(args.warmup + args.steps):
-        dt, u, what = oracle_sample(w, n_units, seed_shift=i)
+        dt, u, what = oracle_sample(w, w.n_h, seed_shift=i)
         if i >= args.warmup:
-            times.append(dt / u)
-    per_unit = sum(times) / len(times)
-    value = 1.0 / (per_unit * w.n_h)     # sequences (tokens) per second for one layer
+            times.append(dt)
+    per_seq = sum(times) / len(times)
+    value = 1.0 / per_seq                # sequences (tokens) per second for one layer
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_unit * w.n_h * w.B * 1e3,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_seq * w.B * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
         "config": config_of(w, max(args.gpus, 1)),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
-                         "sample": f"each step {n_units} (sequence, head) units at full context, "
-                                   "time scaled to the whole batch"},
+                         "sample": f"each step one whole sequence (all {w.n_h} heads, full context) "
+                                   f"of the {w.B}; ms_per_step is that time x {w.B}"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -289,6 +289,116 @@ def step_serial(ek, layer, cache, d, ws, bufs):
 
 KERNELS_PER_STEP = 5   # append, absorb, plan, split-K attention, combine + up-projection
 
+SWEEP = ["7b-75pct-paged-b64-ragged", "13b-75pct-b32-ctx16384", "7b-50pct-b32-ctx8192",
+         "7b-75pct-b32-ctx8192", "7b-87.5pct-b32-ctx8192"]
+
+
+def sweep_entry(ek, w: gen.Workload, device, flush, steps: int = 10, n_check: int = 2):
+    """One of the other benchmark configurations: split-K kernel time and whole-step time on the
+    device, plus the float64 oracle timed on `n_check` (sequence, head) units of the SAME inputs
+    at full context (a cpu_baseline sample for this configuration) and the error of the library's
+    output rows against those oracle rows."""
+    layer, cache, lens, host, dev, ws, bufs, keep = build_workload(w, ek, device, 0)
+    for _ in range(3):
+        step(ek, layer, cache, dev, ws, bufs)
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in ev:
+        flush.fill_(1)
+        a.record()
+        step(ek, layer, cache, dev, ws, bufs)
+        b.record()
+    torch.cuda.synchronize()
+    step_ms = sum(a.elapsed_time(b) for a, b in ev) / steps
+    ek.elitekv_profile_enable(layer, True)
+    for _ in range(steps):
+        flush.fill_(1)
+        step(ek, layer, cache, dev, ws, bufs)
+    torch.cuda.synchronize()
+    kern_ms, kern_n = ek.elitekv_profile_collect(layer)
+    ek.elitekv_profile_enable(layer, False)
+    status = ek.elitekv_check_status(layer)
+    cache_bytes = int(lens.sum()) * 2 * w.cache_elems_per_token
+    kern_s = kern_ms / max(kern_n, 1) * 1e-3
+    peak, peak_kind = measured_peaks()
+    kernel_id = ek.elitekv_decode_plan_info(layer, cache, w.B)[0]
+    out = bufs["out"].float().cpu().double().numpy()
+    # ---- oracle on a few units of the same bytes
+    from oracle import elitekv_oracle as O
+    idx = gen.elite_index_sets(w).numpy().astype(np.int64)
+    W_uk, W_uv = keep[0].double().cpu().numpy(), keep[1].double().cpu().numpy()
+    g = np.random.default_rng(w.seed)
+    t_cpu, num, den, mx = 0.0, 0.0, 0.0, 0.0
+    for b in g.choice(w.B, size=min(n_check, w.B), replace=False).tolist():
+        n = int(lens[b])
+        k_e, c = gen.tokens(w, n - 1, device, stream=10 + b)
+        k_e = torch.cat([k_e.cpu(), host["k_e"][b:b + 1]]).double().numpy()
+        c = torch.cat([c.cpu(), host["c"][b:b + 1]]).double().numpy()
+        h = int(g.integers(w.n_h))
+        t0 = time.perf_counter()
+        want = O.decode_from_raw(host["q"][b].double().numpy(), n - 1, k_e, np.arange(n), c, W_uk, W_uv,
+                                 idx, w.d_h, base=w.rope_base, heads=[h])[0]
+        t_cpu += time.perf_counter() - t0
+        d = out[b, h] - want
+        num += float(d @ d)
+        den += float(want @ want)
+        mx = max(mx, float(np.max(np.abs(d))))
+    entry = {
+        "workload": w.name, "kernel": kernel_id, "kernel_us": kern_s * 1e6,
+        "achieved_gbs": cache_bytes / kern_s / 1e9, "frac": cache_bytes / kern_s / 1e9 / peak,
+        "peak_kind": f"of {peak_kind}", "cache_bytes_per_step": cache_bytes, "ms_per_step": step_ms,
+        "tokens_per_s": w.B / (step_ms * 1e-3), "status": status,
+        "parity": {"units": n_check, "rel_l2": (num / den) ** 0.5 if den else None, "max_abs": mx},
+        "cpu_baseline": {"value": 1.0 / (t_cpu / n_check * w.n_h), "unit": UNIT, "cores": oracle_threads(),
+                         "kind": "oracle", "sample": f"{n_check} (sequence, head) units at full context, "
+                                                     "scaled to all heads of a sequence"},
+    }
+    del layer, cache, dev, ws, bufs, keep
+    torch.cuda.empty_cache()
+    return entry
+
+
+def append_prefill(ek, device, flush, reps: int = 5):
+    """Cache append at prefill size on the 7B 75 % shape: T = 4096 tokens of one sequence, and
+    T = 32 x 4096 (a 4096-token prefill for each of 32 sequences).  Bytes = what the call must
+    read plus what it must write, 2 x cache row bytes per token."""
+    w = gen.SWEEP_75
+    out = {}
+    idx = gen.elite_index_sets(w)
+    W_uk, W_uv = gen.up_projections(w, device)
+    layer = ek.Layer(w.n_h, w.d_h, w.r, w.d_c, idx, W_uk, W_uv, 4096 + 1, rope_base=w.rope_base)
+    peak, peak_kind = measured_peaks()
+    for n_seq in (1, 32):
+        T = n_seq * 4096
+        rope_plane = torch.zeros((T, w.n_h * 2 * w.r), dtype=torch.bfloat16, device=device)
+        latent_plane = torch.zeros((T, w.d_c), dtype=torch.bfloat16, device=device)
+        cache = ek.make_cache(rope_plane, latent_plane, n_seqs=n_seq, max_ctx=4096)
+        k_e, c = gen.tokens(w, T, device, stream=77)
+        seq = torch.arange(n_seq, dtype=torch.int32, device=device).repeat_interleave(4096)
+        pos = torch.arange(4096, dtype=torch.int32, device=device).repeat(n_seq)
+        for _ in range(2):
+            ek.elitekv_append(layer, cache, k_e, c, seq, pos)
+        evs = []
+        for _ in range(reps):
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            ek.elitekv_append(layer, cache, k_e, c, seq, pos)
+            b.record()
+            evs.append((a, b))
+        torch.cuda.synchronize()
+        us = 1e3 * sum(a.elapsed_time(b) for a, b in evs) / reps
+        byts = 2 * T * 2 * w.cache_elems_per_token
+        out[f"T{T}"] = {"tokens": T, "us": us, "bytes_read_plus_written": byts,
+                        "gbs": byts / (us * 1e-6) / 1e9, "frac": byts / (us * 1e-6) / 1e9 / peak,
+                        "peak_kind": f"of {peak_kind}"}
+        del rope_plane, latent_plane, k_e, c, cache
+        torch.cuda.empty_cache()
+    assert ek.elitekv_check_status(layer) == 0
+    return out
+
+
+
 
 def run_gpu(args, w: gen.Workload):
     from paper_2503_01586_b200 import binding as ek
@@ -345,14 +455,28 @@ def run_gpu(args, w: gen.Workload):
     kern_ms, kern_n = ek.elitekv_profile_collect(layer)
     ek.elitekv_profile_enable(layer, False)
 
-    # ---- end to end: host buffers in, host result out, every step
-    h2d = sum(host[k].numel() * host[k].element_size() for k in host)
+    # ---- end to end: host buffers in, host result out, every step.  The step's six small input
+    #      arrays live in ONE pinned staging buffer (256-byte aligned sections) and cross in one
+    #      copy; the device-side tensors are views into its device twin.
+    order = ["k_e", "c", "q", "seq_id", "pos", "lens"]
+    offs, at = {}, 0
+    for k in order:
+        offs[k] = at
+        at = (at + host[k].numel() * host[k].element_size() + 255) & ~255
+    pack_host = torch.empty(at, dtype=torch.uint8).pin_memory()
+    pack_dev = torch.empty(at, dtype=torch.uint8, device=device)
+
+    def view(buf, k):
+        n = host[k].numel() * host[k].element_size()
+        return buf[offs[k]:offs[k] + n].view(host[k].dtype).view(host[k].shape)
+    for k in order:
+        view(pack_host, k).copy_(host[k])
+    staged = {k: view(pack_dev, k) for k in order}
+    h2d = pack_host.numel()
     d2h = bufs["out_host"].numel() * bufs["out_host"].element_size()
-    staged = {k: torch.empty_like(v, device=device) for k, v in host.items()}
 
     def e2e_step():
-        for k in host:
-            staged[k].copy_(host[k], non_blocking=True)
+        pack_dev.copy_(pack_host, non_blocking=True)
         step_serial(ek, layer, cache, staged, ws, bufs)
         bufs["out_host"].copy_(bufs["out"], non_blocking=True)
         torch.cuda.synchronize()
@@ -374,8 +498,7 @@ def run_gpu(args, w: gen.Workload):
         side.wait_stream(torch.cuda.current_stream())
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph, stream=side):
-            for k in host:
-                staged[k].copy_(host[k], non_blocking=True)
+            pack_dev.copy_(pack_host, non_blocking=True)
             step_serial(ek, layer, cache, staged, ws, bufs)
             bufs["out_host"].copy_(bufs["out"], non_blocking=True)
         for _ in range(3):
@@ -448,6 +571,26 @@ def run_gpu(args, w: gen.Workload):
         except torch.cuda.OutOfMemoryError:
             comparator = None
 
+    # ---- the other benchmark configurations and the prefill append (one GPU, rank 0 only)
+    sweep, prefill = None, None
+    if rank == 0 and world == 1 and not args.no_sweep:
+        del layer, cache, dev, ws, bufs, keep, staged, pack_dev
+        torch.cuda.empty_cache()
+        t_sweep = time.perf_counter()
+        prefill = append_prefill(ek, device, flush)
+        sweep = []
+        for name in SWEEP:
+            if name == w.name:
+                continue
+            if time.perf_counter() - t_sweep > args.sweep_budget_s:
+                sweep.append({"workload": name, "skipped": "sweep time budget spent"})
+                continue
+            try:
+                sweep.append(sweep_entry(ek, gen.CONFIGS[name], device, flush))
+            except torch.cuda.OutOfMemoryError:
+                sweep.append({"workload": name, "skipped": "out of device memory"})
+                torch.cuda.empty_cache()
+
     # ---- reduce over ranks
     total_ms, e2e_s, kern_ms = max_over_ranks(dist, [total_ms, e2e_s, kern_ms], device)
     if rank != 0:
@@ -464,7 +607,8 @@ def run_gpu(args, w: gen.Workload):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": config_of(w, world, cache_bytes),
+        "config": config_of(w, world),
+        "cache_bytes_per_step": cache_bytes,
         "hbm_gbs_whole_step": cache_bytes / (ms_per_step * 1e-3) / 1e9,
         "pct_of_nominal_8tbs_whole_step": 100.0 * cache_bytes / (ms_per_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
         "roofline": {"bound": "hbm", "kernel": "split-K decode attention", "achieved": achieved,
@@ -485,6 +629,8 @@ def run_gpu(args, w: gen.Workload):
         line["cpu_baseline"] = cpu_baseline(w)
     else:
         line["cpu_baseline"] = None
+    line["stages"]["append_prefill"] = prefill
+    line["sweep"] = sweep
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -498,6 +644,48 @@ TRAFFIC_BYTES_PER_LAUNCH = {
 }
 
 
+def run_dry(args, w: gen.Workload):
+    """The multi-rank plumbing of the GPU leg on CPU: rank environment, process group (gloo),
+    barrier, max over ranks, aggregate value, one JSON line from rank 0."""
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo", rank=rank, world_size=world)
+    ms = 1.0 + rank                         # the slowest rank decides
+    (ms_max,) = max_over_ranks(dist if world > 1 else None, [ms], "cpu")
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "n_gpus": world, "ms_per_step": ms_max,
+                          "value": aggregate_value(world, w.B, ms_max), "dry_run": True}))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def launch_replicas(args) -> int:
+    """`bench.py --gpus N` started plainly (no torchrun): starts N copies of this script, one per
+    GPU, each with the rank environment torchrun would give it; rank 0 prints the JSON line.
+    Fails loudly when the machine has fewer than N devices or a replica fails."""
+    import socket
+    n = args.gpus
+    if args.impl != "reference" and not args.dry_run_ranks:
+        have = torch.cuda.device_count()
+        if have < n:
+            raise SystemExit(f"bench.py --gpus {n}: only {have} CUDA device(s) visible")
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], env=env))
+    codes = [p.wait() for p in procs]
+    if any(codes):
+        raise SystemExit(f"bench.py --gpus {n}: replica exit codes {codes}")
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -506,12 +694,26 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=gen.LLAMA7B_75.name, choices=sorted(gen.CONFIGS))
     ap.add_argument("--kernel", type=int, default=0,
-                    help="split-K kernel: 0 auto, 1 CUDA-core, 2 tcgen05 single block, 3 tcgen05 pair")
+                    help="split-K kernel: 0 auto, 1 CUDA-core, 2 tcgen05 two-pass, 3 tcgen05 resident tile")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-comparator", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true",
+                    help="skip the other configurations and the prefill-append measurement")
+    ap.add_argument("--sweep-budget-s", type=float, default=150.0)
+    ap.add_argument("--dry-run-ranks", action="store_true",
+                    help="launcher check without a GPU: every rank joins a gloo group, takes part in the "
+                         "max-over-ranks reduction of a dummy timing and rank 0 prints a JSON line")
     args = ap.parse_args()
     w = gen.CONFIGS[args.workload]
-    if args.impl == "reference":
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        launch_replicas(args)
+        return
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world != max(args.gpus, 1):
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={world}")
+    if args.dry_run_ranks:
+        run_dry(args, w)
+    elif args.impl == "reference":
         run_reference(args, w)
     else:
         run_gpu(args, w)

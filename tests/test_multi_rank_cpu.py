@@ -37,11 +37,50 @@ def test_aggregate_value_counts_every_replica():
     assert bench.aggregate_value(8, 16, 0.5) == 8 * 32000.0
 
 
-def test_reference_arm_config_matches_the_gpu_arm():
+def test_both_arms_name_the_workload_the_same_way():
+    """`config` is a function of the workload and the replica count only (the measured cache
+    bytes live beside it, not inside), so the two arms of one run print equal configs."""
     sys.path.insert(0, ROOT)
     import bench
     from paper_2503_01586_b200 import inputs as gen
     a = bench.config_of(gen.LLAMA7B_75, 1)
-    b = bench.config_of(gen.LLAMA7B_75, 1, cache_bytes=123)
-    b.pop("cache_bytes_per_step")
-    assert a == b and a["workload"] == "7b-75pct-b16-ctx4096"
+    assert a == bench.config_of(gen.LLAMA7B_75, 1) and a["workload"] == "7b-75pct-b16-ctx4096"
+    assert "cache_bytes_per_step" not in a
+
+
+def _run_bench(*argv, env=None):
+    import json
+    import subprocess
+    e = dict(os.environ)
+    for k in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT"):
+        e.pop(k, None)
+    e.update(env or {})
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), *argv], env=e,
+                       capture_output=True, text=True, timeout=300)
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    return r.returncode, [json.loads(l) for l in lines], r.stderr
+
+
+def test_gpus_flag_starts_one_replica_per_rank_by_itself():
+    """`bench.py --gpus 2` without torchrun: the script starts its own two ranks (gloo here, no
+    GPU), the slowest rank's time decides, the value counts both replicas and exactly one JSON
+    line comes out, saying n_gpus 2."""
+    code, lines, err = _run_bench("--gpus", "2", "--dry-run-ranks")
+    assert code == 0, err
+    assert len(lines) == 1
+    assert lines[0]["n_gpus"] == 2 and lines[0]["ms_per_step"] == 2.0
+    assert lines[0]["value"] == 2 * 16 / 2.0e-3
+
+
+def test_gpus_flag_must_agree_with_the_launcher_environment():
+    """Under a launcher that already set WORLD_SIZE the flag must say the same number."""
+    code, lines, err = _run_bench("--gpus", "4", "--dry-run-ranks",
+                                  env={"WORLD_SIZE": "1", "RANK": "0", "LOCAL_RANK": "0"})
+    assert code != 0 and not lines and "WORLD_SIZE" in err
+
+
+def test_gpus_flag_fails_loudly_without_enough_devices():
+    if torch.cuda.is_available() and torch.cuda.device_count() >= 2:
+        return
+    code, lines, err = _run_bench("--gpus", "2", "--steps", "1", "--warmup", "1", "--no-sweep")
+    assert code != 0 and not lines and "CUDA device" in err

@@ -1,7 +1,7 @@
 // Fused RoPE + cache append (Section 3.1: the rotated elite chunks of the new token enter the
 // cache once; Section 3.2: the shared latent row is stored beside them).
 //
-// One thread block per token (grid-stride, two tokens in flight per block).  Both rows move with
+// One thread block per token (grid-stride, four tokens in flight per block).  Both rows move with
 // 16-byte accesses: a work item is either 8 latent elements or 4 rope pairs.  For the pairs the
 // thread reads the 4 un-rotated pairs and their 4 chunk ids, looks up (cos, sin) of
 // pos*theta_{idx[h][j]} and writes the 4 rotated pairs in one store.  Every product and sum is
@@ -48,6 +48,8 @@ __device__ __forceinline__ uint32_t rotate_pair(uint32_t raw, float2 w) {
   return *(const uint32_t*)&y;
 }
 
+constexpr int kTok = 4;      // tokens a block works on at once (independent 16-byte loads per thread)
+
 template <bool kVec>
 __global__ void __launch_bounds__(256)
 append_kernel(const AppendArgs a) {
@@ -55,19 +57,22 @@ append_kernel(const AppendArgs a) {
   const int n_vec = a.d_c >> 3;
   const int n_rv = kVec ? n_pairs >> 2 : 0;
   const int n_items = n_vec + n_rv;
-  for (long long t0 = blockIdx.x; t0 < a.T; t0 += 2ll * gridDim.x) {
-    long long tk[2] = {t0, t0 + gridDim.x};
-    long long row[2];
-    int p[2] = {0, 0};
+  for (long long t0 = blockIdx.x; t0 < a.T; t0 += (long long)kTok * gridDim.x) {
+    long long tk[kTok], row[kTok];
+    int p[kTok];
 #pragma unroll
-    for (int e = 0; e < 2; ++e) row[e] = tk[e] < a.T ? append_row(a, tk[e], &p[e]) : -1;
+    for (int e = 0; e < kTok; ++e) {
+      tk[e] = t0 + (long long)e * gridDim.x;
+      p[e] = 0;
+      row[e] = tk[e] < a.T ? append_row(a, tk[e], &p[e]) : -1;
+    }
     for (int v = threadIdx.x; v < n_items; v += blockDim.x) {
-      // loads of both tokens first, then the arithmetic and the stores
-      uint4 x[2];
-      int4 id[2];
+      // loads of all tokens first, then the arithmetic and the stores
+      uint4 x[kTok];
+      int4 id[kTok];
       const bool lat = v < n_vec;
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
+      for (int e = 0; e < kTok; ++e) {
         if (row[e] < 0) continue;
         if (lat) {
           x[e] = __ldcs(a.c + tk[e] * n_vec + v);
@@ -77,7 +82,7 @@ append_kernel(const AppendArgs a) {
         }
       }
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
+      for (int e = 0; e < kTok; ++e) {
         if (row[e] < 0) continue;
         if (lat) {
           a.latent[row[e] * n_vec + v] = x[e];
@@ -94,7 +99,7 @@ append_kernel(const AppendArgs a) {
     }
     if (!kVec) {
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
+      for (int e = 0; e < kTok; ++e) {
         if (row[e] < 0) continue;
         const bf162* ksrc = a.k_e + tk[e] * n_pairs;
         bf162* kdst = a.rope + row[e] * n_pairs;
@@ -131,8 +136,8 @@ int ekv_launch_append(const elitekv_layer* L, const elitekv_cache* cache, const 
   a.half = L->d_h / 2;
   a.max_pos = L->max_pos;
   a.status = L->d_status;
-  const long long pairs_of_blocks = (T + 1) / 2;
-  long long blocks = pairs_of_blocks < (long long)L->sm_count * 8 ? pairs_of_blocks : (long long)L->sm_count * 8;
+  const long long groups = (T + kTok - 1) / kTok;
+  long long blocks = groups < (long long)L->sm_count * 8 ? groups : (long long)L->sm_count * 8;
   // 16-byte rope accesses need rows of whole 4-pair groups (the buffers themselves are 16-byte
   // aligned: checked at the entry point)
   if ((L->n_h * L->r) % 4 == 0 && L->r > 0)

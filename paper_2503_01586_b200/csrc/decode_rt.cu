@@ -31,8 +31,7 @@
 // item each block writes its half of (acc) and block 0 writes (m, l).
 //
 // Roles per block (256 threads):
-//   warps 0, 2   TMA producers (units dealt alternately); warp 0 also loads the query half; both
-//                pull the next tiles into L2 ahead of time
+//   warps 0, 2   TMA producers (units dealt alternately); warp 0 also loads the query half
 //   warp 1       TMEM owner and MMA issuer (warp-uniform, instructions under an elected lane,
 //                as many landed units as possible per election; slot and phase counters advance
 //                incrementally so that the descriptor words stay in uniform registers)
@@ -125,7 +124,7 @@ __device__ __forceinline__ bool rt_wait(uint32_t bar, uint32_t parity, volatile 
 template <int R2>
 __global__ void __launch_bounds__(kRtThreads, 1)
 decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_constant__ CUtensorMap map_q,
-                 const __grid_constant__ CUtensorMap map_pf, const RtArgs a) {
+                 const RtArgs a) {
   constexpr int N = kHeads;
   constexpr int LPT = R2 / 8;           // 16-byte loads per lane per rope row (row = 32 * R2 bf16)
   extern __shared__ unsigned char smem_raw[];
@@ -155,7 +154,6 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   if (threadIdx.x == 32) {
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_lat) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_q) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&map_pf) : "memory");
   }
   if (threadIdx.x == 0) {
     for (int i = 0; i < kMaxRing; ++i) {
@@ -233,18 +231,6 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
             tma_load_2d_hint(smem_u32(s_q + kc * N * 128), &map_q, (int)rank * DH + kc * 64, seq * N, qb, pol_keep);
         }
         __syncwarp();
-        // The ring holds only half a tile beyond the resident one, so a unit's refill can start
-        // only when the value product has released its slot, and would then wait a full HBM
-        // latency.  The producers therefore pull every tile into L2 one tile ahead
-        // ([64 tokens x 256 coordinates] boxes, no shared memory involved): the refill is an
-        // L2 hit, and HBM keeps streaming while the block is busy with the softmax.
-        auto prefetch_tile = [&](int tile) {
-          if (tile < n_tiles && elect_one()) {
-            const int row = (int)tile_row(seq, tok0 + tile * kT, false);
-            for (int x = prod * 256; x < DH; x += 512) tma_prefetch_2d(&map_pf, (int)rank * DH + x, row);
-          }
-          __syncwarp();
-        };
         bool ok = true;
         for (int tile = 0; tile < n_tiles && ok; ++tile) {
           const int row = (int)tile_row(seq, tok0 + tile * kT, prod == 0 && lane == 0);
@@ -263,9 +249,6 @@ decode_rt_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
             }
             if (++slot == (unsigned)NR) { slot = 0; par ^= 1; }
           }
-          // behind this tile's own loads, so that a prefetch never delays data that is waited for
-          if (tile == 0) prefetch_tile(1);
-          prefetch_tile(tile + 2);
         }
         if (!ok) break;
       }
@@ -717,8 +700,7 @@ cudaLaunchAttribute rt_cluster_attr() {
 }
 
 template <int R2>
-int rt_launch(const CUtensorMap& m_lat, const CUtensorMap& m_q, const CUtensorMap& m_pf,
-              const RtArgs& a,
+int rt_launch(const CUtensorMap& m_lat, const CUtensorMap& m_q, const RtArgs& a,
               int n_workers, int smem, cudaStream_t st) {
   EKV_CUDA_OK(cudaFuncSetAttribute(decode_rt_kernel<R2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
   cudaLaunchConfig_t cfg = {};
@@ -732,7 +714,7 @@ int rt_launch(const CUtensorMap& m_lat, const CUtensorMap& m_q, const CUtensorMa
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  EKV_CUDA_OK(cudaLaunchKernelEx(&cfg, decode_rt_kernel<R2>, m_lat, m_q, m_pf, a));
+  EKV_CUDA_OK(cudaLaunchKernelEx(&cfg, decode_rt_kernel<R2>, m_lat, m_q, a));
   EKV_CUDA_OK(cudaGetLastError());
   return ELITEKV_OK;
 }
@@ -800,10 +782,9 @@ int ekv_launch_decode_rt(const elitekv_layer* L, const elitekv_cache* cache, con
   const unsigned long long rows =
       cv.page_table ? (unsigned long long)cv.num_pages << cv.page_shift : (unsigned long long)cv.max_ctx * cv.n_seqs;
   if (rows >= (1ull << 31)) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
-  CUtensorMap m_lat, m_q, m_pf;
+  CUtensorMap m_lat, m_q;
   int rc = make_map(&m_lat, cache->latent, rows, L->d_c, kT);
   if (rc == ELITEKV_OK) rc = make_map(&m_q, q_abs, (unsigned long long)B * L->n_h, L->d_c, kHeads);
-  if (rc == ELITEKV_OK) rc = make_map_plain(&m_pf, cache->latent, rows, L->d_c, 256, kT);
   if (rc != ELITEKV_OK) return rc;
   RtArgs a;
   a.items = ws.items;
@@ -824,8 +805,8 @@ int ekv_launch_decode_rt(const elitekv_layer* L, const elitekv_cache* cache, con
   a.scale_log2e = L->scale * 1.4426950408889634f;
   const int smem = rt_layout(L->d_c, a.n_ring).total;
   switch (2 * L->r) {
-    case 8: return rt_launch<8>(m_lat, m_q, m_pf, a, ws.n_workers, smem, st);
-    case 16: return rt_launch<16>(m_lat, m_q, m_pf, a, ws.n_workers, smem, st);
-    default: return rt_launch<32>(m_lat, m_q, m_pf, a, ws.n_workers, smem, st);
+    case 8: return rt_launch<8>(m_lat, m_q, a, ws.n_workers, smem, st);
+    case 16: return rt_launch<16>(m_lat, m_q, a, ws.n_workers, smem, st);
+    default: return rt_launch<32>(m_lat, m_q, a, ws.n_workers, smem, st);
   }
 }

@@ -365,22 +365,6 @@ static inline int make_map_f32_3d(CUtensorMap* m, const void* ptr, unsigned long
   return r == CUDA_SUCCESS ? ELITEKV_OK : ELITEKV_ERR_CUDA;
 }
 
-// 2-D bf16 tensor [rows][cols] (cols contiguous), box [box_rows][box_cols], no swizzle: for L2
-// prefetches, which have no shared-memory layout to respect and can use wide boxes
-static inline int make_map_plain(CUtensorMap* m, const void* ptr, unsigned long long rows, unsigned long long cols,
-                                 unsigned box_cols, unsigned box_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return ELITEKV_ERR_CUDA;
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {cols * sizeof(bf16)};
-  cuuint32_t box[2] = {box_cols, box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? ELITEKV_OK : ELITEKV_ERR_CUDA;
-}
-
 // 2-D bf16 tensor [rows][cols] (cols contiguous), box [box_rows][64], 128-byte swizzle
 static inline int make_map(CUtensorMap* m, const void* ptr, unsigned long long rows, unsigned long long cols, unsigned box_rows) {
   EncodeTiledFn fn = encode_fn();

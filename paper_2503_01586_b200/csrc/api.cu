@@ -14,6 +14,20 @@ int select_kernel(const elitekv_layer* L, const elitekv_cache* cache) {
   if (L->decode_kernel == 3) return rt ? 3 : -1;
   if (L->decode_kernel == 2) return tc ? 2 : -1;
   if (L->decode_kernel == 1) return ekv_generic_supported(L) ? 1 : -1;
+  // Choice by shape when both tensor-core kernels cover the layer (measured on B200): the
+  // resident-tile kernel has the lower fixed cost and wins on batches of up to a few hundred
+  // thousand cached tokens at d_c = 1536 (80 us against 90 us at 16 x 4096); its per-tile chain
+  // (exchange between the two blocks of a pair, softmax, value product) makes it the slower one
+  // on long streams (0.73 against 0.82 of the copy bandwidth on the 4.6 GB ragged batch) and
+  // at narrow latents (d_c = 768).  Lengths live on the device, so the capacity of the cache
+  // stands in for them.
+  if (rt && tc) {
+    long long capacity = 0;
+    if (cache) capacity = cache->page_table ? (long long)cache->num_pages * cache->page_size
+                                            : (long long)cache->max_ctx * cache->n_seqs;
+    const bool small = cache == nullptr || capacity <= 200000;
+    return (small && L->d_c >= 1024) ? 3 : 2;
+  }
   if (rt) return 3;
   if (tc) return 2;
   return ekv_generic_supported(L) ? 1 : -1;

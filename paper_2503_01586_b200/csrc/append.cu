@@ -1,7 +1,7 @@
 // Fused RoPE + cache append (Section 3.1: the rotated elite chunks of the new token enter the
 // cache once; Section 3.2: the shared latent row is stored beside them).
 //
-// One thread block per token (grid-stride, four tokens in flight per block).  Both rows move with
+// One thread block per token (grid-stride, two tokens in flight per block).  Both rows move with
 // 16-byte accesses: a work item is either 8 latent elements or 4 rope pairs.  For the pairs the
 // thread reads the 4 un-rotated pairs and their 4 chunk ids, looks up (cos, sin) of
 // pos*theta_{idx[h][j]} and writes the 4 rotated pairs in one store.  Every product and sum is
@@ -48,7 +48,9 @@ __device__ __forceinline__ uint32_t rotate_pair(uint32_t raw, float2 w) {
   return *(const uint32_t*)&y;
 }
 
-constexpr int kTok = 4;      // tokens a block works on at once (independent 16-byte loads per thread)
+constexpr int kTok = 2;      // tokens a block works on at once (independent 16-byte loads per thread;
+                             // four were measured slower: the registers cost more occupancy than the
+                             // extra loads in flight bring)
 
 template <bool kVec>
 __global__ void __launch_bounds__(256)

@@ -12,6 +12,7 @@
 namespace {
 
 constexpr int kPlanThreads = 256;
+constexpr int kPlanStage = 4096;       // items whose worker ids are staged in shared memory
 
 // exclusive scan over the block (warp shuffles + one shared array of warp totals)
 __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int* total) {
@@ -116,6 +117,7 @@ plan_balanced_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int 
                      long long max_len, int32_t* status, int overhead) {
   __shared__ int warp_tot[kPlanThreads / 32];
   __shared__ long long s_total;
+  __shared__ short s_wk[kPlanStage];       // worker of each item (n_workers < 32768)
   const int t = threadIdx.x;
   ekv_pdl_wait();         // earlier kernels may still read the arrays written here
   ekv_pdl_trigger();
@@ -135,12 +137,8 @@ plan_balanced_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int 
   const long long nw = total < n_workers ? total : n_workers;
   auto bound = [&](long long w) -> long long { return w * total / nw; };
   auto owner = [&](long long g) -> int { return (int)(((g + 1) * nw - 1) / total); };
-  // pass 1: count items to know n_items (default of worker_first)
   int carry_tiles = 0, carry_items = 0;
-  // per-thread record of its sequences is recomputed in pass 2; B is small compared to the block
-  for (int pass = 0; pass < 2; ++pass) {
-    carry_tiles = 0;
-    carry_items = 0;
+  {
     for (int b0 = 0; b0 < B; b0 += blockDim.x) {
       const int b = b0 + t;
       int n = 0, tiles = 0;
@@ -158,7 +156,7 @@ plan_balanced_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int 
       }
       int chunk_items;
       const int first = carry_items + block_exclusive_scan(pieces, warp_tot, &chunk_items);
-      if (pass == 1 && b < B) {
+      if (b < B) {
         seq_first[b] = first;
         for (int j = 0; j < pieces; ++j) {
           const long long ga = max((long long)g0 + overhead, bound(w0 + j));
@@ -167,30 +165,41 @@ plan_balanced_kernel(const int32_t* __restrict__ seq_lens, int B, int tile, int 
           const int tok1 = min((int)(gb - g0 - overhead) * tile, n);
           const int it = first + j;
           if (it < max_items) *(int4*)(items + 4 * it) = make_int4(b, tok0, tok1 - tok0, w0 + j);
+          if (it < kPlanStage) s_wk[it] = (short)(w0 + j);
         }
       }
       carry_tiles += chunk_tiles;
       carry_items += chunk_items;
     }
-    if (pass == 0) {
-      for (int w = t; w <= n_workers; w += blockDim.x) worker_first[w] = carry_items;
-      __syncthreads();
-    }
   }
   if (t == 0) seq_first[B] = carry_items;
   for (int it = carry_items + t; it < max_items; it += blockDim.x) *(int4*)(items + 4 * it) = make_int4(-1, 0, 0, 0);
-  // worker_first: items are ordered by worker; a worker without items gets an empty range
+  // worker_first[w] = number of items of workers below w (items are ordered by worker; a worker
+  // without items gets an empty range).  The worker ids of up to kPlanStage items are kept in
+  // shared memory while they are written, so that this is a binary search per worker instead of
+  // a second trip to global memory.
   __syncthreads();
   const int n_items = min(carry_items, max_items);
-  for (int it = t; it < n_items; it += blockDim.x) {
-    const int wk = items[4 * it + 3];
-    if (it == 0 || items[4 * (it - 1) + 3] != wk) worker_first[wk] = it;
-  }
-  __syncthreads();
-  if (t == 0) {
-    // unset entries still hold the item count; an entry may not exceed its successor
-    for (int w = n_workers - 1; w >= 0; --w)
-      if (worker_first[w] > worker_first[w + 1]) worker_first[w] = worker_first[w + 1];
+  if (n_items <= kPlanStage) {
+    for (int w = t; w <= n_workers; w += blockDim.x) {
+      int lo = 0, hi = n_items;              // first item whose worker is >= w
+      while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (s_wk[mid] < w) lo = mid + 1; else hi = mid;
+      }
+      worker_first[w] = lo;
+    }
+  } else {
+    for (int w = t; w <= n_workers; w += blockDim.x) worker_first[w] = n_items;
+    __syncthreads();
+    for (int it = t; it < n_items; it += blockDim.x) {
+      const int wk = items[4 * it + 3];
+      if (it == 0 || items[4 * (it - 1) + 3] != wk) worker_first[wk] = it;
+    }
+    __syncthreads();
+    if (t == 0)       // unset entries still hold the item count; an entry may not exceed its successor
+      for (int w = n_workers - 1; w >= 0; --w)
+        if (worker_first[w] > worker_first[w + 1]) worker_first[w] = worker_first[w + 1];
   }
 }
 

@@ -636,11 +636,10 @@ def run_gpu(args, w: gen.Workload):
         dist.destroy_process_group()
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one split-K launch from the ncu capture
-# summarised under profiles/ (None until a capture of the current kernel exists).
+# dram__bytes_read.sum + dram__bytes_write.sum of one split-K launch on the named workload, from an
+# ncu capture of the kernel that serves it (None where no capture of the current kernel exists).
 TRAFFIC_BYTES_PER_LAUNCH = {
-    # profiles/decode_tc_kernel__7b-75pct-b16-ctx4096.md: 274.9 MB read + 4.2 MB written
-    "7b-75pct-b16-ctx4096": 279057408,
+    "7b-75pct-b16-ctx4096": 270263040 + 4182528,     # resident-tile kernel, one launch
 }
 
 

@@ -178,6 +178,34 @@ def append_expected(rope_plane_bits, latent_plane_bits, k_e_bits, c_bits, seq_id
     return rope, lat
 
 
+def project_tokens(x, W_ke, W_down):
+    """The projections that feed the cache (Section 3.2): for hidden states x [T][d],
+    k_e = x W^k_e  (W^k_e [d][n_h*2r]: the columns of W^k that belong to the elite chunks, head
+    by head, Eq. 2) and c = x A^kv (A^kv = W_down [d][d_c]).  Returns float64
+    (k_e [T][n_h*2r], c [T][d_c]), not rounded."""
+    x = np.asarray(x, dtype=F64)
+    return x @ np.asarray(W_ke, dtype=F64), x @ np.asarray(W_down, dtype=F64)
+
+
+def project_append_expected(rope_plane_bits, latent_plane_bits, x, W_ke, W_down, seq_id, pos, idx,
+                            d_h, *, base=10000.0, max_ctx=None, page_table=None, page_size=64):
+    """Projection fused with the append: the float64 projections of `project_tokens`, the elite
+    chunks rotated at the token's position (Section 3.1), every stored element rounded ONCE to
+    bf16.  Returns copies of the planes (uint16 bit patterns) plus the float64 rows before
+    rounding (rope rows [T][n_h*2r], latent rows [T][d_c]) for tolerance checks."""
+    rope = np.array(rope_plane_bits, dtype=np.uint16, copy=True)
+    lat = np.array(latent_plane_bits, dtype=np.uint16, copy=True)
+    idx = np.asarray(idx, dtype=np.int64)
+    n_h, r = idx.shape
+    k_e, c = project_tokens(x, W_ke, W_down)
+    T = k_e.shape[0]
+    rows = rotate_elite_keys(k_e.reshape(T, n_h, r, 2), pos, idx, d_h, base).reshape(T, n_h * 2 * r)
+    slot = token_slot(seq_id, pos, max_ctx=max_ctx, page_table=page_table, page_size=page_size)
+    rope[slot] = f64_to_bf16_bits(rows)
+    lat[slot] = f64_to_bf16_bits(c)
+    return rope, lat, rows, c
+
+
 # --------------------------------------------------------------------------------------------
 # Query side
 # --------------------------------------------------------------------------------------------

@@ -339,3 +339,62 @@ def test_theta_schedule():
     assert th[0] == 1.0 and np.all(np.diff(th) < 0)
     assert abs(th[32] - 10000.0 ** -0.5) < 1e-15
     assert abs(th[63] - 10000.0 ** (-126 / 128)) < 1e-18
+
+
+def test_projection_with_selector_weights_reduces_to_the_plain_append():
+    """Fused projection + append (Section 3.2 projections, Section 3.1 rotation).  With weights
+    that merely SELECT coordinates of x (W^k_e and A^kv columns of the identity) the projection is
+    exact, so the fused result must equal, bit for bit, the plain append of those coordinates,
+    which is pinned on its own above; a swapped weight, a transposed product or a rotation applied
+    to the latent part would all break the equality."""
+    g = np.random.default_rng(31)
+    n_h, d_h, r, d_c = 3, 16, 2, 8
+    rope_w = n_h * 2 * r
+    d = rope_w + d_c + 5                       # five hidden coordinates feed nothing
+    idx = np.stack([g.permutation(d_h // 2)[:r] for _ in range(n_h)])
+    T = 9
+    xb = O.f64_to_bf16_bits(g.standard_normal((T, d)))
+    x = O.bf16_bits_to_f64(xb)
+    perm = g.permutation(d)
+    W_ke = np.zeros((d, rope_w)); W_ke[perm[:rope_w], np.arange(rope_w)] = 1.0
+    W_down = np.zeros((d, d_c)); W_down[perm[rope_w:rope_w + d_c], np.arange(d_c)] = 1.0
+    seq = g.integers(0, 2, T); pos = g.permutation(20)[:T]
+    rope0 = g.integers(0, 2 ** 15, (40, rope_w)).astype(np.uint16)
+    lat0 = g.integers(0, 2 ** 15, (40, d_c)).astype(np.uint16)
+    got_r, got_l, rows, c = O.project_append_expected(rope0, lat0, x, W_ke, W_down, seq, pos, idx, d_h, max_ctx=20)
+    k_bits = xb[:, perm[:rope_w]].reshape(T, n_h, r, 2)
+    c_bits = xb[:, perm[rope_w:rope_w + d_c]]
+    want_r, want_l = O.append_expected(rope0, lat0, k_bits, c_bits, seq, pos, idx, d_h, max_ctx=20)
+    assert np.array_equal(got_r, want_r) and np.array_equal(got_l, want_l)
+
+
+def test_projection_properties_that_need_no_second_implementation():
+    """Linearity in x before rounding; a token at position 0 is stored un-rotated; rotation keeps
+    the norm of every projected pair; the latent part ignores the position."""
+    g = np.random.default_rng(32)
+    n_h, d_h, r, d_c, d, T = 2, 8, 2, 4, 6, 5
+    idx = np.array([[0, 3], [2, 1]])
+    W_ke = g.standard_normal((d, n_h * 2 * r)); W_down = g.standard_normal((d, d_c))
+    x1, x2 = g.standard_normal((T, d)), g.standard_normal((T, d))
+    seq = np.zeros(T, dtype=np.int64); pos = np.array([0, 3, 7, 1, 5])
+    z = np.zeros((8, n_h * 2 * r), dtype=np.uint16), np.zeros((8, d_c), dtype=np.uint16)
+    _, _, r1, c1 = O.project_append_expected(*z, x1, W_ke, W_down, seq, pos, idx, d_h, max_ctx=8)
+    _, _, r2, c2 = O.project_append_expected(*z, x2, W_ke, W_down, seq, pos, idx, d_h, max_ctx=8)
+    _, _, r3, c3 = O.project_append_expected(*z, 2 * x1 - 3 * x2, W_ke, W_down, seq, pos, idx, d_h, max_ctx=8)
+    assert np.allclose(r3, 2 * r1 - 3 * r2, atol=1e-12) and np.allclose(c3, 2 * c1 - 3 * c2, atol=1e-12)
+    # hand-evaluated entries: token 0 sits at position 0 (identity rotation)
+    for col in range(n_h * 2 * r):
+        assert abs(r1[0, col] - sum(x1[0, k] * W_ke[k, col] for k in range(d))) < 1e-12
+    for col in range(d_c):
+        assert abs(c1[2, col] - sum(x1[2, k] * W_down[k, col] for k in range(d))) < 1e-12
+    # norms of pairs survive the rotation; other positions change the rope row, not the latent
+    k_plain = (x1 @ W_ke).reshape(T, n_h * r, 2)
+    assert np.allclose(np.linalg.norm(r1.reshape(T, n_h * r, 2), axis=-1), np.linalg.norm(k_plain, axis=-1))
+    _, _, r4, c4 = O.project_append_expected(*z, x1, W_ke, W_down, seq, (pos + 2) % 8, idx, d_h, max_ctx=8)
+    assert np.allclose(c4, c1) and not np.allclose(r4[1:], r1[1:])
+    # quarter turn: theta_0 = 1, so position p = pi/2 cannot be hit by an integer; use the angle law
+    # instead: rotating by positions 3 and then reading the pair's angle gives atan2 shifted by 3*theta
+    th = O.rope_theta(d_h)[idx.reshape(-1)]
+    a_plain = np.arctan2(k_plain[1, :, 1], k_plain[1, :, 0])
+    a_rot = np.arctan2(r1.reshape(T, n_h * r, 2)[1, :, 1], r1.reshape(T, n_h * r, 2)[1, :, 0])
+    assert np.allclose(np.exp(1j * (a_rot - a_plain)), np.exp(1j * 3 * th))

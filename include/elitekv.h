@@ -78,6 +78,12 @@ typedef struct {
                                  values); 3 = tcgen05 kernel that keeps a 64-token tile
                                  resident in shared memory between the two products.  2 and 3
                                  fail with UNSUPPORTED_SHAPE when the shape is not covered.    */
+  /* Only for elitekv_project_append (all three 0 / NULL otherwise): the projections that make
+   * the cache row of a token from its hidden state x (Section 3.2, Eq. 2). */
+  int32_t d;                  /* model width                                                   */
+  const void* W_ke;           /* bf16 [d][n_h*2r]  columns of W^k of the elite chunks, head by
+                                 head in the order of elite_idx, (even, odd) inside a chunk    */
+  const void* W_down;         /* bf16 [d][d_c]     A^kv                                        */
 } elitekv_params;
 
 /* The two cache planes.  Contiguous (page_table == NULL): sequence s, position p live in row
@@ -114,6 +120,19 @@ int elitekv_layer_destroy(elitekv_layer* layer);
 int elitekv_append(const elitekv_layer* layer, const elitekv_cache* cache, const void* k_e,
                    const void* c, const int32_t* seq_id, const int32_t* pos, int64_t T,
                    elitekv_stream_t stream);
+
+/* Projection fused with the cache append (Section 3.2: k_e = x W^k_e, c = x A^kv; Section 3.1:
+ * rotation of the elite chunks at the token's position): what elitekv_append does, starting
+ * from the hidden states, in one kernel -- x [T][d] . [W^k_e | A^kv] on the tensor cores (fp32
+ * accumulation), rotation and the single rounding to bf16 in the epilogue, rows written straight
+ * into the cache.  k_e and c never exist in memory.
+ *   x bf16 [T][d], 16-byte aligned;  seq_id, pos int32 [T] as for elitekv_append.
+ * Needs a layer created with d, W_ke and W_down; d a multiple of 64 and both n_h*2r and d_c
+ * multiples of 128 (ELITEKV_ERR_UNSUPPORTED_SHAPE otherwise).  Stored values differ from
+ * elitekv_append(bf16(x W^k_e), bf16(x A^kv)) by the intermediate rounding only. */
+int elitekv_project_append(const elitekv_layer* layer, const elitekv_cache* cache, const void* x,
+                           const int32_t* seq_id, const int32_t* pos, int64_t T,
+                           elitekv_stream_t stream);
 
 /* Query preparation (score equation of Section 3.1; absorption of B^k, Section 5).
  *   q      bf16  [B][n_h][d_h]  un-rotated queries,  q_pos int32 [B]

@@ -37,7 +37,8 @@ class Params(C.Structure):
     _fields_ = [("n_h", C.c_int32), ("d_h", C.c_int32), ("r", C.c_int32), ("d_c", C.c_int32),
                 ("elite_idx", C.c_void_p), ("rope_base", C.c_float), ("softmax_scale", C.c_float),
                 ("pair_mode", C.c_int32), ("W_uk", C.c_void_p), ("W_uv", C.c_void_p),
-                ("max_pos", C.c_int32), ("cos_sin", C.c_void_p), ("decode_kernel", C.c_int32)]
+                ("max_pos", C.c_int32), ("cos_sin", C.c_void_p), ("decode_kernel", C.c_int32),
+                ("d", C.c_int32), ("W_ke", C.c_void_p), ("W_down", C.c_void_p)]
 
 
 class CacheDesc(C.Structure):
@@ -61,6 +62,7 @@ def lib() -> C.CDLL:
         L.elitekv_layer_create.argtypes = [C.POINTER(Params), C.POINTER(vp)]
         L.elitekv_layer_destroy.argtypes = [vp]
         L.elitekv_append.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, vp, i64, vp]
+        L.elitekv_project_append.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, i64, vp]
         L.elitekv_absorb_query.argtypes = [vp, vp, vp, i32, vp, vp, vp]
         L.elitekv_decode_workspace_size.argtypes = [vp, i32, C.POINTER(sz)]
         L.elitekv_decode.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, i32, vp, sz, vp, vp]
@@ -82,7 +84,8 @@ def lib() -> C.CDLL:
                      "elitekv_plan", "elitekv_check_status", "elitekv_mha_workspace_size",
                      "elitekv_profile_enable", "elitekv_profile_collect", "elitekv_decode_static",
                      "elitekv_mha_decode", "elitekv_plan_workers", "elitekv_decode_plan_info",
-                     "elitekv_last_status_detail", "elitekv_selftest_bounded_wait"):
+                     "elitekv_last_status_detail", "elitekv_selftest_bounded_wait",
+                     "elitekv_project_append"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -118,7 +121,7 @@ class Layer:
     bf16 CUDA tensors; cos_sin an optional fp32 CUDA tensor [max_pos][d_h/2][2]."""
 
     def __init__(self, n_h, d_h, r, d_c, elite_idx, W_uk, W_uv, max_pos, rope_base=10000.0,
-                 softmax_scale=0.0, pair_mode=0, cos_sin=None, decode_kernel=0):
+                 softmax_scale=0.0, pair_mode=0, cos_sin=None, decode_kernel=0, W_ke=None, W_down=None):
         idx = elite_idx.to(torch.int32).contiguous().cpu()
         assert tuple(idx.shape) == (n_h, r)
         self.n_h, self.d_h, self.r, self.d_c = n_h, d_h, r, d_c
@@ -127,7 +130,10 @@ class Layer:
                    pair_mode, _ptr(W_uk) if W_uk is not None and W_uk.numel() else None,
                    _ptr(_dev(W_uv, torch.bfloat16)), max_pos,
                    _ptr(_dev(cos_sin, torch.float32)) if cos_sin is not None else None,
-                   decode_kernel)
+                   decode_kernel,
+                   W_down.shape[0] if W_down is not None else 0,
+                   _ptr(_dev(W_ke, torch.bfloat16)) if W_ke is not None else None,
+                   _ptr(_dev(W_down, torch.bfloat16)) if W_down is not None else None)
         h = C.c_void_p()
         _check(lib().elitekv_layer_create(C.byref(p), C.byref(h)), "elitekv_layer_create")
         self.handle = h
@@ -171,6 +177,13 @@ def elitekv_append(layer: Layer, cache: CacheDesc, k_e, c, seq_id, pos) -> None:
     _check(lib().elitekv_append(layer.handle, C.byref(cache), _ptr(k_e), _ptr(_dev(c, torch.bfloat16)),
                                 _ptr(_dev(seq_id, torch.int32)), _ptr(_dev(pos, torch.int32)), T,
                                 _stream()), "elitekv_append")
+
+
+def elitekv_project_append(layer: Layer, cache: CacheDesc, x, seq_id, pos) -> None:
+    T = x.shape[0]
+    _check(lib().elitekv_project_append(layer.handle, C.byref(cache), _ptr(_dev(x, torch.bfloat16)),
+                                        _ptr(_dev(seq_id, torch.int32)), _ptr(_dev(pos, torch.int32)), T,
+                                        _stream()), "elitekv_project_append")
 
 
 def elitekv_absorb_query(layer: Layer, q, q_pos, q_rope=None, q_abs=None):

@@ -97,6 +97,19 @@ extern "C" int elitekv_append(const elitekv_layer* L, const elitekv_cache* cache
   return rc;
 }
 
+extern "C" int elitekv_project_append(const elitekv_layer* L, const elitekv_cache* cache, const void* x,
+                                      const int32_t* seq_id, const int32_t* pos, int64_t T,
+                                      elitekv_stream_t stream) {
+  if (!L || !cache || T < 0) return ELITEKV_ERR_INVALID_ARG;
+  if (T == 0) return ELITEKV_OK;
+  if (!x || !seq_id || !pos || ((uintptr_t)x & 15)) return ELITEKV_ERR_INVALID_ARG;
+  if (L->d <= 0 || !L->d_WcatT) return ELITEKV_ERR_INVALID_ARG;     // layer created without W_ke / W_down
+  CacheView cv;
+  int rc = ekv_make_view(cache, &cv);
+  if (rc != ELITEKV_OK) return rc;
+  return ekv_launch_project_append(L, cache, cv, x, seq_id, pos, T, (cudaStream_t)stream);
+}
+
 extern "C" int elitekv_absorb_query(const elitekv_layer* L, const void* q, const int32_t* q_pos,
                                     int32_t B, void* q_rope, void* q_abs, elitekv_stream_t stream) {
   if (!L || !q || !q_pos || !q_abs || B < 0 || (L->r > 0 && !q_rope)) return ELITEKV_ERR_INVALID_ARG;

@@ -35,6 +35,8 @@ struct elitekv_layer {
   int32_t* d_status;               // [4] device status word: code, detail0, detail1, count
   struct EkvProfile* prof;         // optional event pairs around the split-K kernel
   int32_t* last_detail;            // host [3]: detail words + count read by the last check_status
+  int d;                           // model width (0: no projection weights)
+  bf16* d_WcatT;                   // [n_h*2r + d_c][d]: [W^k_e | A^kv] transposed (rows = output columns)
 };
 
 constexpr int kProfileSlots = 512;
@@ -141,6 +143,9 @@ int ekv_make_view(const elitekv_cache* cache, CacheView* out);
 int ekv_launch_append(const elitekv_layer* L, const elitekv_cache* cache, const CacheView& cv,
                       const void* k_e, const void* c, const int32_t* seq_id, const int32_t* pos,
                       long long T, cudaStream_t st);
+int ekv_launch_project_append(const elitekv_layer* L, const elitekv_cache* cache, const CacheView& cv,
+                              const void* x, const int32_t* seq_id, const int32_t* pos, long long T,
+                              cudaStream_t st);
 int ekv_launch_absorb(const elitekv_layer* L, const void* q, const int32_t* q_pos, int B,
                       void* q_rope, void* q_abs, cudaStream_t st);
 // max_len: tokens one sequence can hold in the cache; longer (or negative) lengths are recorded

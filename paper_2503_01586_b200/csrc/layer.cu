@@ -41,6 +41,7 @@ extern "C" int elitekv_layer_create(const elitekv_params* p, elitekv_layer** out
   if (p->decode_kernel < 0 || p->decode_kernel > 3) return ELITEKV_ERR_INVALID_ARG;
   if (p->d_c % 8 != 0 || p->d_h > 512) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
   if (((uintptr_t)p->W_uv & 15) || ((uintptr_t)p->W_uk & 15)) return ELITEKV_ERR_INVALID_ARG;
+  if (p->d < 0 || (p->d > 0 && (!p->W_down || (p->r > 0 && !p->W_ke)))) return ELITEKV_ERR_INVALID_ARG;
   const int n_h = p->n_h, d_h = p->d_h, r = p->r, half = d_h / 2;
 
   // index sets: in range, distinct per head; dims of the query each cache slot pairs with
@@ -111,6 +112,21 @@ extern "C" int elitekv_layer_create(const elitekv_params* p, elitekv_layer** out
       regroup_wuk_kernel<<<grid, block>>>((const bf16*)p->W_uk, L->d_WukT, p->d_c, n_h * L->dn);
       if (cudaGetLastError() != cudaSuccess) break;
     }
+    if (p->d > 0) {
+      // [W^k_e | A^kv] with the output column as the row, so that a tile of it is a K-major operand
+      const int rope_w = n_h * 2 * r;
+      const size_t n_out = (size_t)rope_w + p->d_c;
+      L->d = p->d;
+      if (cudaMalloc(&L->d_WcatT, n_out * p->d * sizeof(bf16)) != cudaSuccess) break;
+      dim3 block(32, 8);
+      if (rope_w > 0) {
+        dim3 grid((rope_w + 31) / 32, (p->d + 31) / 32);
+        regroup_wuk_kernel<<<grid, block>>>((const bf16*)p->W_ke, L->d_WcatT, p->d, rope_w);
+      }
+      dim3 grid2((p->d_c + 31) / 32, (p->d + 31) / 32);
+      regroup_wuk_kernel<<<grid2, block>>>((const bf16*)p->W_down, L->d_WcatT + (size_t)rope_w * p->d, p->d, p->d_c);
+      if (cudaGetLastError() != cudaSuccess) break;
+    }
     if (cudaDeviceSynchronize() != cudaSuccess) break;
     rc = ELITEKV_OK;
   } while (0);
@@ -131,6 +147,7 @@ extern "C" int elitekv_layer_destroy(elitekv_layer* L) {
   cudaFree(L->d_cs_owned);
   cudaFree(L->d_WukT);
   cudaFree(L->d_Wuv);
+  cudaFree(L->d_WcatT);
   if (L->prof) {
     for (int i = 0; i < 2 * kProfileSlots; ++i)
       if (L->prof->ev[i]) cudaEventDestroy(L->prof->ev[i]);

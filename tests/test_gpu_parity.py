@@ -93,6 +93,86 @@ def test_append_bad_position_is_reported_not_written(ek):
     assert np.count_nonzero(lat.any(axis=1)) == 1
 
 
+# ------------------------------------------------------------------ fused projection + append
+def _projection_case(ek, w, d, lens, paged, seed):
+    """Hidden states through elitekv_project_append into a canary-filled cache, against the
+    float64 oracle: untouched rows stay bit for bit, written rows match the single-rounded float64
+    result within bf16 rounding of an fp32-accumulated product."""
+    w = replace(w, paged=paged, seed=seed)
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    rope_w = w.n_h * 2 * w.r
+    W_ke = (torch.randn(d, rope_w, generator=g) / d ** 0.5).to(torch.bfloat16).cuda()
+    W_down = (torch.randn(d, w.d_c, generator=g) / d ** 0.5).to(torch.bfloat16).cuda()
+    idx = gen.elite_index_sets(w)
+    W_uk, W_uv = gen.up_projections(w, "cuda")
+    max_ctx = max(lens) + 1
+    layer = ek.Layer(w.n_h, w.d_h, w.r, w.d_c, idx, W_uk, W_uv, max_ctx + 1, W_ke=W_ke, W_down=W_down)
+    lens_t = torch.tensor(lens, dtype=torch.int32)
+    B = len(lens)
+    if paged:
+        table, num_pages = gen.page_table(replace(w, B=B), lens_t, headroom_tokens=1)
+        rows, page_table, mc = num_pages * w.page_size, table.cuda(), 0
+    else:
+        rows, page_table, mc = B * max_ctx, None, max_ctx
+    rope0 = torch.randint(0, 2 ** 15, (rows, rope_w), generator=g, dtype=torch.int16)
+    lat0 = torch.randint(0, 2 ** 15, (rows, w.d_c), generator=g, dtype=torch.int16)
+    rope_plane = rope0.view(torch.bfloat16).cuda()
+    latent_plane = lat0.view(torch.bfloat16).cuda()
+    cache = ek.make_cache(rope_plane, latent_plane, n_seqs=B, max_ctx=mc, page_table=page_table, page_size=w.page_size)
+    T = int(sum(lens))
+    x = torch.randn(T, d, generator=g).to(torch.bfloat16).cuda()
+    seq = torch.repeat_interleave(torch.arange(B, dtype=torch.int32), lens_t.to(torch.int64))
+    pos = torch.cat([torch.arange(n, dtype=torch.int32) for n in lens])
+    perm = torch.randperm(T, generator=g)
+    ek.elitekv_project_append(layer, cache, x[perm.cuda()].contiguous(), seq[perm].cuda(), pos[perm].cuda())
+    torch.cuda.synchronize()
+    assert ek.elitekv_check_status(layer) == 0
+    exp_r, exp_l, rows64, c64 = O.project_append_expected(
+        rope0.numpy().view(np.uint16), lat0.numpy().view(np.uint16), H.f64(x), H.f64(W_ke), H.f64(W_down),
+        seq.numpy(), pos.numpy(), idx.numpy(), w.d_h, base=w.rope_base, max_ctx=mc if not paged else None,
+        page_table=page_table.cpu().numpy() if paged else None, page_size=w.page_size)
+    slot = O.token_slot(seq.numpy(), pos.numpy(), max_ctx=mc if not paged else None,
+                        page_table=page_table.cpu().numpy() if paged else None, page_size=w.page_size)
+    got_r, got_l = H.bits(rope_plane), H.bits(latent_plane)
+    untouched = np.ones(rows, dtype=bool)
+    untouched[slot] = False
+    assert np.array_equal(got_r[untouched], rope0.numpy().view(np.uint16)[untouched])
+    assert np.array_equal(got_l[untouched], lat0.numpy().view(np.uint16)[untouched])
+    for got, want in ((O.bf16_bits_to_f64(got_r[slot]), rows64), (O.bf16_bits_to_f64(got_l[slot]), c64)):
+        # one bf16 rounding (2^-9 relative) plus fp32 accumulation over d terms
+        assert np.all(np.abs(got - want) <= np.abs(want) * 2.0 ** -8 + 2e-5 * d ** 0.5), float(np.max(np.abs(got - want)))
+        rel = np.linalg.norm(got - want) / np.linalg.norm(want)
+        assert rel < 3e-3, rel
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_project_append_7b_shape(ek, paged):
+    """d = 4096: 64 depth stages through a 4-stage ring; 700 tokens = 5 full token tiles and a
+    ragged sixth; rope part 4 column tiles, latent part 12."""
+    _projection_case(ek, gen.shrink(gen.LLAMA7B_75, B=3, ctx=400), 4096, [400, 237, 63], paged, 91 + paged)
+
+
+def test_project_append_other_shapes(ek):
+    _projection_case(ek, gen.shrink(gen.SWEEP_875, B=2, ctx=100), 1024, [100, 29], False, 93)
+    _projection_case(ek, gen.shrink(gen.LLAMA13B_75, B=2, ctx=140), 5120, [1, 140], False, 94)
+
+
+def test_project_append_needs_projection_weights_and_a_covered_shape(ek):
+    w = replace(SMALL, seed=95)
+    st = H.setup(w, lens=[5, 5, 5])
+    x = torch.zeros((2, 192), dtype=torch.bfloat16, device="cuda")
+    z = torch.zeros(2, dtype=torch.int32, device="cuda")
+    with pytest.raises(ek.ElitekvError) as e:          # layer without W_ke / W_down
+        ek.elitekv_project_append(st.layer, st.cache, x, z, z)
+    assert e.value.code == ek.ERR_INVALID_ARG
+    W_ke = torch.zeros((192, w.n_h * 2 * w.r), dtype=torch.bfloat16, device="cuda")
+    W_down = torch.zeros((192, w.d_c), dtype=torch.bfloat16, device="cuda")
+    layer = ek.Layer(w.n_h, w.d_h, w.r, w.d_c, st.idx, st.W_uk, st.W_uv, 64, W_ke=W_ke, W_down=W_down)
+    with pytest.raises(ek.ElitekvError) as e:          # 36 rope columns and d_c = 72: not 128-column tiles
+        ek.elitekv_project_append(layer, st.cache, x, z, z)
+    assert e.value.code == ek.ERR_UNSUPPORTED_SHAPE
+
+
 # ------------------------------------------------------------------ query preparation
 @pytest.mark.parametrize("pair_mode", [0, 1])
 def test_absorb_query(ek, pair_mode):

@@ -157,7 +157,7 @@ def config_of(w: gen.Workload, world: int):
          "batch_per_gpu": w.B, "context": w.ctx, "paged": w.paged,
          "l2": "256 MiB flush write before every timed step; cache larger than L2",
          "parallelism": f"replicas x{world} (independent sequences, no collective)",
-         "streams": "append on a second stream beside absorb_query; joined before decode"}
+         "streams": "elitekv_decode_step: append + plan on the layer's second stream beside absorb_query; joined before the attention kernel"}
     return c
 
 
@@ -260,31 +260,11 @@ def build_workload(w: gen.Workload, ek, device, decode_kernel: int = 0):
     return layer, cache, lens, host, dev, ws, bufs, keep
 
 
-_SIDE_STREAM = None
-
-
 def step(ek, layer, cache, d, ws, bufs):
-    """One decode step.  The append (writes the cache) and the query preparation (reads only the
-    queries) do not depend on each other, so the append runs on a second stream beside the
-    absorb; both are joined before the attention call."""
-    global _SIDE_STREAM
-    main = torch.cuda.current_stream()
-    if _SIDE_STREAM is None:
-        _SIDE_STREAM = torch.cuda.Stream()
-    _SIDE_STREAM.wait_stream(main)
-    with torch.cuda.stream(_SIDE_STREAM):
-        ek.elitekv_append(layer, cache, d["k_e"], d["c"], d["seq_id"], d["pos"])
-    ek.elitekv_absorb_query(layer, d["q"], d["pos"], bufs["q_rope"], bufs["q_abs"])
-    main.wait_stream(_SIDE_STREAM)
-    ek.elitekv_decode(layer, cache, bufs["q_rope"], bufs["q_abs"], d["lens"], ws, bufs["out"])
-
-
-def step_serial(ek, layer, cache, d, ws, bufs):
-    """The same three calls on one stream (used by the end-to-end leg, which is bound by host
-    latency: the second stream's event bookkeeping costs more there than the overlap saves)."""
-    ek.elitekv_append(layer, cache, d["k_e"], d["c"], d["seq_id"], d["pos"])
-    ek.elitekv_absorb_query(layer, d["q"], d["pos"], bufs["q_rope"], bufs["q_abs"])
-    ek.elitekv_decode(layer, cache, bufs["q_rope"], bufs["q_abs"], d["lens"], ws, bufs["out"])
+    """One decode step through the library's single-call entry: the append and the work plan run
+    on the layer's second stream beside the query preparation, joined before the attention."""
+    ek.elitekv_decode_step(layer, cache, d["k_e"], d["c"], d["seq_id"], d["pos"], d["q"], d["lens"],
+                           bufs["q_rope"], bufs["q_abs"], ws, bufs["out"])
 
 
 KERNELS_PER_STEP = 5   # append, absorb, plan, split-K attention, combine + up-projection
@@ -356,6 +336,56 @@ def sweep_entry(ek, w: gen.Workload, device, flush, steps: int = 10, n_check: in
     del layer, cache, dev, ws, bufs, keep
     torch.cuda.empty_cache()
     return entry
+
+
+def project_append_bench(ek, device, flush, reps: int = 5):
+    """The projection fused with the append (x [W^k_e, A^kv], 7B 75 % shape, d = 4096) at prefill
+    size (T = 4096: tensor bound, bf16 TFLOP/s against the measured cuBLAS figure) and at the
+    size of a decode batch (T = 16: bound by reading the 16.8 MB of weights once)."""
+    w = gen.SWEEP_75
+    d, T_max = 4096, 4096
+    g = torch.Generator(device=device).manual_seed(4242)
+    rope_w = w.n_h * 2 * w.r
+    W_ke = (torch.randn(d, rope_w, generator=g, device=device) / d ** 0.5).to(torch.bfloat16)
+    W_down = (torch.randn(d, w.d_c, generator=g, device=device) / d ** 0.5).to(torch.bfloat16)
+    idx = gen.elite_index_sets(w)
+    W_uk, W_uv = gen.up_projections(w, device)
+    layer = ek.Layer(w.n_h, w.d_h, w.r, w.d_c, idx, W_uk, W_uv, T_max + 1, W_ke=W_ke, W_down=W_down)
+    rope_plane = torch.zeros((T_max, rope_w), dtype=torch.bfloat16, device=device)
+    latent_plane = torch.zeros((T_max, w.d_c), dtype=torch.bfloat16, device=device)
+    cache = ek.make_cache(rope_plane, latent_plane, n_seqs=1, max_ctx=T_max)
+    x = torch.randn(T_max, d, generator=g, device=device).to(torch.bfloat16)
+    seq = torch.zeros(T_max, dtype=torch.int32, device=device)
+    pos = torch.arange(T_max, dtype=torch.int32, device=device)
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            tf_peak, tf_kind = float(json.load(f)["bf16_tflops"]), "of measured"
+    except Exception:
+        tf_peak, tf_kind = 1590.0, "of fallback"
+    hbm_peak, hbm_kind = measured_peaks()
+    out = {}
+    for T in (T_max, 16):
+        for _ in range(2):
+            ek.elitekv_project_append(layer, cache, x[:T], seq[:T], pos[:T])
+        evs = []
+        for _ in range(reps):
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            ek.elitekv_project_append(layer, cache, x[:T], seq[:T], pos[:T])
+            b.record()
+            evs.append((a, b))
+        torch.cuda.synchronize()
+        us = 1e3 * sum(a.elapsed_time(b) for a, b in evs) / reps
+        flops = 2.0 * T * d * (rope_w + w.d_c)
+        weight_bytes = 2 * d * (rope_w + w.d_c)
+        out[f"T{T}"] = {"tokens": T, "us": us, "tflops": flops / (us * 1e-6) / 1e12,
+                        "frac_tensor": flops / (us * 1e-6) / 1e12 / tf_peak, "tensor_peak_kind": tf_kind,
+                        "weight_gbs": weight_bytes / (us * 1e-6) / 1e9,
+                        "frac_hbm_weights": weight_bytes / (us * 1e-6) / 1e9 / hbm_peak, "hbm_peak_kind": f"of {hbm_kind}"}
+    assert ek.elitekv_check_status(layer) == 0
+    return out
+
 
 
 def append_prefill(ek, device, flush, reps: int = 5):
@@ -455,63 +485,34 @@ def run_gpu(args, w: gen.Workload):
     kern_ms, kern_n = ek.elitekv_profile_collect(layer)
     ek.elitekv_profile_enable(layer, False)
 
-    # ---- end to end: host buffers in, host result out, every step.  The step's six small input
-    #      arrays live in ONE pinned staging buffer (256-byte aligned sections) and cross in one
-    #      copy; the device-side tensors are views into its device twin.
-    order = ["k_e", "c", "q", "seq_id", "pos", "lens"]
-    offs, at = {}, 0
-    for k in order:
-        offs[k] = at
-        at = (at + host[k].numel() * host[k].element_size() + 255) & ~255
-    pack_host = torch.empty(at, dtype=torch.uint8).pin_memory()
-    pack_dev = torch.empty(at, dtype=torch.uint8, device=device)
-
-    def view(buf, k):
-        n = host[k].numel() * host[k].element_size()
-        return buf[offs[k]:offs[k] + n].view(host[k].dtype).view(host[k].shape)
-    for k in order:
-        view(pack_host, k).copy_(host[k])
-    staged = {k: view(pack_dev, k) for k in order}
-    h2d = pack_host.numel()
-    d2h = bufs["out_host"].numel() * bufs["out_host"].element_size()
-
-    def e2e_step():
-        pack_dev.copy_(pack_host, non_blocking=True)
-        step_serial(ek, layer, cache, staged, ws, bufs)
-        bufs["out_host"].copy_(bufs["out"], non_blocking=True)
-        torch.cuda.synchronize()
-
-    for _ in range(3):
-        e2e_step()
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(args.steps):
-        e2e_step()           # no flush here: the 268 MB+ cache does not fit the 126 MB L2
-    torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
-
-    # ---- the same end-to-end step captured once in a CUDA graph and replayed (informational:
-    #      what a serving loop that graphs its decode step gets; `e2e.value` stays the eager path)
-    e2e_graph_s = None
-    try:
-        side = torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=side):
-            pack_dev.copy_(pack_host, non_blocking=True)
-            step_serial(ek, layer, cache, staged, ws, bufs)
-            bufs["out_host"].copy_(bufs["out"], non_blocking=True)
+    # ---- end to end: host buffers in, host result out, every step, through the library's step
+    #      runner: the six small input arrays live in ONE pinned staging buffer and cross in one
+    #      copy, the step runs, the result is copied back and the host waits for it.  The headline
+    #      replays the runner's CUDA graph (what a serving loop does); the eager number (same
+    #      work enqueued call by call, bound by host launch latency) is reported beside it.
+    def e2e_time(runner):
+        for k in runner.ORDER:
+            runner.host[k].copy_(host[k].view(runner.host[k].shape))
         for _ in range(3):
-            graph.replay()
-            torch.cuda.synchronize()
+            runner.run()
+        assert torch.equal(runner.out_host, bufs["out"].cpu())      # same step, same bits
+        barrier()
         t0 = time.perf_counter()
         for _ in range(args.steps):
-            graph.replay()
-            torch.cuda.synchronize()
-        e2e_graph_s = time.perf_counter() - t0
-        assert ek.elitekv_check_status(layer) == 0
-    except Exception as exc:      # capture not possible in this environment: report only the eager number
-        print(f"[bench] CUDA-graph end-to-end leg skipped: {exc}", file=sys.stderr)
+            runner.run()         # no flush here: the 268 MB+ cache does not fit the 126 MB L2
+        torch.cuda.synchronize()
+        return time.perf_counter() - t0
+
+    eager_runner = ek.DecodeStepRunner(layer, cache, w.B, device, graph=False)
+    h2d, d2h = eager_runner.h2d_bytes, eager_runner.d2h_bytes
+    e2e_eager_s = e2e_time(eager_runner)
+    e2e_mode = "cuda graph replay (DecodeStepRunner)"
+    try:
+        e2e_s = e2e_time(ek.DecodeStepRunner(layer, cache, w.B, device, graph=True))
+    except Exception as exc:      # capture not possible in this environment: the eager number stands
+        print(f"[bench] CUDA-graph end-to-end leg failed, reporting the eager one: {exc}", file=sys.stderr)
+        e2e_s, e2e_mode = e2e_eager_s, "eager (DecodeStepRunner, graph capture failed)"
+    assert ek.elitekv_check_status(layer) == 0
 
     # ---- per-call breakdown (informational; same kernels, a few extra untimed-by-the-metric calls)
     def timed(fn, n=10):
@@ -572,12 +573,13 @@ def run_gpu(args, w: gen.Workload):
             comparator = None
 
     # ---- the other benchmark configurations and the prefill append (one GPU, rank 0 only)
-    sweep, prefill = None, None
+    sweep, prefill, projection = None, None, None
     if rank == 0 and world == 1 and not args.no_sweep:
-        del layer, cache, dev, ws, bufs, keep, staged, pack_dev
+        del layer, cache, dev, ws, bufs, keep, eager_runner
         torch.cuda.empty_cache()
         t_sweep = time.perf_counter()
         prefill = append_prefill(ek, device, flush)
+        projection = project_append_bench(ek, device, flush)
         sweep = []
         for name in SWEEP:
             if name == w.name:
@@ -618,8 +620,8 @@ def run_gpu(args, w: gen.Workload):
                      "kernel_us": kern_avg_s * 1e6, "launches_timed": kern_n,
                      "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(w.name)},
         "e2e": {"value": world * w.B * args.steps / e2e_s, "unit": UNIT,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "value_cuda_graph": (world * w.B * args.steps / e2e_graph_s) if e2e_graph_s else None},
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "mode": e2e_mode,
+                "value_eager": world * w.B * args.steps / e2e_eager_s},
         "gpu_launches": KERNELS_PER_STEP * args.steps,
         "clocks": clocks,
         "stages": stages,
@@ -630,6 +632,7 @@ def run_gpu(args, w: gen.Workload):
     else:
         line["cpu_baseline"] = None
     line["stages"]["append_prefill"] = prefill
+    line["stages"]["project_append"] = projection
     line["sweep"] = sweep
     print(json.dumps(line))
     if dist is not None:

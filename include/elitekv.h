@@ -13,7 +13,8 @@
  *   W_uv = B^v_J  [d_c][n_h d_h]          head h owns columns [h d_h, (h+1) d_h)
  *   theta_i = rope_base^(-2 i / d_h), chunk i = dims (2i, 2i+1)            (Section 2.2)
  *
- * One decode step of a layer is   elitekv_append -> elitekv_absorb_query -> elitekv_decode.
+ * One decode step of a layer is   elitekv_append -> elitekv_absorb_query -> elitekv_decode,
+ * or the single call elitekv_decode_step, which overlaps the independent parts.
  *
  * General rules
  *   - Pointers are DEVICE pointers unless a comment says "host".  All floating-point tensors
@@ -161,6 +162,21 @@ int elitekv_decode_workspace_size(const elitekv_layer* layer, int32_t B, size_t*
 int elitekv_decode(const elitekv_layer* layer, const elitekv_cache* cache, const void* q_rope,
                    const void* q_abs, const int32_t* seq_lens, int32_t B, void* workspace,
                    size_t workspace_bytes, void* out, elitekv_stream_t stream);
+
+/* One whole decode step of a layer in one call (Sections 3.1, 3.2, 5): token b (cache entries
+ * k_e[b], c[b]) is appended to sequence seq_id[b] at position pos[b], the query q[b] is
+ * prepared at that same position (elitekv_absorb_query with q_pos = pos) into the caller's
+ * q_rope / q_abs buffers, and elitekv_decode runs over seq_lens (the lengths INCLUDING the new
+ * tokens).  Arguments, shapes, alignment and errors are those of the three calls; the result
+ * is bit-identical to calling them in order.  The append and the work plan depend only on the
+ * new tokens and the lengths, so they run on a stream the layer owns, beside the query
+ * preparation on `stream`, and are joined before the attention kernel; to the caller the call
+ * behaves like work enqueued on `stream` alone (it may be captured in a CUDA graph).  Two
+ * threads must not run steps of the same layer object at the same time. */
+int elitekv_decode_step(const elitekv_layer* layer, const elitekv_cache* cache, const void* k_e,
+                        const void* c, const int32_t* seq_id, const int32_t* pos, const void* q,
+                        const int32_t* seq_lens, int32_t B, void* q_rope, void* q_abs,
+                        void* workspace, size_t workspace_bytes, void* out, elitekv_stream_t stream);
 
 /* Decode attention without any allocation (the paper has no counterpart; this is a packaging
  * variant of elitekv_decode).  For callers that must not, or cannot, call cudaMalloc: engines

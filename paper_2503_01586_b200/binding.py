@@ -66,6 +66,7 @@ def lib() -> C.CDLL:
         L.elitekv_absorb_query.argtypes = [vp, vp, vp, i32, vp, vp, vp]
         L.elitekv_decode_workspace_size.argtypes = [vp, i32, C.POINTER(sz)]
         L.elitekv_decode.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, i32, vp, sz, vp, vp]
+        L.elitekv_decode_step.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, sz, vp, vp]
         L.elitekv_decode_static.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, i32, vp, vp]
         L.elitekv_plan.argtypes = [vp, i32, i32, i32, vp, vp, vp]
         L.elitekv_plan_workers.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp]
@@ -85,7 +86,7 @@ def lib() -> C.CDLL:
                      "elitekv_profile_enable", "elitekv_profile_collect", "elitekv_decode_static",
                      "elitekv_mha_decode", "elitekv_plan_workers", "elitekv_decode_plan_info",
                      "elitekv_last_status_detail", "elitekv_selftest_bounded_wait",
-                     "elitekv_project_append"):
+                     "elitekv_project_append", "elitekv_decode_step"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -214,6 +215,89 @@ def elitekv_decode(layer: Layer, cache: CacheDesc, q_rope, q_abs, seq_lens, work
                                 workspace.numel() * workspace.element_size(), _ptr(out), _stream()),
            "elitekv_decode")
     return out
+
+
+def elitekv_decode_step(layer: Layer, cache: CacheDesc, k_e, c, seq_id, pos, q, seq_lens, q_rope, q_abs,
+                        workspace, out):
+    """Append + query preparation + decode attention of one step in one call (buffers are the
+    caller's: nothing is allocated here)."""
+    B = q.shape[0]
+    _check(lib().elitekv_decode_step(layer.handle, C.byref(cache), _ptr(k_e), _ptr(_dev(c, torch.bfloat16)),
+                                     _ptr(_dev(seq_id, torch.int32)), _ptr(_dev(pos, torch.int32)),
+                                     _ptr(_dev(q, torch.bfloat16)), _ptr(_dev(seq_lens, torch.int32)), B,
+                                     _ptr(q_rope), _ptr(_dev(q_abs, torch.bfloat16)), workspace.data_ptr(),
+                                     workspace.numel() * workspace.element_size(),
+                                     _ptr(_dev(out, torch.bfloat16)), _stream()), "elitekv_decode_step")
+    return out
+
+
+class DecodeStepRunner:
+    """Host-to-host decode step of one layer at a fixed batch size B.  The step's six input
+    arrays live in ONE pinned staging buffer (`host[...]`: k_e [B][n_h][2r], c [B][d_c],
+    q [B][n_h][d_h], seq_id / pos / lens [B] int32) that crosses in one copy; the result comes
+    back into the pinned `out_host` [B][n_h][d_h].  With `graph=True` the copy in, the
+    elitekv_decode_step call and the copy out are captured in a CUDA graph on the second `run()`
+    and replayed from then on; otherwise `run()` enqueues the three eagerly.  Marshalling only: every byte of
+    arithmetic happens in the library's kernels."""
+
+    ORDER = ("k_e", "c", "q", "seq_id", "pos", "lens")
+
+    def __init__(self, layer: Layer, cache: CacheDesc, B: int, device, graph: bool = True):
+        self.layer, self.cache, self.B = layer, cache, B
+        bf, i32 = torch.bfloat16, torch.int32
+        shapes = {"k_e": ((B, layer.n_h, 2 * layer.r), bf), "c": ((B, layer.d_c), bf),
+                  "q": ((B, layer.n_h, layer.d_h), bf), "seq_id": ((B,), i32), "pos": ((B,), i32),
+                  "lens": ((B,), i32)}
+        offs, at = {}, 0
+        for k in self.ORDER:
+            shape, dt = shapes[k]
+            n = 1
+            for e in shape:
+                n *= e
+            offs[k] = (at, n * torch.empty((), dtype=dt).element_size())
+            at = (at + offs[k][1] + 255) & ~255
+        self.pack_host = torch.zeros(max(at, 256), dtype=torch.uint8).pin_memory()
+        self.pack_dev = torch.zeros(max(at, 256), dtype=torch.uint8, device=device)
+
+        def views(buf):
+            return {k: buf[offs[k][0]:offs[k][0] + offs[k][1]].view(shapes[k][1]).view(shapes[k][0])
+                    for k in self.ORDER}
+        self.host, self.dev = views(self.pack_host), views(self.pack_dev)
+        self.q_rope = torch.empty((B, layer.n_h, 2 * layer.r), dtype=bf, device=device)
+        self.q_abs = torch.empty((B, layer.n_h, layer.d_c), dtype=bf, device=device)
+        self.out = torch.empty((B, layer.n_h, layer.d_h), dtype=bf, device=device)
+        self.out_host = torch.empty((B, layer.n_h, layer.d_h), dtype=bf).pin_memory()
+        self.workspace = torch.empty(elitekv_decode_workspace_size(layer, B), dtype=torch.uint8, device=device)
+        self.h2d_bytes = self.pack_host.numel()
+        self.d2h_bytes = self.out_host.numel() * self.out_host.element_size()
+        self.graph = None
+        self._want_graph, self._warm = graph, False
+
+    def _enqueue(self):
+        d = self.dev
+        self.pack_dev.copy_(self.pack_host, non_blocking=True)
+        elitekv_decode_step(self.layer, self.cache, d["k_e"], d["c"], d["seq_id"], d["pos"], d["q"], d["lens"],
+                            self.q_rope, self.q_abs, self.workspace, self.out)
+        self.out_host.copy_(self.out, non_blocking=True)
+
+    def run(self, wait: bool = True):
+        """One step from `host[...]` to `out_host`; with `wait`, returns once the result is there.
+        Nothing runs before the first call (the staging buffer is the caller's to fill first):
+        that call goes eagerly, the second one captures the graph."""
+        if self._want_graph and self.graph is None and self._warm:
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                self._enqueue()
+            self.graph = g
+        if self.graph is not None:
+            self.graph.replay()
+        else:
+            self._enqueue()
+            self._warm = True
+        if wait:
+            torch.cuda.current_stream().synchronize()
+        return self.out_host
 
 
 def elitekv_decode_static(layer: Layer, cache: CacheDesc, q_rope, q_abs, seq_lens, out):

@@ -140,10 +140,16 @@ extern "C" int elitekv_decode_plan_info(const elitekv_layer* L, const elitekv_ca
   return ELITEKV_OK;
 }
 
-extern "C" int elitekv_decode(const elitekv_layer* L, const elitekv_cache* cache,
-                              const void* q_rope, const void* q_abs, const int32_t* seq_lens,
-                              int32_t B, void* workspace, size_t workspace_bytes, void* out,
-                              elitekv_stream_t stream) {
+namespace {
+
+// Plan, split-K kernel and combine of one attention call.  With `plan_stream` set, the plan is
+// launched there (beside whatever runs on `st`), `ev_join` is recorded behind it and `st` waits
+// for that event before the split-K kernel; `before_kernel` (may be empty) is enqueued on `st`
+// in between, i.e. beside the plan.
+template <class Fn>
+int decode_impl(const elitekv_layer* L, const elitekv_cache* cache, const void* q_rope, const void* q_abs,
+                const int32_t* seq_lens, int32_t B, void* workspace, size_t workspace_bytes, void* out,
+                cudaStream_t st, cudaStream_t plan_stream, Fn before_kernel) {
   if (!L || !cache || !q_abs || !seq_lens || !workspace || !out || B <= 0 || (L->r > 0 && !q_rope))
     return ELITEKV_ERR_INVALID_ARG;
   if (((uintptr_t)q_abs & 15) || ((uintptr_t)out & 3)) return ELITEKV_ERR_INVALID_ARG;
@@ -168,17 +174,25 @@ extern "C" int elitekv_decode(const elitekv_layer* L, const elitekv_cache* cache
   ws.n_counters = ekv_combine_counters(L, B);
   ws.worker_first = (int32_t*)(base + cw.off_wfirst);
   ws.n_workers = workers_for(L, kernel);
-  cudaStream_t st = (cudaStream_t)stream;
   // tokens one sequence can hold: longer lengths are reported by the plan kernel and clamped
   const long long max_len = cv.page_table ? (long long)cv.max_pages_per_seq << cv.page_shift : cv.max_ctx;
+  cudaStream_t ps = plan_stream ? plan_stream : st;
   if (ws.n_workers > 0)
     rc = ekv_launch_plan_balanced(seq_lens, B, plan_tile_for(kernel), ws.n_workers, max_items, ws.items, ws.seq_first,
                                   ws.worker_first, ws.counters, ws.n_counters, max_len, L->d_status,
-                                  item_overhead_for(kernel), st);
+                                  item_overhead_for(kernel), ps);
   else
     rc = ekv_launch_plan(seq_lens, B, plan_tile_for(kernel), max_items, ws.items, ws.seq_first,
-                         ws.counters, ws.n_counters, max_len, L->d_status, st);
+                         ws.counters, ws.n_counters, max_len, L->d_status, ps);
+  int rc_mid = ELITEKV_OK;
+  if (plan_stream) {
+    // the join is enqueued whatever happened above, so that the side stream never stays forked
+    if (cudaEventRecord(L->ev_join, plan_stream) != cudaSuccess) return ELITEKV_ERR_CUDA;
+    rc_mid = before_kernel();
+    if (cudaStreamWaitEvent(st, L->ev_join, 0) != cudaSuccess) return ELITEKV_ERR_CUDA;
+  }
   if (rc != ELITEKV_OK) return rc;
+  if (rc_mid != ELITEKV_OK) return rc_mid;
   EkvProfile* prof = (L->prof && L->prof->enabled && L->prof->count < kProfileSlots) ? L->prof : nullptr;
   if (prof) EKV_CUDA_OK(cudaEventRecord(prof->ev[2 * prof->count], st));
   rc = kernel == 3   ? ekv_launch_decode_rt(L, cache, cv, q_rope, q_abs, B, ws, st)
@@ -189,6 +203,45 @@ extern "C" int elitekv_decode(const elitekv_layer* L, const elitekv_cache* cache
     EKV_CUDA_OK(cudaEventRecord(prof->ev[2 * prof->count + 1], st));
     prof->count++;
   }
-  rc = ekv_launch_combine(L, B, ws, out, st);
-  return rc;
+  return ekv_launch_combine(L, B, ws, out, st);
+}
+
+}  // namespace
+
+extern "C" int elitekv_decode(const elitekv_layer* L, const elitekv_cache* cache,
+                              const void* q_rope, const void* q_abs, const int32_t* seq_lens,
+                              int32_t B, void* workspace, size_t workspace_bytes, void* out,
+                              elitekv_stream_t stream) {
+  return decode_impl(L, cache, q_rope, q_abs, seq_lens, B, workspace, workspace_bytes, out,
+                     (cudaStream_t)stream, nullptr, [] { return (int)ELITEKV_OK; });
+}
+
+extern "C" int elitekv_decode_step(const elitekv_layer* L, const elitekv_cache* cache, const void* k_e,
+                                   const void* c, const int32_t* seq_id, const int32_t* pos,
+                                   const void* q, const int32_t* seq_lens, int32_t B, void* q_rope,
+                                   void* q_abs, void* workspace, size_t workspace_bytes, void* out,
+                                   elitekv_stream_t stream) {
+  if (!L || !cache || B <= 0) return ELITEKV_ERR_INVALID_ARG;
+  if (!c || !seq_id || !pos || !q || !q_abs || !seq_lens || !workspace || !out) return ELITEKV_ERR_INVALID_ARG;
+  if (L->r > 0 && (!k_e || !q_rope)) return ELITEKV_ERR_INVALID_ARG;
+  if (((uintptr_t)k_e & 15) || ((uintptr_t)c & 15) || ((uintptr_t)q & 15) || ((uintptr_t)q_abs & 15) ||
+      ((uintptr_t)q_rope & 3))
+    return ELITEKV_ERR_INVALID_ARG;
+  CacheView cv;
+  int rc = ekv_make_view(cache, &cv);
+  if (rc != ELITEKV_OK) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  // fork: the append (writes the cache) and, behind it, the plan (reads only the lengths) run
+  // on the layer's second stream, beside the query preparation on the caller's stream
+  EKV_CUDA_OK(cudaEventRecord(L->ev_fork, st));
+  EKV_CUDA_OK(cudaStreamWaitEvent(L->side, L->ev_fork, 0));
+  const int rc_append = ekv_launch_append(L, cache, cv, k_e, c, seq_id, pos, B, L->side);
+  rc = decode_impl(L, cache, q_rope, q_abs, seq_lens, B, workspace, workspace_bytes, out, st, L->side,
+                   [&] { return ekv_launch_absorb(L, q, pos, B, q_rope, q_abs, st); });
+  if (rc != ELITEKV_OK) {
+    // a call that gave up before its own join: bring the side stream back all the same
+    cudaEventRecord(L->ev_join, L->side);
+    cudaStreamWaitEvent(st, L->ev_join, 0);
+  }
+  return rc_append != ELITEKV_OK ? rc_append : rc;
 }

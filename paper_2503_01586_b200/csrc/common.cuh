@@ -37,6 +37,8 @@ struct elitekv_layer {
   int32_t* last_detail;            // host [3]: detail words + count read by the last check_status
   int d;                           // model width (0: no projection weights)
   bf16* d_WcatT;                   // [n_h*2r + d_c][d]: [W^k_e | A^kv] transposed (rows = output columns)
+  cudaStream_t side;               // second stream of elitekv_decode_step (append + plan beside the absorb)
+  cudaEvent_t ev_fork, ev_join;    // its fork from / join into the caller's stream
 };
 
 constexpr int kProfileSlots = 512;

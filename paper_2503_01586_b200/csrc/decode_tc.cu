@@ -21,8 +21,9 @@
 //
 // A block is a persistent worker: it walks the items of the balanced plan that fall into its
 // share of the batch's tiles and writes one partial result (m, l, acc) per item.  Layers whose
-// fp32 output does not fit TMEM's 512 columns for 32 heads (d_c > 1920 or n_h != 32) run with
-// 16 heads per block; the head groups of an item are adjacent blocks so that they share L2.
+// fp32 output does not fit TMEM's 512 columns for 32 heads (d_c > 1920) run with 16 heads per
+// block, layers with more than 32 heads as several head groups; the head groups of an item are
+// adjacent blocks so that they share L2.
 //
 // Roles (288 threads):
 //   warps 0,7,8  latent TMA producers (ring uses dealt round-robin)
@@ -52,6 +53,7 @@ constexpr int kRopeSlots = 3;
 constexpr int kThreads = 288;         // warps 0,7,8 latent loads, 1 MMA, 2-5 softmax, 6 rope loads
 constexpr int kProdWarps = 3;         // latent-load warps: 0, 7, 8
 constexpr int kSoftmaxThreads = 128;
+constexpr int kOutBufs = 12;          // [N heads][128 coords] fp32 staging tiles of the epilogue (ring + rope area)
 
 struct TcArgs {
   const int32_t* items;
@@ -517,7 +519,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         float v[N];
         tc_ld_cols<N>(tmem_base + blk * N + lane_base, v);
         tc_wait_ld();
-        float* tile_s = stage + (size_t)blk * N * 128;
+        if (blk >= kOutBufs) {     // a staging buffer comes round again: its store must have read it
+          if (threadIdx.x == 64) bulk_wait_group_read<kOutBufs - 1>();
+          named_bar_sync(1, kSoftmaxThreads);
+        }
+        float* tile_s = stage + (size_t)(blk % kOutBufs) * N * 128;
 #pragma unroll
         for (int h = 0; h < N; ++h) tile_s[h * 128 + trow] = v[h];
         fence_proxy_async();
@@ -553,12 +559,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
 
 }  // namespace
 
-// Heads per block: all 32 when the fp32 output of every head fits TMEM's 512 columns, else
-// groups of 16 heads (each group streams the token tile itself; the groups of an item are
-// adjacent blocks so that the second and third reader hit L2).
+// Heads per block: 32 when 32 fp32 output columns per 128 latent coordinates plus the score
+// columns fit TMEM's 512 columns (d_c <= 1920), else 16.  A layer with more heads than that runs
+// as head groups (the last one partly filled: 40 heads = 32 + 8); each group streams the token
+// tile itself, and the groups of an item are adjacent blocks so that the later readers hit L2.
 static int tc_pick_n(const elitekv_layer* L) {
   const int nb = L->d_c / 128;
-  if (L->n_h == 32 && (nb + 1) * 32 <= 512) return 32;
+  if ((nb + 1) * 32 <= 512) return 32;
   if ((nb + 1) * 16 <= 512) return 16;
   return 0;
 }
@@ -571,8 +578,8 @@ int ekv_tc_supported(const elitekv_layer* L, const elitekv_cache* cache) {
   if (n == 0) return 0;
   if ((L->n_h * r2) % 64 != 0 || L->n_h % 8 != 0) return 0;
   if ((n == 32 ? Smem<32>::total(L->d_c) : Smem<16>::total(L->d_c)) > L->smem_optin) return 0;
-  // the epilogue stages the whole fp32 output of a block ([d_c][n] floats) in the ring + rope area
-  if ((size_t)L->d_c * n * 4 > (size_t)kLatSlots * (kChunkBytes + n * 128) + (size_t)kRopeSlots * kChunkBytes) return 0;
+  // the epilogue cycles through kOutBufs staging tiles of [n][128] floats in the ring + rope area
+  if ((size_t)kOutBufs * n * 128 * 4 > (size_t)kLatSlots * (kChunkBytes + n * 128) + (size_t)kRopeSlots * kChunkBytes) return 0;
   if (cache && cache->page_table && (cache->page_size % 64 != 0)) return 0;
   return 1;
 }

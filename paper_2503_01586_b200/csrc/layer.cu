@@ -127,6 +127,9 @@ extern "C" int elitekv_layer_create(const elitekv_params* p, elitekv_layer** out
       regroup_wuk_kernel<<<grid2, block>>>((const bf16*)p->W_down, L->d_WcatT + (size_t)rope_w * p->d, p->d, p->d_c);
       if (cudaGetLastError() != cudaSuccess) break;
     }
+    if (cudaStreamCreateWithFlags(&L->side, cudaStreamNonBlocking) != cudaSuccess) break;
+    if (cudaEventCreateWithFlags(&L->ev_fork, cudaEventDisableTiming) != cudaSuccess) break;
+    if (cudaEventCreateWithFlags(&L->ev_join, cudaEventDisableTiming) != cudaSuccess) break;
     if (cudaDeviceSynchronize() != cudaSuccess) break;
     rc = ELITEKV_OK;
   } while (0);
@@ -148,6 +151,9 @@ extern "C" int elitekv_layer_destroy(elitekv_layer* L) {
   cudaFree(L->d_WukT);
   cudaFree(L->d_Wuv);
   cudaFree(L->d_WcatT);
+  if (L->side) cudaStreamDestroy(L->side);
+  if (L->ev_fork) cudaEventDestroy(L->ev_fork);
+  if (L->ev_join) cudaEventDestroy(L->ev_join);
   if (L->prof) {
     for (int i = 0; i < 2 * kProfileSlots; ++i)
       if (L->prof->ev[i]) cudaEventDestroy(L->prof->ev[i]);

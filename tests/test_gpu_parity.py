@@ -157,6 +157,24 @@ def test_project_append_other_shapes(ek):
     _projection_case(ek, gen.shrink(gen.LLAMA13B_75, B=2, ctx=140), 5120, [1, 140], False, 94)
 
 
+@pytest.mark.parametrize("paged", [False, True])
+@pytest.mark.parametrize("lens", [[1] * 16, [40, 37, 51], [1], [17, 100]], ids=["b16", "128tok", "1tok", "117tok"])
+def test_project_append_decode_batches_split_depth(ek, lens, paged):
+    """At most 128 tokens (a decode step's batch): the call runs as clusters of 8 blocks that
+    split the depth d and exchange partial sums through distributed shared memory.  One token,
+    a batch of 16 one-token sequences, a full tile of 128 and a ragged 117 (the rows a block
+    finishes, 16 per block, end inside block 7)."""
+    _projection_case(ek, gen.shrink(gen.LLAMA7B_75, B=len(lens), ctx=max(lens) + 1), 4096, lens, paged, 96 + paged)
+
+
+def test_project_append_split_depth_uneven_shares(ek):
+    """d = 5120: 80 depth stages over 8 blocks (10 each); d = 1024 at d_c = 768: 16 stages, 2 each;
+    d = 576: 9 stages, shares of 1 and 2."""
+    _projection_case(ek, gen.shrink(gen.LLAMA13B_75, B=2, ctx=30), 5120, [30, 9], False, 97)
+    _projection_case(ek, gen.shrink(gen.SWEEP_875, B=2, ctx=60), 1024, [60, 60], False, 98)
+    _projection_case(ek, gen.shrink(gen.SWEEP_875, B=1, ctx=5), 576, [5], False, 99)
+
+
 def test_project_append_needs_projection_weights_and_a_covered_shape(ek):
     w = replace(SMALL, seed=95)
     st = H.setup(w, lens=[5, 5, 5])
@@ -348,6 +366,103 @@ def test_back_to_back_steps_share_one_workspace(ek):
         assert torch.equal(o1, alone1)
         assert torch.equal(o2, alone2)
     H.check_parity(st, alone1, H.all_units(st))
+
+
+def _step_state(ek, paged):
+    """A cache filled up to, not including, the decoding tokens, and the step's own inputs."""
+    w = gen.shrink(gen.LLAMA7B_75, B=4, ctx=700)
+    if paged:
+        w = replace(w, paged=True, page_size=64)
+    lens = [700, 257, 129, 1]
+    st = H.setup(w, lens=lens, fill=False)
+    last = torch.tensor([int(st.starts[b + 1]) - 1 for b in range(4)], device="cuda")
+    keep = torch.ones(int(st.starts[-1]), dtype=torch.bool, device="cuda")
+    keep[last] = False
+    ek.elitekv_append(st.layer, st.cache, st.k_e[keep], st.c[keep], st.seq_id[keep], st.pos[keep])
+    new = {"k_e": st.k_e[last].contiguous(), "c": st.c[last].contiguous(),
+           "seq_id": st.seq_id[last].contiguous(), "pos": st.pos[last].contiguous()}
+    return w, st, new
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_single_call_step_equals_the_three_calls(ek, paged):
+    """elitekv_decode_step (append and plan on the layer's second stream, joined before the
+    attention kernel) against append -> absorb -> decode on one stream: same cache rows, same
+    output bits, several steps queued back to back without a synchronisation, and parity with the
+    oracle from the raw inputs."""
+    w, st, new = _step_state(ek, paged)
+    q_rope = torch.empty((4, w.n_h, 2 * w.r), dtype=torch.bfloat16, device="cuda")
+    q_abs = torch.empty((4, w.n_h, w.d_c), dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros((4, w.n_h, w.d_h), dtype=torch.bfloat16, device="cuda")
+    for _ in range(3):
+        ek.elitekv_decode_step(st.layer, st.cache, new["k_e"], new["c"], new["seq_id"], new["pos"], st.q,
+                               st.lens_dev, q_rope, q_abs, st.workspace, out)
+    torch.cuda.synchronize()
+    assert ek.elitekv_check_status(st.layer) == 0
+    rope_rows, lat_rows = st.rope_plane.clone(), st.latent_plane.clone()
+    # the three calls on a cache that is built the same way
+    w2, st2, new2 = _step_state(ek, paged)
+    ek.elitekv_append(st2.layer, st2.cache, new2["k_e"], new2["c"], new2["seq_id"], new2["pos"])
+    want = H.run_decode(st2)
+    assert torch.equal(st2.rope_plane, rope_rows) and torch.equal(st2.latent_plane, lat_rows)
+    assert torch.equal(out, want)
+    H.check_parity(st, out, H.sample_units(st, 48, seed=5))
+
+
+def test_single_call_step_replays_from_a_cuda_graph(ek):
+    """The fork to the layer's second stream and the join are event edges, so the whole step
+    can be captured from the caller's stream alone."""
+    w, st, new = _step_state(ek, False)
+    q_live = st.q.clone()
+    q_rope = torch.empty((4, w.n_h, 2 * w.r), dtype=torch.bfloat16, device="cuda")
+    q_abs = torch.empty((4, w.n_h, w.d_c), dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros((4, w.n_h, w.d_h), dtype=torch.bfloat16, device="cuda")
+
+    def one():
+        ek.elitekv_decode_step(st.layer, st.cache, new["k_e"], new["c"], new["seq_id"], new["pos"], q_live,
+                               st.lens_dev, q_rope, q_abs, st.workspace, out)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        one()
+        one()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    eager = out.clone()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        one()
+    out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, eager)
+    q_live.copy_(torch.flip(st.q, dims=[1]))
+    graph.replay()
+    torch.cuda.synchronize()
+    assert ek.elitekv_check_status(st.layer) == 0
+    want = H.run_decode(replace(st, q=q_live))
+    assert torch.equal(out, want)
+
+
+def test_step_runner_host_to_host(ek):
+    """The host-to-host runner (one packed copy in, the single-call step, one copy out; eager and
+    as a replayed CUDA graph) returns the bits of the same step made call by call."""
+    w, st, new = _step_state(ek, False)
+    runners = [ek.DecodeStepRunner(st.layer, st.cache, 4, "cuda", graph=g) for g in (False, True)]
+    w2, st2, new2 = _step_state(ek, False)
+    ek.elitekv_append(st2.layer, st2.cache, new2["k_e"], new2["c"], new2["seq_id"], new2["pos"])
+    want = H.run_decode(st2).cpu()
+    for r in runners:
+        assert r.h2d_bytes >= sum(v.numel() * v.element_size() for v in r.host.values())
+        for k, v in (("k_e", new["k_e"]), ("c", new["c"]), ("seq_id", new["seq_id"]), ("pos", new["pos"]),
+                     ("q", st.q), ("lens", st.lens_dev)):
+            r.host[k].copy_(v.cpu().view(r.host[k].shape))
+        for _ in range(3):       # eager, capture + replay, replay
+            r.out_host.zero_()
+            got = r.run()
+            assert torch.equal(got, want)
+    assert runners[0].graph is None and runners[1].graph is not None
+    assert ek.elitekv_check_status(st.layer) == 0
 
 
 KERNELS = [1, 2, 3]

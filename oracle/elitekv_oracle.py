@@ -313,6 +313,42 @@ def decode_from_raw(q, q_pos, k_e, pos, c, W_uk, W_uv, idx, d_h, base=10000.0, s
 
 
 # --------------------------------------------------------------------------------------------
+# Separated low-rank decomposition (S-LRD, Section 3.2): keys and values have their own latents
+# --------------------------------------------------------------------------------------------
+def decode_slrd(q, q_pos, k_rope, c_k, c_v, W_uk_S, W_uv_S, idx, d_h, base=10000.0, scale=None,
+                pair_mode=0, heads=None):
+    """Decode attention when W^k_e ~ A^k B^k_S and W^v ~ A^v B^v_S are factorised separately:
+    the cache holds c_k = x A^k [n][d_ck] and c_v = x A^v [n][d_cv] beside the rotated elite
+    rows; the un-rotated key dims of head h are c_k . B^k_S,h and its values c_v . B^v_S,h.
+    W_uk_S [d_ck][n_h (d_h-2r)], W_uv_S [d_cv][n_h d_h].  Returns [len(heads)][d_h]."""
+    k_rope = np.asarray(k_rope, dtype=F64)
+    c_k = np.asarray(c_k, dtype=F64)
+    c_v = np.asarray(c_v, dtype=F64)
+    W_uk_S = np.asarray(W_uk_S, dtype=F64)
+    W_uv_S = np.asarray(W_uv_S, dtype=F64)
+    n_h = np.asarray(idx).shape[0]
+    heads = list(range(n_h)) if heads is None else list(heads)
+    if c_k.shape[0] == 0:
+        return np.zeros((len(heads), d_h), dtype=F64)
+    scale = 1.0 / np.sqrt(F64(d_h)) if scale is None else F64(scale)
+    q_rope, q_nope = query_parts(q, q_pos, idx, d_h, base, pair_mode)
+    dn = q_nope.shape[1]
+    out = []
+    for h in heads:
+        K_nope = c_k @ W_uk_S[:, h * dn:(h + 1) * dn]        # [n][d_h-2r]
+        V = c_v @ W_uv_S[:, h * d_h:(h + 1) * d_h]           # [n][d_h]
+        s = k_rope[:, h, :] @ q_rope[h] + K_nope @ q_nope[h]
+        p = softmax_rows(scale * s[None, :])[0]
+        out.append(p @ V)
+    return np.stack(out)
+
+
+def cache_elements_per_token_slrd(n_h, r, d_ck, d_cv):
+    """KV-cache elements per token per layer under S-LRD (Section 3.2)."""
+    return 2 * r * n_h + d_ck + d_cv
+
+
+# --------------------------------------------------------------------------------------------
 # Uncompressed RoPE multi-head attention (Section 2.1 + 2.2): the comparator's definition
 # --------------------------------------------------------------------------------------------
 def mha_decode(q_hat, K_hat, V, scale=None, heads=None):

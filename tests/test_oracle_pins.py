@@ -398,3 +398,91 @@ def test_projection_properties_that_need_no_second_implementation():
     a_plain = np.arctan2(k_plain[1, :, 1], k_plain[1, :, 0])
     a_rot = np.arctan2(r1.reshape(T, n_h * r, 2)[1, :, 1], r1.reshape(T, n_h * r, 2)[1, :, 0])
     assert np.allclose(np.exp(1j * (a_rot - a_plain)), np.exp(1j * 3 * th))
+
+
+# ------------------------------------------------------------------ separated latents (S-LRD)
+def _slrd_case(seed, n_h=3, d_h=12, r=2, d_ck=7, d_cv=5, n=8):
+    g = _rng(seed)
+    dn = d_h - 2 * r
+    return dict(
+        idx=np.stack([g.permutation(d_h // 2)[:r] for _ in range(n_h)]).astype(np.int64),
+        q=g.standard_normal((n_h, d_h)), k_e=g.standard_normal((n, n_h, r, 2)),
+        c_k=g.standard_normal((n, d_ck)), c_v=g.standard_normal((n, d_cv)),
+        W_uk=g.standard_normal((d_ck, n_h * dn)), W_uv=g.standard_normal((d_cv, n_h * d_h)),
+        pos=np.sort(g.choice(40, n, replace=False)), q_pos=41, d_h=d_h, n_h=n_h, r=r, dn=dn, n=n)
+
+
+def test_slrd_is_textbook_rope_attention_on_the_reconstructed_keys_and_values():
+    """Section 3.2 (S-LRD): keys of a head = its elite chunks as cached plus c_k . B^k_S,h on the
+    other dims (un-rotated), values = c_v . B^v_S,h.  Rebuild full K and V by hand and run the
+    complex-number textbook attention with RoPE on the elite chunks only (the others get the
+    identity rotation: their positions are set to the query's, so the relative angle is zero)."""
+    z = _slrd_case(31)
+    n, n_h, d_h, r, dn = z["n"], z["n_h"], z["d_h"], z["r"], z["dn"]
+    k_rope = O.rotate_elite_keys(z["k_e"], z["pos"], z["idx"], d_h, 777.0)
+    got = O.decode_slrd(z["q"], z["q_pos"], k_rope, z["c_k"], z["c_v"], z["W_uk"], z["W_uv"], z["idx"], d_h,
+                        base=777.0)
+    want = np.zeros((n_h, d_h))
+    for h in range(n_h):
+        elite = [int(i) for i in z["idx"][h]]
+        rest = [d for d in range(d_h) if d // 2 not in elite]
+        Kn = z["c_k"] @ z["W_uk"][:, h * dn:(h + 1) * dn]
+        V = z["c_v"] @ z["W_uv"][:, h * d_h:(h + 1) * d_h]
+        s = []
+        for t in range(n):
+            acc = 0.0
+            for j, i in enumerate(elite):
+                th = 777.0 ** (-2.0 * i / d_h)
+                qh = complex(z["q"][h][2 * i], z["q"][h][2 * i + 1]) * cmath.exp(1j * z["q_pos"] * th)
+                kh = complex(z["k_e"][t][h][j][0], z["k_e"][t][h][j][1]) * cmath.exp(1j * z["pos"][t] * th)
+                acc += (qh * kh.conjugate()).real
+            for a, d in enumerate(rest):
+                acc += z["q"][h][d] * Kn[t][a]
+            s.append(acc / math.sqrt(d_h))
+        p = scipy.special.softmax(np.array(s))
+        want[h] = p @ V
+    assert np.allclose(got, want, atol=1e-12)
+    # a head subset, in the order asked for
+    sub = O.decode_slrd(z["q"], z["q_pos"], k_rope, z["c_k"], z["c_v"], z["W_uk"], z["W_uv"], z["idx"], d_h,
+                        base=777.0, heads=[2, 0])
+    assert np.allclose(sub, want[[2, 0]], atol=1e-12)
+
+
+def test_slrd_equals_the_joint_form_with_block_diagonal_up_projections():
+    """[c_k | c_v] with B^kv = diag(B^k_S, B^v_S) is a joint latent whose key half ignores c_v and
+    whose value half ignores c_k: the joint oracle on the stacked latent must agree.  Swapping
+    the two latents, or the two weights, breaks it."""
+    z = _slrd_case(32, d_ck=6, d_cv=9)
+    d_h = z["d_h"]
+    k_rope = O.rotate_elite_keys(z["k_e"], z["pos"], z["idx"], d_h)
+    got = O.decode_slrd(z["q"], z["q_pos"], k_rope, z["c_k"], z["c_v"], z["W_uk"], z["W_uv"], z["idx"], d_h)
+    c = np.concatenate([z["c_k"], z["c_v"]], axis=1)
+    W_uk = np.concatenate([z["W_uk"], np.zeros((9, z["W_uk"].shape[1]))], axis=0)
+    W_uv = np.concatenate([np.zeros((6, z["W_uv"].shape[1])), z["W_uv"]], axis=0)
+    want = O.decode(z["q"], z["q_pos"], k_rope, c, W_uk, W_uv, z["idx"], d_h)
+    assert np.allclose(got, want, atol=1e-12)
+    # equal latents and one shared pair of weights: S-LRD with c_k = c_v = c is J-LRD
+    z2 = _random_case(33)
+    k2 = O.rotate_elite_keys(z2["k_e"], z2["pos"], z2["idx"], z2["d_h"])
+    a = O.decode_slrd(z2["q"], z2["q_pos"], k2, z2["c"], z2["c"], z2["W_uk"], z2["W_uv"], z2["idx"], z2["d_h"])
+    b = O.decode(z2["q"], z2["q_pos"], k2, z2["c"], z2["W_uk"], z2["W_uv"], z2["idx"], z2["d_h"])
+    assert np.allclose(a, b, atol=1e-12)
+
+
+def test_slrd_special_cases_and_cache_size():
+    z = _slrd_case(34)
+    d_h = z["d_h"]
+    k_rope = O.rotate_elite_keys(z["k_e"], z["pos"], z["idx"], d_h)
+    # one cached token: the output is that token's value, whatever the scores
+    one = O.decode_slrd(z["q"], 5, k_rope[:1], z["c_k"][:1], z["c_v"][:1], z["W_uk"], z["W_uv"], z["idx"], d_h)
+    assert np.allclose(one, (z["c_v"][0] @ z["W_uv"]).reshape(z["n_h"], d_h), atol=1e-12)
+    # zero query: uniform attention, the mean of the values
+    flat = O.decode_slrd(np.zeros_like(z["q"]), 5, k_rope, z["c_k"], z["c_v"], z["W_uk"], z["W_uv"], z["idx"], d_h)
+    assert np.allclose(flat, (z["c_v"].mean(axis=0) @ z["W_uv"]).reshape(z["n_h"], d_h), atol=1e-12)
+    # empty cache
+    none = O.decode_slrd(z["q"], 0, k_rope[:0], z["c_k"][:0], z["c_v"][:0], z["W_uk"], z["W_uv"], z["idx"], d_h)
+    assert none.shape == (z["n_h"], d_h) and not none.any()
+    # cache elements per token (Section 3.2): 2 r n_h + d_ck + d_cv; with d_ck + d_cv = d_c it is the
+    # joint count
+    assert O.cache_elements_per_token_slrd(32, 8, 512, 1024) == 2 * 8 * 32 + 512 + 1024
+    assert O.cache_elements_per_token_slrd(32, 8, 512, 1024) == O.cache_elements_per_token(32, 8, 1536)

@@ -84,7 +84,15 @@ typedef struct {
   int32_t d;                  /* model width                                                   */
   const void* W_ke;           /* bf16 [d][n_h*2r]  columns of W^k of the elite chunks, head by
                                  head in the order of elite_idx, (even, odd) inside a chunk    */
-  const void* W_down;         /* bf16 [d][d_c]     A^kv                                        */
+  const void* W_down;         /* bf16 [d][d_c]     A^kv  (separated latents: [A^k | A^v])      */
+  /* Separated low-rank decomposition (S-LRD, Section 3.2): keys and values have latents of
+   * their own.  0: joint latent (J-LRD, everything above as written).  d_ck > 0: a latent row
+   * of the cache is [c_k (d_ck) | c_v (d_cv = d_c - d_ck)]; scores read c_k only, outputs c_v
+   * only; W_uk is B^k_S, bf16 [d_ck][n_h*(d_h-2r)], W_uv is B^v_S, bf16 [d_cv][n_h*d_h]; q_abs
+   * is [B][n_h][d_ck].  d_ck and d_cv must be multiples of 8 (the tcgen05 two-pass kernel wants
+   * multiples of 128; the resident-tile kernel does not serve separated latents).  The cache
+   * costs 2 r n_h + d_ck + d_cv elements per token. */
+  int32_t d_ck;
 } elitekv_params;
 
 /* The two cache planes.  Contiguous (page_table == NULL): sequence s, position p live in row
@@ -138,7 +146,7 @@ int elitekv_project_append(const elitekv_layer* layer, const elitekv_cache* cach
 /* Query preparation (score equation of Section 3.1; absorption of B^k, Section 5).
  *   q      bf16  [B][n_h][d_h]  un-rotated queries,  q_pos int32 [B]
  *   q_rope bf16  [B][n_h][2r]   elite chunks of q rotated at q_pos
- *   q_abs  bf16  [B][n_h][d_c]  q_nope[b,h,:] . W_uk,h^T, q_nope = the other d_h-2r dims of
+ *   q_abs  bf16  [B][n_h][d_c]  (separated latents: [B][n_h][d_ck])  q_nope[b,h,:] . W_uk,h^T, q_nope = the other d_h-2r dims of
  *                               q[b,h] in ascending order; fp32 accumulation. */
 int elitekv_absorb_query(const elitekv_layer* layer, const void* q, const int32_t* q_pos,
                          int32_t B, void* q_rope, void* q_abs, elitekv_stream_t stream);

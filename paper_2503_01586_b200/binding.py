@@ -38,7 +38,8 @@ class Params(C.Structure):
                 ("elite_idx", C.c_void_p), ("rope_base", C.c_float), ("softmax_scale", C.c_float),
                 ("pair_mode", C.c_int32), ("W_uk", C.c_void_p), ("W_uv", C.c_void_p),
                 ("max_pos", C.c_int32), ("cos_sin", C.c_void_p), ("decode_kernel", C.c_int32),
-                ("d", C.c_int32), ("W_ke", C.c_void_p), ("W_down", C.c_void_p)]
+                ("d", C.c_int32), ("W_ke", C.c_void_p), ("W_down", C.c_void_p),
+                ("d_ck", C.c_int32)]
 
 
 class CacheDesc(C.Structure):
@@ -122,10 +123,14 @@ class Layer:
     bf16 CUDA tensors; cos_sin an optional fp32 CUDA tensor [max_pos][d_h/2][2]."""
 
     def __init__(self, n_h, d_h, r, d_c, elite_idx, W_uk, W_uv, max_pos, rope_base=10000.0,
-                 softmax_scale=0.0, pair_mode=0, cos_sin=None, decode_kernel=0, W_ke=None, W_down=None):
+                 softmax_scale=0.0, pair_mode=0, cos_sin=None, decode_kernel=0, W_ke=None, W_down=None,
+                 d_ck=0):
         idx = elite_idx.to(torch.int32).contiguous().cpu()
         assert tuple(idx.shape) == (n_h, r)
         self.n_h, self.d_h, self.r, self.d_c = n_h, d_h, r, d_c
+        # separated latents (d_ck > 0): a latent row is [c_k (d_ck) | c_v (d_c - d_ck)]
+        self.d_ck = d_ck
+        self.kw = d_ck if d_ck > 0 else d_c          # width of the absorbed query
         self._keep = (idx, cos_sin)
         p = Params(n_h, d_h, r, d_c, idx.data_ptr() if r > 0 else None, rope_base, softmax_scale,
                    pair_mode, _ptr(W_uk) if W_uk is not None and W_uk.numel() else None,
@@ -134,7 +139,7 @@ class Layer:
                    decode_kernel,
                    W_down.shape[0] if W_down is not None else 0,
                    _ptr(_dev(W_ke, torch.bfloat16)) if W_ke is not None else None,
-                   _ptr(_dev(W_down, torch.bfloat16)) if W_down is not None else None)
+                   _ptr(_dev(W_down, torch.bfloat16)) if W_down is not None else None, d_ck)
         h = C.c_void_p()
         _check(lib().elitekv_layer_create(C.byref(p), C.byref(h)), "elitekv_layer_create")
         self.handle = h
@@ -193,7 +198,7 @@ def elitekv_absorb_query(layer: Layer, q, q_pos, q_rope=None, q_abs=None):
     if q_rope is None:
         q_rope = torch.empty((B, layer.n_h, 2 * layer.r), dtype=torch.bfloat16, device=q.device)
     if q_abs is None:
-        q_abs = torch.empty((B, layer.n_h, layer.d_c), dtype=torch.bfloat16, device=q.device)
+        q_abs = torch.empty((B, layer.n_h, layer.kw), dtype=torch.bfloat16, device=q.device)
     _check(lib().elitekv_absorb_query(layer.handle, _ptr(q), _ptr(_dev(q_pos, torch.int32)), B,
                                       _ptr(q_rope), _ptr(q_abs), _stream()), "elitekv_absorb_query")
     return q_rope, q_abs
@@ -264,7 +269,7 @@ class DecodeStepRunner:
                     for k in self.ORDER}
         self.host, self.dev = views(self.pack_host), views(self.pack_dev)
         self.q_rope = torch.empty((B, layer.n_h, 2 * layer.r), dtype=bf, device=device)
-        self.q_abs = torch.empty((B, layer.n_h, layer.d_c), dtype=bf, device=device)
+        self.q_abs = torch.empty((B, layer.n_h, layer.kw), dtype=bf, device=device)
         self.out = torch.empty((B, layer.n_h, layer.d_h), dtype=bf, device=device)
         self.out_host = torch.empty((B, layer.n_h, layer.d_h), dtype=bf).pin_memory()
         self.workspace = torch.empty(elitekv_decode_workspace_size(layer, B), dtype=torch.uint8, device=device)

@@ -12,7 +12,9 @@
 // per weight row, all issued at once by one warp, so the slab costs one trip to memory and
 // overlaps the gather of the queries.  The kernel is bound by latency, not by its 11 MB of
 // traffic or its 0.2 GFLOP.  The blocks of the last grid row do the query RoPE (three dependent
-// loads per element), off the path of the others.
+// loads per element), off the path of the others.  d_c below is the width of the latent the
+// scores read: the whole latent row, or the key latent d_ck when keys and values have latents of
+// their own (S-LRD, Section 3.2).
 #include "tc_ptx.cuh"
 
 namespace {
@@ -153,14 +155,15 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
 int ekv_launch_absorb(const elitekv_layer* L, const void* q, const int32_t* q_pos, int B,
                       void* q_rope, void* q_abs, cudaStream_t st) {
   if (B == 0) return ELITEKV_OK;
-  dim3 grid(L->n_h, (L->d_c + kAbsorbCoords - 1) / kAbsorbCoords + 1);   // + one row of rope blocks
+  // the absorbed query spans the latent columns the scores read (all of them, or the key latent)
+  dim3 grid(L->n_h, (L->kw + kAbsorbCoords - 1) / kAbsorbCoords + 1);   // + one row of rope blocks
   const int kpad = (L->dn + 15) & ~15;
   const size_t smem = sizeof(bf16) * ((size_t)kpad * kAbsorbPitch + (size_t)kAbsorbBatch * (kpad + 8)) + 16;
-  if ((int)smem > L->smem_optin || L->d_c % 8 != 0) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
+  if ((int)smem > L->smem_optin || L->kw % 8 != 0) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
   EKV_CUDA_OK(cudaFuncSetAttribute(absorb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   absorb_kernel<<<grid, kAbsorbThreads, smem, st>>>(
       (const bf16*)q, q_pos, B, L->d_WukT, L->d_qdims, L->d_idx, L->d_cs, (bf16*)q_rope,
-      (bf16*)q_abs, L->n_h, L->d_h, L->r, L->d_c, L->max_pos, L->d_status);
+      (bf16*)q_abs, L->n_h, L->d_h, L->r, L->kw, L->max_pos, L->d_status);
   EKV_CUDA_OK(cudaGetLastError());
   return ELITEKV_OK;
 }

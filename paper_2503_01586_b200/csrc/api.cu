@@ -73,7 +73,7 @@ Carve carve(const elitekv_layer* L, int B, int max_items) {
   c.off_items = o; o = align256(o + sizeof(int32_t) * 4 * (size_t)max_items);
   c.off_first = o; o = align256(o + sizeof(int32_t) * ((size_t)B + 1));
   c.off_ml = o;    o = align256(o + sizeof(float) * 2 * (size_t)max_items * L->n_h);
-  c.off_acc = o;   o = align256(o + sizeof(float) * (size_t)max_items * L->n_h * L->d_c);
+  c.off_acc = o;   o = align256(o + sizeof(float) * (size_t)max_items * L->n_h * L->vw);
   c.off_slice = o; o = align256(o + ekv_combine_scratch_bytes(L, B));
   c.off_cnt = o;   o = align256(o + sizeof(int32_t) * (size_t)ekv_combine_counters(L, B));
   c.off_wfirst = o; o = align256(o + sizeof(int32_t) * ((size_t)L->sm_count + 2));

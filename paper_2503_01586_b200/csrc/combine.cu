@@ -14,6 +14,9 @@
 // a fixed order and writes bf16, so the result does not depend on scheduling.
 //
 // Generic kernel: any even d_h <= 512, any d_c; block per (head, 8 sequences).
+//
+// With separated latents (S-LRD) the partial outputs span the value latent only; `d_c` below is
+// then d_cv and W_uv is B^v_S.
 #include "common.cuh"
 
 namespace {
@@ -294,11 +297,11 @@ combine_upproj_kernel(const float* __restrict__ part_acc, const float* __restric
 
 }  // namespace
 
-int ekv_combine_fast_ok(const elitekv_layer* L) { return L->d_h == kFD && L->d_c % kFK == 0; }
+int ekv_combine_fast_ok(const elitekv_layer* L) { return L->d_h == kFD && L->vw % kFK == 0; }
 
 size_t ekv_combine_scratch_bytes(const elitekv_layer* L, int B) {
   if (!ekv_combine_fast_ok(L)) return 0;
-  return sizeof(float) * (size_t)(L->d_c / kFK) * B * L->n_h * kFD;
+  return sizeof(float) * (size_t)(L->vw / kFK) * B * L->n_h * kFD;
 }
 
 int ekv_combine_counters(const elitekv_layer* L, int B) {
@@ -308,10 +311,10 @@ int ekv_combine_counters(const elitekv_layer* L, int B) {
 int ekv_launch_combine(const elitekv_layer* L, int B, const DecodeScratch& ws, void* out,
                        cudaStream_t st) {
   if (ekv_combine_fast_ok(L)) {
-    dim3 grid(L->n_h, L->d_c / kFK);
+    dim3 grid(L->n_h, L->vw / kFK);
     EKV_CUDA_OK(ekv_launch_pdl(combine_fast_kernel, grid, dim3(kFThreads), 0, st, (const float*)ws.part_acc,
                                (const float*)ws.part_ml, (const int32_t*)ws.seq_first, (const bf16*)L->d_Wuv,
-                               ws.slice_out, ws.counters, (bf16*)out, B, L->n_h, L->d_c));
+                               ws.slice_out, ws.counters, (bf16*)out, B, L->n_h, L->vw));
     EKV_CUDA_OK(cudaGetLastError());
     return ELITEKV_OK;
   }
@@ -324,7 +327,7 @@ int ekv_launch_combine(const elitekv_layer* L, int B, const DecodeScratch& ws, v
                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   combine_upproj_kernel<<<grid, kCombThreads, smem, st>>>(ws.part_acc, ws.part_ml, ws.seq_first,
                                                           L->d_Wuv, (bf16*)out, B, L->n_h, L->d_h,
-                                                          L->d_c);
+                                                          L->vw);
   EKV_CUDA_OK(cudaGetLastError());
   return ELITEKV_OK;
 }

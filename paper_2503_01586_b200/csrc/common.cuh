@@ -16,7 +16,9 @@ typedef __nv_bfloat162 bf162;
 #define ELITEKV_TILE_TOKENS 64
 
 struct elitekv_layer {
-  int n_h, d_h, r, d_c, dn;        // dn = d_h - 2r (un-rotated key dims per head)
+  int n_h, d_h, r, d_c, dn;        // dn = d_h - 2r (un-rotated key dims per head); d_c = width of a latent row
+  int kw, voff, vw;                // latent columns the scores read: [0, kw); the outputs: [voff, voff + vw).
+                                   // Joint latent: kw = vw = d_c, voff = 0.  Separated: kw = d_ck, voff = d_ck, vw = d_cv.
   float rope_base;
   float scale;                     // softmax scale actually used
   int pair_mode;
@@ -30,8 +32,8 @@ struct elitekv_layer {
                                    // then the dn remaining dims ascending
   const float2* d_cs;              // [max_pos][d_h/2] (cos, sin)
   float2* d_cs_owned;              // same pointer when the library built the table
-  bf16* d_WukT;                    // [n_h][dn][d_c]: W_uk regrouped per head, d_c contiguous
-  bf16* d_Wuv;                     // [d_c][n_h*d_h] private copy
+  bf16* d_WukT;                    // [n_h][dn][kw]: W_uk regrouped per head, latent axis contiguous
+  bf16* d_Wuv;                     // [vw][n_h*d_h] private copy
   int32_t* d_status;               // [4] device status word: code, detail0, detail1, count
   struct EkvProfile* prof;         // optional event pairs around the split-K kernel
   int32_t* last_detail;            // host [3]: detail words + count read by the last check_status
@@ -165,9 +167,9 @@ struct DecodeScratch {
   int max_items;          // capacity of the plan
   int32_t* items;         // [max_items][4]
   int32_t* seq_first;     // [B+1]
-  float* part_acc;        // [max_items][n_h][d_c]
+  float* part_acc;        // [max_items][n_h][vw]
   float* part_ml;         // [max_items][n_h][2]  (running max in log2 units, running sum)
-  float* slice_out;       // combine: per latent slice partial outputs [d_c/128][B][n_h][128]
+  float* slice_out;       // combine: per latent slice partial outputs [vw/128][B][n_h][128]
   int32_t* counters;      // combine: arrival counters, zeroed by the plan kernel
   int n_counters;
   int32_t* worker_first;  // balanced plan: [n_workers+1] first item of each worker

@@ -25,12 +25,13 @@ struct GenericArgs {
   const bf16* latent;
   CacheView cv;
   const bf16* q_rope;     // [B][n_h][2r]
-  const bf16* q_abs;      // [B][n_h][d_c]
+  const bf16* q_abs;      // [B][n_h][kw]
   const int32_t* items;   // [max_items][4]
   float* part_acc;
   float* part_ml;
   int32_t* status;
   int n_h, r2, d_c, sub_tokens;
+  int kw, voff, vw;       // latent columns of the scores [0, kw) and of the outputs [voff, voff + vw)
   float scale_log2e;
 };
 
@@ -64,7 +65,8 @@ decode_generic_kernel(const GenericArgs a) {
   for (int ch = 0; ch < NCH; ++ch) {
     const int d = (ch * 32 + lane) * 8;
     uint4 v = make_uint4(0, 0, 0, 0);
-    if (active && d < d_c) v = *(const uint4*)(a.q_abs + ((size_t)seq * a.n_h + h) * d_c + d);
+    // columns the scores do not read (the value latent of S-LRD) get a zero query
+    if (active && d < a.kw) v = *(const uint4*)(a.q_abs + ((size_t)seq * a.n_h + h) * a.kw + d);
     qa[ch][0] = *(bf162*)&v.x; qa[ch][1] = *(bf162*)&v.y; qa[ch][2] = *(bf162*)&v.z; qa[ch][3] = *(bf162*)&v.w;
   }
 #pragma unroll
@@ -216,11 +218,11 @@ decode_generic_kernel(const GenericArgs a) {
   }
 
   if (active) {
-    float* pa = a.part_acc + ((size_t)item * a.n_h + h) * d_c;
+    float* pa = a.part_acc + ((size_t)item * a.n_h + h) * a.vw;
 #pragma unroll
     for (int ch = 0; ch < NCH; ++ch) {
-      const int d = (ch * 32 + lane) * 8;
-      if (d < d_c) {
+      const int d = (ch * 32 + lane) * 8 - a.voff;      // only the columns the outputs read leave the block
+      if (d >= 0 && d < a.vw) {
         *(float4*)(pa + d) = make_float4(acc[ch][0], acc[ch][1], acc[ch][2], acc[ch][3]);
         *(float4*)(pa + d + 4) = make_float4(acc[ch][4], acc[ch][5], acc[ch][6], acc[ch][7]);
       }
@@ -280,6 +282,9 @@ int ekv_launch_decode_generic(const elitekv_layer* L, const elitekv_cache* cache
   a.n_h = L->n_h;
   a.r2 = 2 * L->r;
   a.d_c = L->d_c;
+  a.kw = L->kw;
+  a.voff = L->voff;
+  a.vw = L->vw;
   a.sub_tokens = pick_sub_tokens(L);
   a.scale_log2e = L->scale * 1.4426950408889634f;
   const int rope_w_pad = (kHeadsPerBlock * a.r2 + 7) & ~7;

@@ -747,6 +747,7 @@ int ekv_rt_supported(const elitekv_layer* L, const elitekv_cache* cache) {
   const int r2 = 2 * L->r;
   if (L->n_h != kHeads) return 0;
   if (L->d_c % 256 != 0 || L->d_c > 1536) return 0;
+  if (L->kw != L->d_c || L->voff != 0) return 0;     // separated latents: nothing is read twice, the two-pass kernel serves them
   if (!(r2 == 8 || r2 == 16 || r2 == 32)) return 0;
   if (rt_ring_units(L) < L->d_c / 256 + 1) return 0;          // one tile resident plus a spare unit
   if (cache && cache->page_table && (cache->page_size % kT != 0)) return 0;

@@ -19,6 +19,9 @@
 // latents into the TMEM-resident output.  L2 eviction hints (keep after pass A, drop after pass
 // B) make the second read an L2 hit, so HBM sees every cache byte once per step.
 //
+// With separated latents (S-LRD, Section 3.2: a latent row is [c_k | c_v]) pass A streams only
+// the key latent's chunks and pass B only the value latent's, so nothing is read twice.
+//
 // A block is a persistent worker: it walks the items of the balanced plan that fall into its
 // share of the batch's tiles and writes one partial result (m, l, acc) per item.  Layers whose
 // fp32 output does not fit TMEM's 512 columns for 32 heads (d_c > 1920) run with 16 heads per
@@ -67,6 +70,7 @@ struct TcArgs {
   long long num_pages;
   int page_shift, page_mask, max_pages_per_seq;
   int n_h, d_c;
+  int kw, voff, vw;         // latent columns of the scores [0, kw) and of the outputs [voff, voff + vw)
   int n_groups;             // head groups of N heads; blockIdx.x = item * n_groups + group
   float scale_log2e;
 };
@@ -105,8 +109,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   const int h0 = (blockIdx.x % a.n_groups) * N;       // first head of this block's group
   const int nh_here = min(N, a.n_h - h0);
   const int d_c = a.d_c;
-  const int NKC = d_c >> 6;      // 64-wide latent chunks
-  const int NB = d_c >> 7;       // 128-row output blocks
+  const int NKC = a.kw >> 6;     // 64-wide latent chunks of pass A
+  const int NB = a.vw >> 7;      // 128-row output blocks = slot pairs of pass B
+  const int NUSE = NKC + 2 * NB; // ring uses per tile
+  const int vc0 = a.voff >> 6;   // first 64-wide chunk of the columns pass B reads
+  const bool reread = a.voff == 0;   // joint latent: pass B reads what pass A read
   constexpr int NRB = N * R2 / 64;   // rope boxes per tile
   constexpr int HPB = 64 / R2;       // heads per rope box
 
@@ -224,10 +231,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       const bool whole = halves == 2 && row[1] == row[0] + 64;
       if (!rope_role) {
         // ring uses of this tile: NKC chunks of pass A (each with its query chunk), then the
-        // same NKC chunks again for pass B (served by L2)
-        for (int u = prod; u < 2 * NKC; u += kProdWarps) {
+        // 2 NB chunks of pass B (joint latent: the same chunks again, served by L2)
+        for (int u = prod; u < NUSE; u += kProdWarps) {
           const bool with_q = u < NKC;
-          const int kc = with_q ? u : u - NKC;
+          const int kc = with_q ? u : vc0 + u - NKC;
           const unsigned n = lat_n + (unsigned)u, slot = n % kLatSlots;
           const uint32_t eb = smem_u32(&bars->lat_empty[slot]), epar = ((n / kLatSlots) & 1) ^ 1;
           ok = warp_wait(eb, epar, s_abort, 1);
@@ -237,7 +244,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
             mbar_expect_tx(fb, (uint32_t)(halves * 8192 + (with_q ? N * 128 : 0)));
             if (with_q)   // the sequence's absorbed queries for these 64 latent coordinates (L2-resident)
               tma_load_2d_hint(smem_u32(s_lat + slot * kSlot + kChunkBytes), &map_q, kc * 64, seq * a.n_h + h0, fb, pol_keep);
-            const uint64_t pol = with_q ? pol_keep : pol_drop;
+            const uint64_t pol = (with_q && reread) ? pol_keep : pol_drop;
             if (whole) {
               tma_load_2d_hint(smem_u32(s_lat + slot * kSlot), &map_lat128, kc * 64, (int)row[0], fb, pol);
             } else {
@@ -247,7 +254,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
           }
           __syncwarp();
         }
-        lat_n += 2u * (unsigned)NKC;
+        lat_n += (unsigned)NUSE;
       } else {
         // warp 6: the rope boxes of the tile
         for (int cb = 0; cb < NRB; ++cb) {
@@ -360,7 +367,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       if (!ok) break;
       if (elect_one()) tc_commit(smem_u32(&bars->pv_done));
       __syncwarp();
-      lat_n = n0 + 2u * (unsigned)NKC;
+      lat_n = n0 + (unsigned)NUSE;
     }
   }
   // ============================================================== warps 2-5: softmax
@@ -564,7 +571,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
 // as head groups (the last one partly filled: 40 heads = 32 + 8); each group streams the token
 // tile itself, and the groups of an item are adjacent blocks so that the later readers hit L2.
 static int tc_pick_n(const elitekv_layer* L) {
-  const int nb = L->d_c / 128;
+  const int nb = L->vw / 128;
   if ((nb + 1) * 32 <= 512) return 32;
   if ((nb + 1) * 16 <= 512) return 16;
   return 0;
@@ -572,7 +579,8 @@ static int tc_pick_n(const elitekv_layer* L) {
 
 int ekv_tc_supported(const elitekv_layer* L, const elitekv_cache* cache) {
   const int r2 = 2 * L->r;
-  if (L->d_c % 128 != 0) return 0;
+  // pass A takes 64-wide chunks, pass B slot pairs that must start on an even ring use
+  if (L->kw % 128 != 0 || L->vw % 128 != 0) return 0;
   if (!(r2 == 8 || r2 == 16 || r2 == 32)) return 0;
   const int n = tc_pick_n(L);
   if (n == 0) return 0;
@@ -606,8 +614,8 @@ int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, con
   if (rc == ELITEKV_OK) rc = make_map(&m_lat128, cache->latent, rows, L->d_c, 128);
   if (rc == ELITEKV_OK) rc = make_map(&m_rope128, cache->rope, rows, (unsigned long long)L->n_h * 2 * L->r, 128);
   const int N = tc_pick_n(L);
-  if (rc == ELITEKV_OK) rc = make_map(&m_q, q_abs, (unsigned long long)B * L->n_h, L->d_c, N);
-  if (rc == ELITEKV_OK) rc = make_map_f32_3d(&m_part, ws.part_acc, L->d_c, L->n_h, (unsigned long long)ws.max_items, N);
+  if (rc == ELITEKV_OK) rc = make_map(&m_q, q_abs, (unsigned long long)B * L->n_h, L->kw, N);
+  if (rc == ELITEKV_OK) rc = make_map_f32_3d(&m_part, ws.part_acc, L->vw, L->n_h, (unsigned long long)ws.max_items, N);
   if (rc != ELITEKV_OK) return rc;
   TcArgs a;
   a.items = ws.items;
@@ -624,6 +632,9 @@ int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, con
   a.max_pages_per_seq = cv.max_pages_per_seq;
   a.n_h = L->n_h;
   a.d_c = L->d_c;
+  a.kw = L->kw;
+  a.voff = L->voff;
+  a.vw = L->vw;
   a.n_groups = tc_groups(L);
   a.scale_log2e = L->scale * 1.4426950408889634f;
   const int smem = N == 32 ? Smem<32>::total(L->d_c) : Smem<16>::total(L->d_c);

@@ -40,6 +40,8 @@ extern "C" int elitekv_layer_create(const elitekv_params* p, elitekv_layer** out
   if (p->pair_mode != 0 && p->pair_mode != 1) return ELITEKV_ERR_INVALID_ARG;
   if (p->decode_kernel < 0 || p->decode_kernel > 3) return ELITEKV_ERR_INVALID_ARG;
   if (p->d_c % 8 != 0 || p->d_h > 512) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
+  if (p->d_ck < 0 || p->d_ck >= p->d_c) return ELITEKV_ERR_INVALID_ARG;
+  if (p->d_ck % 8 != 0) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
   if (((uintptr_t)p->W_uv & 15) || ((uintptr_t)p->W_uk & 15)) return ELITEKV_ERR_INVALID_ARG;
   if (p->d < 0 || (p->d > 0 && (!p->W_down || (p->r > 0 && !p->W_ke)))) return ELITEKV_ERR_INVALID_ARG;
   const int n_h = p->n_h, d_h = p->d_h, r = p->r, half = d_h / 2;
@@ -66,6 +68,9 @@ extern "C" int elitekv_layer_create(const elitekv_params* p, elitekv_layer** out
   elitekv_layer* L = (elitekv_layer*)calloc(1, sizeof(elitekv_layer));
   if (!L) return ELITEKV_ERR_CUDA;
   L->n_h = n_h; L->d_h = d_h; L->r = r; L->d_c = p->d_c; L->dn = d_h - 2 * r;
+  L->kw = p->d_ck > 0 ? p->d_ck : p->d_c;
+  L->voff = p->d_ck > 0 ? p->d_ck : 0;
+  L->vw = p->d_c - L->voff;
   L->rope_base = p->rope_base;
   L->scale = p->softmax_scale > 0.f ? p->softmax_scale : (float)(1.0 / sqrt((double)d_h));
   L->pair_mode = p->pair_mode; L->max_pos = p->max_pos; L->decode_kernel = p->decode_kernel;
@@ -102,14 +107,14 @@ extern "C" int elitekv_layer_create(const elitekv_params* p, elitekv_layer** out
       L->d_cs = L->d_cs_owned;
     }
 
-    size_t wuv_elems = (size_t)p->d_c * n_h * d_h;
+    size_t wuv_elems = (size_t)L->vw * n_h * d_h;
     if (cudaMalloc(&L->d_Wuv, wuv_elems * sizeof(bf16)) != cudaSuccess) break;
     if (cudaMemcpy(L->d_Wuv, p->W_uv, wuv_elems * sizeof(bf16), cudaMemcpyDeviceToDevice) != cudaSuccess) break;
     if (L->dn > 0) {
-      size_t wuk_elems = (size_t)p->d_c * n_h * L->dn;
+      size_t wuk_elems = (size_t)L->kw * n_h * L->dn;
       if (cudaMalloc(&L->d_WukT, wuk_elems * sizeof(bf16)) != cudaSuccess) break;
-      dim3 grid((n_h * L->dn + 31) / 32, (p->d_c + 31) / 32), block(32, 8);
-      regroup_wuk_kernel<<<grid, block>>>((const bf16*)p->W_uk, L->d_WukT, p->d_c, n_h * L->dn);
+      dim3 grid((n_h * L->dn + 31) / 32, (L->kw + 31) / 32), block(32, 8);
+      regroup_wuk_kernel<<<grid, block>>>((const bf16*)p->W_uk, L->d_WukT, L->kw, n_h * L->dn);
       if (cudaGetLastError() != cudaSuccess) break;
     }
     if (p->d > 0) {

@@ -46,17 +46,21 @@ class State:
     lens_dev: torch.Tensor
     workspace: torch.Tensor
     pos_offset: int = 0
+    d_ck: int = 0                # > 0: separated latents, a latent row is [c_k (d_ck) | c_v]
 
 
 def setup(w: gen.Workload, *, lens: Optional[Sequence[int]] = None, decode_kernel: int = 0,
           pos_offset: int = 0, cos_sin=None, fill: bool = True, device="cuda",
-          q_scale: float = 1.0, edit_tokens=None) -> State:
+          q_scale: float = 1.0, edit_tokens=None, d_ck: int = 0) -> State:
     """Builds layer, cache planes and the token stream; when `fill`, appends every token of
     every sequence (so the cache holds lens[b] tokens, the last being the decoding token).
     `q_scale` multiplies the drawn queries (exactly, for a power of two); `edit_tokens(st)` may
     overwrite rows of st.k_e / st.c before they are appended."""
     idx = gen.elite_index_sets(w)
     W_uk, W_uv = gen.up_projections(w, device)
+    if d_ck:
+        # S-LRD: B^k_S reads the first d_ck latent columns, B^v_S the remaining ones
+        W_uk, W_uv = W_uk[:d_ck].contiguous(), W_uv[d_ck:].contiguous()
     lens_t = gen.sequence_lengths(w) if lens is None else torch.tensor(list(lens), dtype=torch.int32)
     B = w.B
     assert lens_t.numel() == B
@@ -77,7 +81,7 @@ def setup(w: gen.Workload, *, lens: Optional[Sequence[int]] = None, decode_kerne
         tab = O.rope_table_f32(max_pos + pos_offset, w.d_h, w.rope_base)[pos_offset:]
         cos_sin = torch.from_numpy(np.ascontiguousarray(tab)).to(device)
     layer = ek.Layer(w.n_h, w.d_h, w.r, w.d_c, idx, W_uk, W_uv, max_pos, rope_base=w.rope_base,
-                     cos_sin=cos_sin, decode_kernel=decode_kernel)
+                     cos_sin=cos_sin, decode_kernel=decode_kernel, d_ck=d_ck)
     rope_w = w.n_h * 2 * w.r
     if w.paged:
         table, num_pages = gen.page_table(w, lens_t, headroom_tokens=1)
@@ -96,7 +100,7 @@ def setup(w: gen.Workload, *, lens: Optional[Sequence[int]] = None, decode_kerne
     ws = torch.empty(ek.elitekv_decode_workspace_size(layer, B), dtype=torch.uint8, device=device)
     st = State(w, idx, W_uk, W_uv, lens_t, starts, k_e, c, seq_id.to(device), pos.to(device), q,
                q_pos.to(torch.int32).to(device), layer, cache, rope_plane, latent_plane, page_table,
-               lens_t.to(device), ws, pos_offset)
+               lens_t.to(device), ws, pos_offset, d_ck)
     if edit_tokens is not None:
         edit_tokens(st)
     if fill and N:
@@ -130,8 +134,13 @@ def oracle_units(st: State, units: Sequence[Tuple[int, int]]) -> np.ndarray:
         posv = np.arange(hi - lo) + st.pos_offset
         q = f64(st.q[b])
         heads = [h for _, h in lst]
-        o = O.decode_from_raw(q, int(max(hi - lo - 1, 0)) + st.pos_offset, k_e, posv, c, W_uk, W_uv,
-                              idx, w.d_h, base=w.rope_base, heads=heads)
+        q_pos = int(max(hi - lo - 1, 0)) + st.pos_offset
+        if st.d_ck:
+            k_rope = O.rotate_elite_keys(k_e, posv, idx, w.d_h, w.rope_base)
+            o = O.decode_slrd(q, q_pos, k_rope, c[:, :st.d_ck], c[:, st.d_ck:], W_uk, W_uv, idx, w.d_h,
+                              base=w.rope_base, heads=heads)
+        else:
+            o = O.decode_from_raw(q, q_pos, k_e, posv, c, W_uk, W_uv, idx, w.d_h, base=w.rope_base, heads=heads)
         for (u, _), row in zip(lst, o):
             res[u] = row
     return np.stack(res)

@@ -191,6 +191,51 @@ def test_project_append_needs_projection_weights_and_a_covered_shape(ek):
     assert e.value.code == ek.ERR_UNSUPPORTED_SHAPE
 
 
+# ------------------------------------------------------------------ separated latents (S-LRD)
+@pytest.mark.parametrize("kernel", [1, 2], ids=["generic", "two-pass"])
+@pytest.mark.parametrize("d_ck", [512, 1024, 128])
+@pytest.mark.parametrize("paged", [False, True])
+def test_decode_separated_latents_7b_shape(ek, kernel, d_ck, paged):
+    """S-LRD (Section 3.2) at the 7B 75 % cache size: a latent row is [c_k (d_ck) | c_v (1536 - d_ck)],
+    scores read c_k through B^k_S, outputs read c_v through B^v_S.  All (sequence, head) units
+    against the float64 oracle; several tiles, ragged tails, a one-token and an empty sequence."""
+    w = gen.shrink(gen.LLAMA7B_75, B=5, ctx=700)
+    if paged:
+        w = replace(w, paged=True, page_size=64)
+    st = H.setup(w, lens=[700, 385, 128, 1, 0], decode_kernel=kernel, d_ck=d_ck)
+    assert ek.elitekv_decode_plan_info(st.layer, st.cache, 5)[0] == kernel
+    out = H.run_decode(st)
+    assert not out[4].any()
+    H.check_parity(st, out, [(b, h) for b in range(4) for h in range(w.n_h)])
+
+
+def test_decode_separated_latents_choice_and_other_shapes(ek):
+    """Left to itself the library serves separated latents with the two-pass kernel (nothing is
+    read twice there); the resident-tile kernel refuses them; widths the tensor-core kernel does
+    not cover (multiples of 8, not of 128) go to the generic kernel.  13B-like: 40 heads."""
+    w = gen.shrink(gen.LLAMA7B_75, B=2, ctx=300)
+    st = H.setup(w, lens=[300, 77], d_ck=768)
+    assert ek.elitekv_decode_plan_info(st.layer, st.cache, 2)[0] == 2
+    H.check_parity(st, H.run_decode(st), H.sample_units(st, 24, seed=2))
+    with pytest.raises(ek.ElitekvError) as e:
+        H.run_decode(H.setup(w, lens=[300, 77], d_ck=768, decode_kernel=3))
+    assert e.value.code == ek.ERR_UNSUPPORTED_SHAPE
+    st = H.setup(w, lens=[300, 77], d_ck=200)
+    assert ek.elitekv_decode_plan_info(st.layer, st.cache, 2)[0] == 1
+    H.check_parity(st, H.run_decode(st), H.sample_units(st, 24, seed=3))
+    w13 = gen.shrink(gen.LLAMA13B_75, B=2, ctx=260)
+    st = H.setup(w13, lens=[260, 129], d_ck=640)
+    H.check_parity(st, H.run_decode(st), H.sample_units(st, 40, seed=4))
+
+
+def test_separated_latents_bad_widths_are_rejected(ek):
+    w = gen.shrink(gen.LLAMA7B_75, B=1, ctx=10)
+    for d_ck, code in ((1536, "ERR_INVALID_ARG"), (-8, "ERR_INVALID_ARG"), (100, "ERR_UNSUPPORTED_SHAPE")):
+        with pytest.raises(ek.ElitekvError) as e:
+            H.setup(w, lens=[10], d_ck=d_ck, fill=False)
+        assert e.value.code == getattr(ek, code)
+
+
 # ------------------------------------------------------------------ query preparation
 @pytest.mark.parametrize("pair_mode", [0, 1])
 def test_absorb_query(ek, pair_mode):

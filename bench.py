@@ -211,11 +211,13 @@ def build_workload(w: gen.Workload, ek, device, decode_kernel: int = 0):
     """Cache prefilled with len-1 tokens per sequence; the step appends the last one."""
     idx = gen.elite_index_sets(w)
     W_uk, W_uv = gen.up_projections(w, device)
+    if w.d_ck:      # separated latents: B^k_S reads the first d_ck latent columns, B^v_S the rest
+        W_uk, W_uv = W_uk[:w.d_ck].contiguous(), W_uv[w.d_ck:].contiguous()
     lens = gen.sequence_lengths(w)                       # tokens INCLUDING the decoded one
     B = w.B
     max_pos = int(lens.max()) + 1
     layer = ek.Layer(w.n_h, w.d_h, w.r, w.d_c, idx, W_uk, W_uv, max_pos, rope_base=w.rope_base,
-                     decode_kernel=decode_kernel)
+                     decode_kernel=decode_kernel, d_ck=w.d_ck)
     rope_w = w.n_h * 2 * w.r
     page_table = None
     if w.paged:
@@ -252,7 +254,7 @@ def build_workload(w: gen.Workload, ek, device, decode_kernel: int = 0):
     ws = torch.empty(ek.elitekv_decode_workspace_size(layer, B), dtype=torch.uint8, device=device)
     bufs = {
         "q_rope": torch.empty((B, w.n_h, 2 * w.r), dtype=torch.bfloat16, device=device),
-        "q_abs": torch.empty((B, w.n_h, w.d_c), dtype=torch.bfloat16, device=device),
+        "q_abs": torch.empty((B, w.n_h, layer.kw), dtype=torch.bfloat16, device=device),
         "out": torch.empty((B, w.n_h, w.d_h), dtype=torch.bfloat16, device=device),
         "out_host": torch.empty((B, w.n_h, w.d_h), dtype=torch.bfloat16).pin_memory(),
     }
@@ -270,7 +272,7 @@ def step(ek, layer, cache, d, ws, bufs):
 KERNELS_PER_STEP = 5   # append, absorb, plan, split-K attention, combine + up-projection
 
 SWEEP = ["7b-75pct-paged-b64-ragged", "13b-75pct-b32-ctx16384", "7b-50pct-b32-ctx8192",
-         "7b-75pct-b32-ctx8192", "7b-87.5pct-b32-ctx8192"]
+         "7b-75pct-b32-ctx8192", "7b-87.5pct-b32-ctx8192", "7b-75pct-slrd512+1024-b32-ctx8192"]
 
 
 def sweep_entry(ek, w: gen.Workload, device, flush, steps: int = 10, n_check: int = 2):
@@ -316,8 +318,13 @@ def sweep_entry(ek, w: gen.Workload, device, flush, steps: int = 10, n_check: in
         c = torch.cat([c.cpu(), host["c"][b:b + 1]]).double().numpy()
         h = int(g.integers(w.n_h))
         t0 = time.perf_counter()
-        want = O.decode_from_raw(host["q"][b].double().numpy(), n - 1, k_e, np.arange(n), c, W_uk, W_uv,
-                                 idx, w.d_h, base=w.rope_base, heads=[h])[0]
+        if w.d_ck:
+            k_rope = O.rotate_elite_keys(k_e, np.arange(n), idx, w.d_h, w.rope_base)
+            want = O.decode_slrd(host["q"][b].double().numpy(), n - 1, k_rope, c[:, :w.d_ck], c[:, w.d_ck:],
+                                 W_uk, W_uv, idx, w.d_h, base=w.rope_base, heads=[h])[0]
+        else:
+            want = O.decode_from_raw(host["q"][b].double().numpy(), n - 1, k_e, np.arange(n), c, W_uk, W_uv,
+                                     idx, w.d_h, base=w.rope_base, heads=[h])[0]
         t_cpu += time.perf_counter() - t0
         d = out[b, h] - want
         num += float(d @ d)

@@ -349,6 +349,44 @@ def cache_elements_per_token_slrd(n_h, r, d_ck, d_cv):
 
 
 # --------------------------------------------------------------------------------------------
+# Several query rows over the cache (prefill chunk, speculative tokens): causal attention
+# --------------------------------------------------------------------------------------------
+def attend_causal(q, q_pos, k_rope, key_pos, c, W_uk, W_uv, idx, d_h, base=10000.0, scale=None,
+                  pair_mode=0, heads=None):
+    """The score equation of Section 3.1 for general query position m and key position n, with
+    the causal rule of a decoder: query row i (q[i] at position q_pos[i]) sees the cached tokens
+    whose position key_pos[t] <= q_pos[i].  q [m][n_h][d_h], k_rope [n][n_h][2r] (cached rotated
+    rows), c [n][d_c].  Returns [m][len(heads)][d_h]; a row that sees no token is zero."""
+    q = np.asarray(q, dtype=F64)
+    k_rope = np.asarray(k_rope, dtype=F64)
+    c = np.asarray(c, dtype=F64)
+    W_uk = np.asarray(W_uk, dtype=F64)
+    W_uv = np.asarray(W_uv, dtype=F64)
+    key_pos = np.asarray(key_pos)
+    n_h = np.asarray(idx).shape[0]
+    heads = list(range(n_h)) if heads is None else list(heads)
+    m, n = q.shape[0], c.shape[0]
+    scale = 1.0 / np.sqrt(F64(d_h)) if scale is None else F64(scale)
+    out = np.zeros((m, len(heads), d_h), dtype=F64)
+    parts = [query_parts(q[i], int(q_pos[i]), idx, d_h, base, pair_mode) for i in range(m)]
+    for j, h in enumerate(heads):
+        dn = parts[0][1].shape[1]
+        K_nope = c @ W_uk[:, h * dn:(h + 1) * dn]              # [n][d_h-2r]
+        V = c @ W_uv[:, h * d_h:(h + 1) * d_h]                 # [n][d_h]
+        S = np.empty((m, n), dtype=F64)
+        for i in range(m):
+            q_rope, q_nope = parts[i]
+            S[i] = k_rope[:, h, :] @ q_rope[h] + K_nope @ q_nope[h]
+        for i in range(m):
+            seen = key_pos <= int(q_pos[i])
+            if not seen.any():
+                continue
+            p = softmax_rows((scale * S[i, seen])[None, :])[0]
+            out[i, j] = p @ V[seen]
+    return out
+
+
+# --------------------------------------------------------------------------------------------
 # Uncompressed RoPE multi-head attention (Section 2.1 + 2.2): the comparator's definition
 # --------------------------------------------------------------------------------------------
 def mha_decode(q_hat, K_hat, V, scale=None, heads=None):

@@ -31,6 +31,7 @@ class Workload:
     page_size: int = 64
     rope_base: float = 10000.0
     seed: int = 0
+    d_ck: int = 0       # > 0: separated latents, a latent row is [c_k (d_ck) | c_v (d_c - d_ck)]
 
     @property
     def cache_elems_per_token(self) -> int:
@@ -53,9 +54,11 @@ SWEEP_50 = Workload("7b-50pct-b32-ctx8192", n_h=32, d_h=128, r=16, d_c=3072, d=4
                     ctx=8192, seed=1005)
 SWEEP_75 = replace(SWEEP_50, name="7b-75pct-b32-ctx8192", r=8, d_c=1536)
 SWEEP_875 = replace(SWEEP_50, name="7b-87.5pct-b32-ctx8192", r=4, d_c=768)
+# the 75 % cache split into a key latent of 512 and a value latent of 1024 (S-LRD)
+SWEEP_75_SLRD = replace(SWEEP_75, name="7b-75pct-slrd512+1024-b32-ctx8192", d_ck=512)
 
 CONFIGS = {w.name: w for w in
-           (TINY, LLAMA7B_75, LLAMA7B_75_PAGED, LLAMA13B_75, SWEEP_50, SWEEP_75, SWEEP_875)}
+           (TINY, LLAMA7B_75, LLAMA7B_75_PAGED, LLAMA13B_75, SWEEP_50, SWEEP_75, SWEEP_875, SWEEP_75_SLRD)}
 
 
 def shrink(w: Workload, *, B: int, ctx: int, ctx_lo: Optional[int] = None) -> Workload:

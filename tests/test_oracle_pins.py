@@ -486,3 +486,59 @@ def test_slrd_special_cases_and_cache_size():
     # joint count
     assert O.cache_elements_per_token_slrd(32, 8, 512, 1024) == 2 * 8 * 32 + 512 + 1024
     assert O.cache_elements_per_token_slrd(32, 8, 512, 1024) == O.cache_elements_per_token(32, 8, 1536)
+
+
+# ------------------------------------------------------------------ several query rows, causal
+def test_causal_rows_match_the_library_attention_when_every_chunk_is_elite():
+    """Every chunk elite, latent = all heads' values, W_uv = I: the method is standard causal
+    RoPE attention.  Queries and keys are rotated here with complex arithmetic and handed to
+    torch's scaled_dot_product_attention (square causal mask: a prefill of n tokens)."""
+    n_h, d_h, n = 2, 8, 7
+    g = _rng(41)
+    q = g.standard_normal((n, n_h, d_h))
+    k = g.standard_normal((n, n_h, d_h))
+    v = g.standard_normal((n, n_h, d_h))
+    pos = np.arange(n)
+    idx = np.stack([g.permutation(d_h // 2) for _ in range(n_h)])
+    k_e = np.zeros((n, n_h, d_h // 2, 2))
+    for h in range(n_h):
+        for j, i in enumerate(idx[h]):
+            k_e[:, h, j, 0] = k[:, h, 2 * i]
+            k_e[:, h, j, 1] = k[:, h, 2 * i + 1]
+    k_rope = O.rotate_elite_keys(k_e, pos, idx, d_h, 300.0)
+    got = O.attend_causal(q, pos, k_rope, pos, v.reshape(n, n_h * d_h), np.zeros((n_h * d_h, 0)),
+                          np.eye(n_h * d_h), idx, d_h, base=300.0)
+
+    def rot(x):      # [n][n_h][d_h] rotated at its own position, chunk (2i, 2i+1) as a complex number
+        z = x[..., 0::2] + 1j * x[..., 1::2]
+        th = 300.0 ** (-2.0 * np.arange(d_h // 2) / d_h)
+        z = z * np.exp(1j * pos[:, None, None] * th[None, None, :])
+        y = np.empty_like(x)
+        y[..., 0::2], y[..., 1::2] = z.real, z.imag
+        return y
+    tq, tk, tv = (torch.from_numpy(a).permute(1, 0, 2) for a in (rot(q), rot(k), v))
+    want = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True).permute(1, 0, 2).numpy()
+    assert np.allclose(got, want, atol=1e-12)
+
+
+def test_causal_rows_are_single_query_decodes_over_their_prefixes():
+    """Row i equals the one-query definition on the tokens it may see; key positions need not be
+    sorted or contiguous; a row before every key is zero; with one row and everything visible it
+    is `decode` itself."""
+    z = _random_case(42, n=11)
+    d_h = z["d_h"]
+    key_pos = np.array([4, 0, 9, 2, 7, 5, 1, 8, 3, 6, 12])
+    k_rope = O.rotate_elite_keys(z["k_e"], key_pos, z["idx"], d_h)
+    g = _rng(43)
+    q = g.standard_normal((4, 3, d_h))
+    q_pos = np.array([5, 9, 12, -1])
+    got = O.attend_causal(q, q_pos, k_rope, key_pos, z["c"], z["W_uk"], z["W_uv"], z["idx"], d_h)
+    for i in range(3):
+        seen = key_pos <= q_pos[i]
+        want = O.decode(q[i], int(q_pos[i]), k_rope[seen], z["c"][seen], z["W_uk"], z["W_uv"], z["idx"], d_h)
+        assert np.allclose(got[i], want, atol=1e-12)
+    assert not got[3].any()
+    assert int((key_pos <= 5).sum()) == 6 and int((key_pos <= 9).sum()) == 10     # the masks differ
+    assert not np.allclose(got[0], got[1])
+    sub = O.attend_causal(q, q_pos, k_rope, key_pos, z["c"], z["W_uk"], z["W_uv"], z["idx"], d_h, heads=[2])
+    assert np.allclose(sub[:, 0], got[:, 2], atol=1e-12)

@@ -186,6 +186,27 @@ int elitekv_decode_step(const elitekv_layer* layer, const elitekv_cache* cache, 
                         const int32_t* seq_lens, int32_t B, void* q_rope, void* q_abs,
                         void* workspace, size_t workspace_bytes, void* out, elitekv_stream_t stream);
 
+/* Several query rows per sequence over the cache, with the causal rule (Section 3.1: the score
+ * equation holds for any query position m and key position n): a chunk of a prefill, or the
+ * draft tokens of speculative decoding.  The m new tokens of every sequence are in the cache
+ * already (elitekv_append / elitekv_project_append); seq_lens[b] counts them.  Query row i of
+ * sequence b sits at position seq_lens[b] - m + i and attends to the cached tokens at positions
+ * <= its own, i.e. to the first seq_lens[b] - (m - 1 - i) tokens; a row that sees none gives a
+ * zero row.
+ *   q_rope bf16 [B][m][n_h][2r], q_abs bf16 [B][m][n_h][d_c]: elitekv_absorb_query on the B*m
+ *          rows with q_pos[b*m + i] = seq_lens[b] - m + i
+ *   out    bf16 [B][m][n_h][d_h]
+ *   workspace: as for elitekv_decode, sized by elitekv_attend_rows_workspace_size(B, m)
+ * 1 <= m <= ELITEKV_MAX_QUERY_ROWS.  Runs on the two-pass tcgen05 kernel only (shapes it does
+ * not cover, or a layer created with decode_kernel 1 or 3: ELITEKV_ERR_UNSUPPORTED_SHAPE): one
+ * block per query row and head group walks the same token tiles at the same time, so a tile
+ * comes from HBM once and the other rows read it from L2.  m = 1 is elitekv_decode. */
+#define ELITEKV_MAX_QUERY_ROWS 16
+int elitekv_attend_rows_workspace_size(const elitekv_layer* layer, int32_t B, int32_t m, size_t* bytes);
+int elitekv_attend_rows(const elitekv_layer* layer, const elitekv_cache* cache, const void* q_rope,
+                        const void* q_abs, const int32_t* seq_lens, int32_t B, int32_t m,
+                        void* workspace, size_t workspace_bytes, void* out, elitekv_stream_t stream);
+
 /* Decode attention without any allocation (the paper has no counterpart; this is a packaging
  * variant of elitekv_decode).  For callers that must not, or cannot, call cudaMalloc: engines
  * that give all device memory to one arena up front, plugins running inside another

@@ -68,6 +68,8 @@ def lib() -> C.CDLL:
         L.elitekv_decode_workspace_size.argtypes = [vp, i32, C.POINTER(sz)]
         L.elitekv_decode.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, i32, vp, sz, vp, vp]
         L.elitekv_decode_step.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, sz, vp, vp]
+        L.elitekv_attend_rows_workspace_size.argtypes = [vp, i32, i32, C.POINTER(sz)]
+        L.elitekv_attend_rows.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, i32, i32, vp, sz, vp, vp]
         L.elitekv_decode_static.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, i32, vp, vp]
         L.elitekv_plan.argtypes = [vp, i32, i32, i32, vp, vp, vp]
         L.elitekv_plan_workers.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp]
@@ -87,7 +89,8 @@ def lib() -> C.CDLL:
                      "elitekv_profile_enable", "elitekv_profile_collect", "elitekv_decode_static",
                      "elitekv_mha_decode", "elitekv_plan_workers", "elitekv_decode_plan_info",
                      "elitekv_last_status_detail", "elitekv_selftest_bounded_wait",
-                     "elitekv_project_append", "elitekv_decode_step"):
+                     "elitekv_project_append", "elitekv_decode_step",
+                     "elitekv_attend_rows_workspace_size", "elitekv_attend_rows"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -233,6 +236,25 @@ def elitekv_decode_step(layer: Layer, cache: CacheDesc, k_e, c, seq_id, pos, q, 
                                      _ptr(q_rope), _ptr(_dev(q_abs, torch.bfloat16)), workspace.data_ptr(),
                                      workspace.numel() * workspace.element_size(),
                                      _ptr(_dev(out, torch.bfloat16)), _stream()), "elitekv_decode_step")
+    return out
+
+
+def elitekv_attend_rows_workspace_size(layer: Layer, B: int, m: int) -> int:
+    n = C.c_size_t()
+    _check(lib().elitekv_attend_rows_workspace_size(layer.handle, B, m, C.byref(n)),
+           "elitekv_attend_rows_workspace_size")
+    return n.value
+
+
+def elitekv_attend_rows(layer: Layer, cache: CacheDesc, q_rope, q_abs, seq_lens, m: int, workspace, out=None):
+    """q_rope [B][m][n_h][2r], q_abs [B][m][n_h][kw] -> out [B][m][n_h][d_h] (causal over the cache)."""
+    B = seq_lens.shape[0]
+    if out is None:
+        out = torch.empty((B, m, layer.n_h, layer.d_h), dtype=torch.bfloat16, device=q_abs.device)
+    _check(lib().elitekv_attend_rows(layer.handle, C.byref(cache), _ptr(q_rope), _ptr(_dev(q_abs, torch.bfloat16)),
+                                     _ptr(_dev(seq_lens, torch.int32)), B, m, workspace.data_ptr(),
+                                     workspace.numel() * workspace.element_size(), _ptr(out), _stream()),
+           "elitekv_attend_rows")
     return out
 
 

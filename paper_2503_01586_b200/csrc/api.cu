@@ -33,9 +33,9 @@ int select_kernel(const elitekv_layer* L, const elitekv_cache* cache) {
   return ekv_generic_supported(L) ? 1 : -1;
 }
 
-int max_items_for(const elitekv_layer* L, int B, int kernel) {
+int max_items_for(const elitekv_layer* L, int B, int kernel, int rows = 1) {
   if (kernel == 3) return ekv_rt_max_items(L, B);
-  return kernel == 2 ? ekv_tc_max_items(L, B) : ekv_generic_max_items(L, B);
+  return kernel == 2 ? ekv_tc_max_items(L, B, rows) : ekv_generic_max_items(L, B);
 }
 
 // Tokens per plan tile and persistent workers (0: the plain plan) of each kernel.
@@ -43,8 +43,8 @@ int plan_tile_for(int kernel) { return kernel == 2 ? 128 : ELITEKV_TILE_TOKENS; 
 // Tiles' worth of time that starting an item costs a worker (measured on B200: about one
 // 64-token tile for the resident-tile kernel).
 int item_overhead_for(int kernel) { return kernel == 3 ? 1 : 0; }
-int workers_for(const elitekv_layer* L, int kernel) {
-  return kernel == 3 ? ekv_rt_workers(L) : kernel == 2 ? ekv_tc_workers(L) : 0;
+int workers_for(const elitekv_layer* L, int kernel, int rows = 1) {
+  return kernel == 3 ? ekv_rt_workers(L) : kernel == 2 ? ekv_tc_workers(L, rows) : 0;
 }
 
 // The workspace is sized for whichever kernel may be picked once the cache layout is known.
@@ -53,7 +53,7 @@ int max_items_any(const elitekv_layer* L, int B) {
   const int want = L->decode_kernel;
   if (ekv_generic_supported(L) && (want == 0 || want == 1)) m = ekv_generic_max_items(L, B);
   if (ekv_tc_supported(L, nullptr) && (want == 0 || want == 2)) {
-    const int t = ekv_tc_max_items(L, B);
+    const int t = ekv_tc_max_items(L, B, 1);
     if (t > m) m = t;
   }
   if (ekv_rt_supported(L, nullptr) && (want == 0 || want == 3)) {
@@ -67,15 +67,17 @@ struct Carve {
   size_t off_items, off_first, off_ml, off_acc, off_slice, off_cnt, off_wfirst, total;
 };
 
-Carve carve(const elitekv_layer* L, int B, int max_items) {
+// `rows` query rows per sequence: the partial results, the combine's scratch and its counters
+// hold rows x n_h entries where decoding holds n_h.
+Carve carve(const elitekv_layer* L, int B, int max_items, int rows = 1) {
   Carve c;
   size_t o = 0;
   c.off_items = o; o = align256(o + sizeof(int32_t) * 4 * (size_t)max_items);
   c.off_first = o; o = align256(o + sizeof(int32_t) * ((size_t)B + 1));
-  c.off_ml = o;    o = align256(o + sizeof(float) * 2 * (size_t)max_items * L->n_h);
-  c.off_acc = o;   o = align256(o + sizeof(float) * (size_t)max_items * L->n_h * L->vw);
-  c.off_slice = o; o = align256(o + ekv_combine_scratch_bytes(L, B));
-  c.off_cnt = o;   o = align256(o + sizeof(int32_t) * (size_t)ekv_combine_counters(L, B));
+  c.off_ml = o;    o = align256(o + sizeof(float) * 2 * (size_t)max_items * L->n_h * rows);
+  c.off_acc = o;   o = align256(o + sizeof(float) * (size_t)max_items * L->n_h * rows * L->vw);
+  c.off_slice = o; o = align256(o + ekv_combine_scratch_bytes(L, B) * rows);
+  c.off_cnt = o;   o = align256(o + sizeof(int32_t) * (size_t)ekv_combine_counters(L, B) * rows);
   c.off_wfirst = o; o = align256(o + sizeof(int32_t) * ((size_t)L->sm_count + 2));
   c.total = o;
   return c;
@@ -149,21 +151,29 @@ namespace {
 template <class Fn>
 int decode_impl(const elitekv_layer* L, const elitekv_cache* cache, const void* q_rope, const void* q_abs,
                 const int32_t* seq_lens, int32_t B, void* workspace, size_t workspace_bytes, void* out,
-                cudaStream_t st, cudaStream_t plan_stream, Fn before_kernel) {
+                cudaStream_t st, cudaStream_t plan_stream, Fn before_kernel, int rows = 1) {
   if (!L || !cache || !q_abs || !seq_lens || !workspace || !out || B <= 0 || (L->r > 0 && !q_rope))
     return ELITEKV_ERR_INVALID_ARG;
   if (((uintptr_t)q_abs & 15) || ((uintptr_t)out & 3)) return ELITEKV_ERR_INVALID_ARG;
-  if (B > cache->n_seqs) return ELITEKV_ERR_INVALID_ARG;
-  const int kernel = select_kernel(L, cache);
+  if (B > cache->n_seqs || rows < 1 || rows > ELITEKV_MAX_QUERY_ROWS) return ELITEKV_ERR_INVALID_ARG;
+  int kernel = select_kernel(L, cache);
+  if (rows > 1) {
+    // several query rows run on the two-pass tensor-core kernel only (one block per row and head
+    // group walks the same tiles at the same time, so the rows share the tile through L2)
+    if (L->decode_kernel != 0 && L->decode_kernel != 2) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
+    kernel = ekv_tc_supported(L, cache) ? 2 : -1;
+  }
   if (kernel < 0) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
   CacheView cv;
   int rc = ekv_make_view(cache, &cv);
   if (rc != ELITEKV_OK) return rc;
-  const int max_items = max_items_for(L, B, kernel);
-  const Carve cw = carve(L, B, max_items);
+  const int max_items = max_items_for(L, B, kernel, rows);
+  const Carve cw = carve(L, B, max_items, rows);
   if (((uintptr_t)workspace & 255) || workspace_bytes < cw.total) return ELITEKV_ERR_WORKSPACE_TOO_SMALL;
   unsigned char* base = (unsigned char*)workspace;
   DecodeScratch ws;
+  ws.rows = rows;
+  ws.seq_lens = seq_lens;
   ws.max_items = max_items;
   ws.items = (int32_t*)(base + cw.off_items);
   ws.seq_first = (int32_t*)(base + cw.off_first);
@@ -171,9 +181,9 @@ int decode_impl(const elitekv_layer* L, const elitekv_cache* cache, const void* 
   ws.part_acc = (float*)(base + cw.off_acc);
   ws.slice_out = (float*)(base + cw.off_slice);
   ws.counters = (int32_t*)(base + cw.off_cnt);
-  ws.n_counters = ekv_combine_counters(L, B);
+  ws.n_counters = ekv_combine_counters(L, B) * rows;
   ws.worker_first = (int32_t*)(base + cw.off_wfirst);
-  ws.n_workers = workers_for(L, kernel);
+  ws.n_workers = workers_for(L, kernel, rows);
   // tokens one sequence can hold: longer lengths are reported by the plan kernel and clamped
   const long long max_len = cv.page_table ? (long long)cv.max_pages_per_seq << cv.page_shift : cv.max_ctx;
   cudaStream_t ps = plan_stream ? plan_stream : st;
@@ -244,4 +254,19 @@ extern "C" int elitekv_decode_step(const elitekv_layer* L, const elitekv_cache* 
     cudaStreamWaitEvent(st, L->ev_join, 0);
   }
   return rc_append != ELITEKV_OK ? rc_append : rc;
+}
+
+extern "C" int elitekv_attend_rows_workspace_size(const elitekv_layer* L, int32_t B, int32_t m, size_t* bytes) {
+  if (!L || !bytes || B <= 0 || m < 1 || m > ELITEKV_MAX_QUERY_ROWS) return ELITEKV_ERR_INVALID_ARG;
+  if (!ekv_tc_supported(L, nullptr)) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
+  *bytes = carve(L, B, ekv_tc_max_items(L, B, m), m).total;
+  return ELITEKV_OK;
+}
+
+extern "C" int elitekv_attend_rows(const elitekv_layer* L, const elitekv_cache* cache, const void* q_rope,
+                                   const void* q_abs, const int32_t* seq_lens, int32_t B, int32_t m,
+                                   void* workspace, size_t workspace_bytes, void* out,
+                                   elitekv_stream_t stream) {
+  return decode_impl(L, cache, q_rope, q_abs, seq_lens, B, workspace, workspace_bytes, out,
+                     (cudaStream_t)stream, nullptr, [] { return (int)ELITEKV_OK; }, m);
 }

@@ -15,6 +15,9 @@
 //
 // Generic kernel: any even d_h <= 512, any d_c; block per (head, 8 sequences).
 //
+// With several query rows per sequence the kernels see rows x heads "heads" (n_h below); entry
+// i * heads + h multiplies with head h's columns of W_uv (n_phys = heads).
+//
 // With separated latents (S-LRD) the partial outputs span the value latent only; `d_c` below is
 // then d_cv and W_uv is B^v_S.
 #include "common.cuh"
@@ -44,7 +47,8 @@ combine_fast_kernel(const float* part_acc, const float* part_ml,   // written by
                     const int32_t* seq_first, const bf16* __restrict__ Wuv,
                     float* __restrict__ slice_out /* [n_slices][B][n_h][128] */,
                     int32_t* __restrict__ counters /* [n_h][n_groups], zeroed by the plan kernel */,
-                    bf16* __restrict__ out, int B, int n_h, int d_c) {
+                    bf16* __restrict__ out, int B, int n_h /* query rows x heads */, int n_phys /* heads */,
+                    int d_c) {
   __shared__ __align__(16) bf16 s_w[kFK][kFD + 8];      // W_uv slice; rows padded by 16 bytes so that the
                                                         // fragment loads of the product spread over the banks
   __shared__ __align__(16) float s_x[kFB][kFK + 8];     // merged latent outputs (padded rows: bank spread)
@@ -61,7 +65,7 @@ combine_fast_kernel(const float* part_acc, const float* part_ml,   // written by
   // statistics of the first group are worked out
   for (int e = tid; e < kFK * (kFD / 8); e += kFThreads) {
     const int k = e / (kFD / 8), v = e % (kFD / 8);
-    cp_async16(&s_w[k][v * 8], Wuv + (size_t)(k0 + k) * n_h * kFD + (size_t)h * kFD + v * 8);
+    cp_async16(&s_w[k][v * 8], Wuv + (size_t)(k0 + k) * n_phys * kFD + (size_t)(h % n_phys) * kFD + v * 8);
   }
   cp_async_commit();
   ekv_pdl_wait();         // the weights above are constant; everything below reads the split-K kernel's output
@@ -207,7 +211,8 @@ constexpr int kCombChunk = 128;
 __global__ void __launch_bounds__(kCombThreads)
 combine_upproj_kernel(const float* __restrict__ part_acc, const float* __restrict__ part_ml,
                       const int32_t* __restrict__ seq_first, const bf16* __restrict__ Wuv,
-                      bf16* __restrict__ out, int B, int n_h, int d_h, int d_c) {
+                      bf16* __restrict__ out, int B, int n_h /* query rows x heads */, int n_phys /* heads */,
+                      int d_h, int d_c) {
   __shared__ float s_olat[kCombBatch][kCombChunk];
   __shared__ float s_M[kCombBatch], s_invL[kCombBatch];
   __shared__ int s_first[kCombBatch + 1];
@@ -267,7 +272,7 @@ combine_upproj_kernel(const float* __restrict__ part_acc, const float* __restric
     if (worker) {
       for (int k = kg; k < kc; k += kgroups) {
         const float2 w = __bfloat1622float2(
-            *(const bf162*)(Wuv + (size_t)(k0 + k) * n_h * d_h + (size_t)h * d_h + 2 * pair));
+            *(const bf162*)(Wuv + (size_t)(k0 + k) * n_phys * d_h + (size_t)(h % n_phys) * d_h + 2 * pair));
 #pragma unroll
         for (int bb = 0; bb < kCombBatch; ++bb) {
           const float x = s_olat[bb][k];
@@ -310,11 +315,14 @@ int ekv_combine_counters(const elitekv_layer* L, int B) {
 
 int ekv_launch_combine(const elitekv_layer* L, int B, const DecodeScratch& ws, void* out,
                        cudaStream_t st) {
+  // several query rows per sequence: row i, head h is "head" i * n_h + h of the partial results
+  // and of the output; it uses head h's slice of W_uv
+  const int nv = (ws.rows > 0 ? ws.rows : 1) * L->n_h;
   if (ekv_combine_fast_ok(L)) {
-    dim3 grid(L->n_h, L->vw / kFK);
+    dim3 grid(nv, L->vw / kFK);
     EKV_CUDA_OK(ekv_launch_pdl(combine_fast_kernel, grid, dim3(kFThreads), 0, st, (const float*)ws.part_acc,
                                (const float*)ws.part_ml, (const int32_t*)ws.seq_first, (const bf16*)L->d_Wuv,
-                               ws.slice_out, ws.counters, (bf16*)out, B, L->n_h, L->vw));
+                               ws.slice_out, ws.counters, (bf16*)out, B, nv, L->n_h, L->vw));
     EKV_CUDA_OK(cudaGetLastError());
     return ELITEKV_OK;
   }
@@ -322,11 +330,11 @@ int ekv_launch_combine(const elitekv_layer* L, int B, const DecodeScratch& ws, v
   if (npair > kCombThreads) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
   const int kgroups = kCombThreads / npair > 0 ? kCombThreads / npair : 1;
   const size_t smem = sizeof(float) * (size_t)kgroups * kCombBatch * L->d_h;
-  dim3 grid(L->n_h, (B + kCombBatch - 1) / kCombBatch);
+  dim3 grid(nv, (B + kCombBatch - 1) / kCombBatch);
   EKV_CUDA_OK(cudaFuncSetAttribute(combine_upproj_kernel,
                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   combine_upproj_kernel<<<grid, kCombThreads, smem, st>>>(ws.part_acc, ws.part_ml, ws.seq_first,
-                                                          L->d_Wuv, (bf16*)out, B, L->n_h, L->d_h,
+                                                          L->d_Wuv, (bf16*)out, B, nv, L->n_h, L->d_h,
                                                           L->vw);
   EKV_CUDA_OK(cudaGetLastError());
   return ELITEKV_OK;

@@ -174,6 +174,9 @@ struct DecodeScratch {
   int n_counters;
   int32_t* worker_first;  // balanced plan: [n_workers+1] first item of each worker
   int n_workers;
+  int rows;               // query rows per sequence (1: decode).  With rows > 1 every "n_h" in the shapes
+                          // above reads rows * n_h: row i, head h is entry i * n_h + h
+  const int32_t* seq_lens;   // rows > 1: the lengths, for the causal limit of each row
 };
 
 int ekv_combine_fast_ok(const elitekv_layer* L);
@@ -186,8 +189,8 @@ int ekv_launch_decode_generic(const elitekv_layer* L, const elitekv_cache* cache
                               const CacheView& cv, const void* q_rope, const void* q_abs, int B,
                               const DecodeScratch& ws, cudaStream_t st);
 int ekv_tc_supported(const elitekv_layer* L, const elitekv_cache* cache);   // cache may be null
-int ekv_tc_max_items(const elitekv_layer* L, int B);
-int ekv_tc_workers(const elitekv_layer* L);
+int ekv_tc_max_items(const elitekv_layer* L, int B, int rows);
+int ekv_tc_workers(const elitekv_layer* L, int rows);
 int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, const CacheView& cv,
                          const void* q_rope, const void* q_abs, int B, const DecodeScratch& ws,
                          cudaStream_t st);

@@ -269,6 +269,7 @@ int ekv_launch_decode_generic(const elitekv_layer* L, const elitekv_cache* cache
                               const CacheView& cv, const void* q_rope, const void* q_abs, int B,
                               const DecodeScratch& ws, cudaStream_t st) {
   if (!ekv_generic_supported(L)) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
+  if (ws.rows > 1) return ELITEKV_ERR_UNSUPPORTED_SHAPE;      // one query row per sequence here
   GenericArgs a;
   a.rope = (const bf16*)cache->rope;
   a.latent = (const bf16*)cache->latent;

@@ -778,7 +778,7 @@ int ekv_rt_max_items(const elitekv_layer* L, int B) { return L->sm_count / 2 + B
 int ekv_launch_decode_rt(const elitekv_layer* L, const elitekv_cache* cache, const CacheView& cv,
                          const void* q_rope, const void* q_abs, int B, const DecodeScratch& ws,
                          cudaStream_t st) {
-  if (!ekv_rt_supported(L, cache)) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
+  if (!ekv_rt_supported(L, cache) || ws.rows > 1) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
   if ((uintptr_t)q_rope & 15) return ELITEKV_ERR_INVALID_ARG;   // rope rows are read with 16-byte loads
   const unsigned long long rows =
       cv.page_table ? (unsigned long long)cv.num_pages << cv.page_shift : (unsigned long long)cv.max_ctx * cv.n_seqs;

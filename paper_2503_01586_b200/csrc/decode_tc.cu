@@ -71,7 +71,9 @@ struct TcArgs {
   int page_shift, page_mask, max_pages_per_seq;
   int n_h, d_c;
   int kw, voff, vw;         // latent columns of the scores [0, kw) and of the outputs [voff, voff + vw)
-  int n_groups;             // head groups of N heads; blockIdx.x = item * n_groups + group
+  int n_groups;             // blocks per worker: query rows x head groups of N heads; blockIdx.x = worker * n_groups + group
+  int rows, gpr, nv;        // query rows per sequence, head groups per row, rows * n_h
+  const int32_t* seq_lens;  // rows > 1: row i of sequence b sees seq_lens[b] - (rows - 1 - i) tokens
   float scale_log2e;
 };
 
@@ -106,7 +108,10 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
                  const TcArgs a) {
   extern __shared__ unsigned char smem_raw[];
   const int worker = blockIdx.x / a.n_groups;         // persistent worker: walks its plan items
-  const int h0 = (blockIdx.x % a.n_groups) * N;       // first head of this block's group
+  const int grp = blockIdx.x % a.n_groups;
+  const int qrow = grp / a.gpr;                       // query row of this block (0 when decoding)
+  const int h0 = (grp % a.gpr) * N;                   // first head of this block's group
+  const int vh0 = qrow * a.n_h + h0;                  // the same in the [rows][n_h] layout of queries and results
   const int nh_here = min(N, a.n_h - h0);
   const int d_c = a.d_c;
   const int NKC = a.kw >> 6;     // 64-wide latent chunks of pass A
@@ -190,7 +195,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
   if (warp >= 2 && warp <= 5) {
     for (int e = threadIdx.x - 64; e < N * R2; e += kSoftmaxThreads) {
       const int h = e / R2;
-      s_qrope[e] = h < nh_here ? __bfloat162float(a.q_rope[((size_t)seq * a.n_h + h0 + h) * R2 + (e % R2)]) : 0.f;
+      s_qrope[e] = h < nh_here ? __bfloat162float(a.q_rope[((size_t)seq * a.nv + vh0 + h) * R2 + (e % R2)]) : 0.f;
     }
     named_bar_sync(1, kSoftmaxThreads);
   }
@@ -243,7 +248,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
             const uint32_t fb = smem_u32(&bars->lat_full[slot]);
             mbar_expect_tx(fb, (uint32_t)(halves * 8192 + (with_q ? N * 128 : 0)));
             if (with_q)   // the sequence's absorbed queries for these 64 latent coordinates (L2-resident)
-              tma_load_2d_hint(smem_u32(s_lat + slot * kSlot + kChunkBytes), &map_q, kc * 64, seq * a.n_h + h0, fb, pol_keep);
+              tma_load_2d_hint(smem_u32(s_lat + slot * kSlot + kChunkBytes), &map_q, kc * 64, seq * a.nv + vh0, fb, pol_keep);
             const uint64_t pol = (with_q && reread) ? pol_keep : pol_drop;
             if (whole) {
               tma_load_2d_hint(smem_u32(s_lat + slot * kSlot), &map_lat128, kc * 64, (int)row[0], fb, pol);
@@ -378,13 +383,19 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
     float l_part[N];                              // per-thread partial softmax denominators
 #pragma unroll
     for (int h = 0; h < N; ++h) l_part[h] = 0.f;
-    float m_ref = -INFINITY;                      // lane h holds head h's reference max (N <= 32 per group)
+    // lane h holds head h's reference max (N <= 32 per group).  With several query rows a row
+    // may see nothing of an item (its causal limit lies before it): a finite start keeps
+    // exp2(-inf - m_ref) at zero instead of NaN.
+    float m_ref = a.rows > 1 ? -1e30f : -INFINITY;
+    // tokens of this item the block's query row may see (causal rule; all of them when decoding)
+    int vis = ntok;
+    if (a.rows > 1) vis = max(0, min(ntok, a.seq_lens[seq] - (a.rows - 1 - qrow) - tok0));
     bool ok = true;
     const bool leader = threadIdx.x == 64;
     static_assert(N == 16 || N == 32, "softmax threads keep one head per lane (lanes >= N idle)");
 
     for (int tile = 0; tile < n_tiles && ok; ++tile) {
-      const int nvalid = min(kTile, ntok - tile * kTile);
+      const int nvis = min(kTile, vis - tile * kTile);     // rows of the tile this query row sees (may be <= 0)
       float s[N];
 #pragma unroll
       for (int h = 0; h < N; ++h) s[h] = 0.f;
@@ -433,7 +444,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
 #pragma unroll
         for (int h = 0; h < N; ++h) {
           const float x = (s[h] + sv[h]) * a.scale_log2e;
-          s[h] = trow < nvalid ? x : -INFINITY;
+          s[h] = trow < nvis ? x : -INFINITY;
         }
       }
       // ---- per-head max over the 128 tokens of the tile
@@ -509,8 +520,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       named_bar_sync(1, kSoftmaxThreads);
       if (quarter == 0 && lane < nh_here) {
         const float lsum = s_wmax[lane] + s_wmax[N + lane] + s_wmax[2 * N + lane] + s_wmax[3 * N + lane];
-        a.part_ml[((size_t)item * a.n_h + h0 + lane) * 2 + 0] = m_ref;
-        a.part_ml[((size_t)item * a.n_h + h0 + lane) * 2 + 1] = lsum;
+        a.part_ml[((size_t)item * a.nv + vh0 + lane) * 2 + 0] = m_ref;
+        a.part_ml[((size_t)item * a.nv + vh0 + lane) * 2 + 1] = lsum;
       }
     }
     // ---- ... and its partial output
@@ -519,8 +530,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       tc_fence_after();
       // The output block [128 coords x N heads] leaves TMEM with one thread per coordinate; it is
       // turned into [N heads][128 coords] tiles in shared memory (the ring is idle by now) and
-      // written with one TMA store per block: part_acc[item][h0 + h][blk*128 ...].  Rows of a
-      // last, partly filled head group fall outside the tensor and are clipped by the store.
+      // written with one TMA store per block: part_acc[item][query row][h0 + h][blk*128 ...].
+      // Rows of a last, partly filled head group fall outside the head axis of the tensor and
+      // are clipped by the store.
       float* stage = (float*)s_lat;
       for (int blk = 0; blk < NB; ++blk) {
         float v[N];
@@ -536,7 +548,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         fence_proxy_async();
         named_bar_sync(1, kSoftmaxThreads);
         if (threadIdx.x == 64) {
-          tma_store_3d(&map_part, blk * 128, h0, item, smem_u32(tile_s));
+          tma_store_4d(&map_part, blk * 128, h0, qrow, item, smem_u32(tile_s));
           bulk_commit_group();
         }
       }
@@ -597,9 +609,13 @@ static int tc_groups(const elitekv_layer* L) {
   return n ? (L->n_h + n - 1) / n : 1;
 }
 
-// One persistent worker (a block per head group) per SM share; items = workers + sequences at most.
-int ekv_tc_workers(const elitekv_layer* L) { return L->sm_count / tc_groups(L) > 0 ? L->sm_count / tc_groups(L) : 1; }
-int ekv_tc_max_items(const elitekv_layer* L, int B) { return ekv_tc_workers(L) + B; }
+// One persistent worker (a block per query row and head group) per SM share; items = workers +
+// sequences at most.
+int ekv_tc_workers(const elitekv_layer* L, int rows) {
+  const int per = tc_groups(L) * (rows > 0 ? rows : 1);
+  return L->sm_count / per > 0 ? L->sm_count / per : 1;
+}
+int ekv_tc_max_items(const elitekv_layer* L, int B, int rows) { return ekv_tc_workers(L, rows) + B; }
 
 int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, const CacheView& cv,
                          const void* q_rope, const void* q_abs, int B, const DecodeScratch& ws,
@@ -614,8 +630,9 @@ int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, con
   if (rc == ELITEKV_OK) rc = make_map(&m_lat128, cache->latent, rows, L->d_c, 128);
   if (rc == ELITEKV_OK) rc = make_map(&m_rope128, cache->rope, rows, (unsigned long long)L->n_h * 2 * L->r, 128);
   const int N = tc_pick_n(L);
-  if (rc == ELITEKV_OK) rc = make_map(&m_q, q_abs, (unsigned long long)B * L->n_h, L->kw, N);
-  if (rc == ELITEKV_OK) rc = make_map_f32_3d(&m_part, ws.part_acc, L->vw, L->n_h, (unsigned long long)ws.max_items, N);
+  const int rows_q = ws.rows > 0 ? ws.rows : 1;
+  if (rc == ELITEKV_OK) rc = make_map(&m_q, q_abs, (unsigned long long)B * rows_q * L->n_h, L->kw, N);
+  if (rc == ELITEKV_OK) rc = make_map_f32_4d(&m_part, ws.part_acc, L->vw, L->n_h, rows_q, (unsigned long long)ws.max_items, N);
   if (rc != ELITEKV_OK) return rc;
   TcArgs a;
   a.items = ws.items;
@@ -635,7 +652,11 @@ int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, con
   a.kw = L->kw;
   a.voff = L->voff;
   a.vw = L->vw;
-  a.n_groups = tc_groups(L);
+  a.rows = rows_q;
+  a.gpr = tc_groups(L);
+  a.n_groups = a.gpr * rows_q;
+  a.nv = rows_q * L->n_h;
+  a.seq_lens = ws.seq_lens;
   a.scale_log2e = L->scale * 1.4426950408889634f;
   const int smem = N == 32 ? Smem<32>::total(L->d_c) : Smem<16>::total(L->d_c);
   auto launch = [&](auto kern) -> int {

@@ -140,10 +140,10 @@ __device__ __forceinline__ uint64_t make_l2_policy_evict_first() {
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
   return p;
 }
-// TMA store of one 3-D box from shared memory (bulk async-group completion)
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, int x, int y, int z, uint32_t src) {
-  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
-               ::"l"((uint64_t)map), "r"(x), "r"(y), "r"(z), "r"(src) : "memory");
+// TMA store of one 4-D box from shared memory (bulk async-group completion)
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, int x, int y, int z, int w, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
+               ::"l"((uint64_t)map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(src) : "memory");
 }
 __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_group_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
@@ -354,17 +354,17 @@ static inline EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// 3-D fp32 tensor [d2][d1][d0] (d0 contiguous), box [1][box1][128], no swizzle: the target of
-// the TMA stores of the partial results (stores clip at the tensor's edges)
-static inline int make_map_f32_3d(CUtensorMap* m, const void* ptr, unsigned long long d0, unsigned long long d1,
-                                  unsigned long long d2, unsigned box1) {
+// 4-D fp32 tensor [d3][d2][d1][d0] (d0 contiguous), box [1][1][box1][128], no swizzle: the target
+// of the TMA stores of the partial results (stores clip at the tensor's edges)
+static inline int make_map_f32_4d(CUtensorMap* m, const void* ptr, unsigned long long d0, unsigned long long d1,
+                                  unsigned long long d2, unsigned long long d3, unsigned box1) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return ELITEKV_ERR_CUDA;
-  cuuint64_t dims[3] = {d0, d1, d2};
-  cuuint64_t strides[2] = {d0 * sizeof(float), d0 * d1 * sizeof(float)};
-  cuuint32_t box[3] = {128, box1, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+  cuuint64_t dims[4] = {d0, d1, d2, d3};
+  cuuint64_t strides[3] = {d0 * sizeof(float), d0 * d1 * sizeof(float), d0 * d1 * d2 * sizeof(float)};
+  cuuint32_t box[4] = {128, box1, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(ptr), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? ELITEKV_OK : ELITEKV_ERR_CUDA;

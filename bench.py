@@ -437,6 +437,44 @@ def append_prefill(ek, device, flush, reps: int = 5):
 
 
 
+def attend_rows_bench(ek, layer, cache, w, lens, device, flush, cache_bytes, reps: int = 5):
+    """m query rows per sequence over the bench workload's cache (causal; the rows sit at the last
+    m positions): time of elitekv_attend_rows (plan + two-pass kernel + combine) and the cache
+    bytes, counted ONCE, over that time.  Every row's block reads the whole tile, the first from
+    HBM and the others from L2, so the ideal is still one pass over the cache."""
+    peak, peak_kind = measured_peaks()
+    out = {}
+    lens_dev = lens.to(torch.int32).to(device)
+    g = torch.Generator(device=device).manual_seed(99)
+    for m in (2, 4, 8):
+        try:
+            q = torch.randn((w.B * m, w.n_h, w.d_h), generator=g, device=device).to(torch.bfloat16)
+            q_pos = (lens_dev.view(-1, 1) - m + torch.arange(m, device=device, dtype=torch.int32).view(1, m))
+            q_rope, q_abs = ek.elitekv_absorb_query(layer, q, q_pos.reshape(-1).to(torch.int32).contiguous())
+            ws = torch.empty(ek.elitekv_attend_rows_workspace_size(layer, w.B, m), dtype=torch.uint8, device=device)
+            res = torch.empty((w.B, m, w.n_h, w.d_h), dtype=torch.bfloat16, device=device)
+            for _ in range(2):
+                ek.elitekv_attend_rows(layer, cache, q_rope, q_abs, lens_dev, m, ws, res)
+            evs = []
+            for _ in range(reps):
+                flush.fill_(1)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                ek.elitekv_attend_rows(layer, cache, q_rope, q_abs, lens_dev, m, ws, res)
+                b.record()
+                evs.append((a, b))
+            torch.cuda.synchronize()
+            us = 1e3 * sum(a.elapsed_time(b) for a, b in evs) / reps
+            out[f"m{m}"] = {"rows": m, "us": us, "query_rows_per_s": w.B * m / (us * 1e-6),
+                            "cache_gbs_counted_once": cache_bytes / (us * 1e-6) / 1e9,
+                            "frac": cache_bytes / (us * 1e-6) / 1e9 / peak, "peak_kind": f"of {peak_kind}"}
+            del q, q_rope, q_abs, ws, res
+        except ek.ElitekvError as exc:
+            out[f"m{m}"] = {"rows": m, "skipped": str(exc)}
+    assert ek.elitekv_check_status(layer) == 0
+    return out
+
+
 def run_gpu(args, w: gen.Workload):
     from paper_2503_01586_b200 import binding as ek
     ek.lib()   # fail loudly if the CUDA library is missing
@@ -580,8 +618,9 @@ def run_gpu(args, w: gen.Workload):
             comparator = None
 
     # ---- the other benchmark configurations and the prefill append (one GPU, rank 0 only)
-    sweep, prefill, projection = None, None, None
+    sweep, prefill, projection, rows = None, None, None, None
     if rank == 0 and world == 1 and not args.no_sweep:
+        rows = attend_rows_bench(ek, layer, cache, w, lens, device, flush, cache_bytes)
         del layer, cache, dev, ws, bufs, keep, eager_runner
         torch.cuda.empty_cache()
         t_sweep = time.perf_counter()
@@ -640,6 +679,7 @@ def run_gpu(args, w: gen.Workload):
         line["cpu_baseline"] = None
     line["stages"]["append_prefill"] = prefill
     line["stages"]["project_append"] = projection
+    line["stages"]["attend_rows"] = rows
     line["sweep"] = sweep
     print(json.dumps(line))
     if dist is not None:

@@ -58,6 +58,45 @@ def test_append_layout_and_bits(ek, paged):
     assert np.array_equal(H.bits(st.rope_plane), rope_exp)
 
 
+@pytest.mark.parametrize("paged", [False, True])
+def test_append_prefill_sized_call_bits(ek, paged):
+    """A call of thousands of tokens takes the staged form (groups of tokens through a
+    shared-memory ring with bulk copies).  7B shape, 4200 tokens in shuffled order in one call
+    (groups of 8: a ragged last group), a token with a position outside the table in the middle:
+    reported, not written, everything else bit for bit as the oracle's append says."""
+    w = replace(gen.shrink(gen.LLAMA7B_75, B=3, ctx=2100), paged=paged, seed=48 + paged)
+    lens = [2100, 2000, 100]
+    table32 = torch.from_numpy(O.rope_table_f32(2104, w.d_h, w.rope_base)).cuda()
+    st = H.setup(w, lens=lens, cos_sin=table32, fill=False)
+    g = torch.Generator(device="cpu").manual_seed(6)
+    rope0 = torch.randint(0, 2 ** 15, tuple(st.rope_plane.shape), generator=g, dtype=torch.int16)
+    lat0 = torch.randint(0, 2 ** 15, tuple(st.latent_plane.shape), generator=g, dtype=torch.int16)
+    st.rope_plane.copy_(rope0.view(torch.bfloat16))
+    st.latent_plane.copy_(lat0.view(torch.bfloat16))
+    N = st.c.shape[0]
+    assert N == 4200
+    perm = torch.randperm(N, generator=g).cuda()
+    pos = st.pos[perm].contiguous()
+    bad = 1234
+    good = torch.ones(N, dtype=torch.bool)
+    good[bad] = False
+    pos_bad = pos.clone()
+    pos_bad[bad] = 1_000_000
+    ek.elitekv_append(st.layer, st.cache, st.k_e[perm].contiguous(), st.c[perm].contiguous(),
+                      st.seq_id[perm].contiguous(), pos_bad)
+    torch.cuda.synchronize()
+    assert ek.elitekv_check_status(st.layer) == ek.ERR_BAD_POSITION
+    sel = perm.cpu()[good]
+    pt = st.page_table.cpu().numpy() if paged else None
+    max_ctx = st.cache.max_ctx if not paged else None
+    rope_exp, lat_exp = O.append_expected(
+        rope0.numpy().view(np.uint16), lat0.numpy().view(np.uint16), H.bits(st.k_e)[sel], H.bits(st.c)[sel],
+        st.seq_id.cpu().numpy()[sel], st.pos.cpu().numpy()[sel], st.idx.numpy(), w.d_h, base=w.rope_base,
+        max_ctx=max_ctx, page_table=pt, page_size=w.page_size, table32=table32.cpu().numpy())
+    assert np.array_equal(H.bits(st.latent_plane), lat_exp)
+    assert np.array_equal(H.bits(st.rope_plane), rope_exp)
+
+
 def test_append_own_table_within_one_ulp(ek):
     w = replace(SMALL, seed=44)
     st = H.setup(w, lens=[64, 65, 129])

@@ -207,6 +207,29 @@ int elitekv_attend_rows(const elitekv_layer* layer, const elitekv_cache* cache, 
                         const void* q_abs, const int32_t* seq_lens, int32_t B, int32_t m,
                         void* workspace, size_t workspace_bytes, void* out, elitekv_stream_t stream);
 
+/* RoPElite search (Algorithm 1, Section 3.1) on calibration activations: which r chunks of every
+ * head keep their rotation.  Q, K: bf16 [n_heads][n][d_h], un-rotated queries and keys of a
+ * calibration sequence of n tokens (token t at position t), heads of all layers side by side;
+ * d_h is 64 or 128.  A round computes, per head and per chunk j not yet chosen, the L1 distance
+ * over all causal pairs (query position m, key position <= m) between the pre-softmax scores
+ * q K^T with RoPE on every chunk and with RoPE on the chosen chunks plus j only; the first
+ * minimum joins the head's list.
+ *   elitekv_ropelite_distances: one round for given lists.  elite_mask: uint64 [n_heads], bit i
+ *     set = chunk i already chosen (NULL: none).  dist: fp32 [n_heads][d_h/2], +inf at chosen
+ *     chunks.
+ *   elitekv_ropelite_search: r rounds.  elite_idx: int32 [n_heads][r], chunks in the order
+ *     chosen (the order elitekv_params.elite_idx wants).  dist_trace: optional fp32
+ *     [r][n_heads][d_h/2], the distances of every round.
+ * Sums are fp32 and added in a fixed order (results do not depend on scheduling).  workspace:
+ * 256-byte aligned, elitekv_ropelite_workspace_size bytes. */
+int elitekv_ropelite_workspace_size(int32_t n_heads, int32_t n, int32_t d_h, size_t* bytes);
+int elitekv_ropelite_distances(const void* Q, const void* K, int32_t n_heads, int32_t n, int32_t d_h,
+                               float rope_base, const uint64_t* elite_mask, void* workspace,
+                               size_t workspace_bytes, float* dist, elitekv_stream_t stream);
+int elitekv_ropelite_search(const void* Q, const void* K, int32_t n_heads, int32_t n, int32_t d_h,
+                            float rope_base, int32_t r, void* workspace, size_t workspace_bytes,
+                            int32_t* elite_idx, float* dist_trace, elitekv_stream_t stream);
+
 /* Decode attention without any allocation (the paper has no counterpart; this is a packaging
  * variant of elitekv_decode).  For callers that must not, or cannot, call cudaMalloc: engines
  * that give all device memory to one arena up front, plugins running inside another

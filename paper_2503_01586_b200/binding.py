@@ -70,6 +70,9 @@ def lib() -> C.CDLL:
         L.elitekv_decode_step.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, sz, vp, vp]
         L.elitekv_attend_rows_workspace_size.argtypes = [vp, i32, i32, C.POINTER(sz)]
         L.elitekv_attend_rows.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, i32, i32, vp, sz, vp, vp]
+        L.elitekv_ropelite_workspace_size.argtypes = [i32, i32, i32, C.POINTER(sz)]
+        L.elitekv_ropelite_distances.argtypes = [vp, vp, i32, i32, i32, C.c_float, vp, vp, sz, vp, vp]
+        L.elitekv_ropelite_search.argtypes = [vp, vp, i32, i32, i32, C.c_float, i32, vp, sz, vp, vp, vp]
         L.elitekv_decode_static.argtypes = [vp, C.POINTER(CacheDesc), vp, vp, vp, i32, vp, vp]
         L.elitekv_plan.argtypes = [vp, i32, i32, i32, vp, vp, vp]
         L.elitekv_plan_workers.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp]
@@ -90,7 +93,8 @@ def lib() -> C.CDLL:
                      "elitekv_mha_decode", "elitekv_plan_workers", "elitekv_decode_plan_info",
                      "elitekv_last_status_detail", "elitekv_selftest_bounded_wait",
                      "elitekv_project_append", "elitekv_decode_step",
-                     "elitekv_attend_rows_workspace_size", "elitekv_attend_rows"):
+                     "elitekv_attend_rows_workspace_size", "elitekv_attend_rows",
+                     "elitekv_ropelite_workspace_size", "elitekv_ropelite_distances", "elitekv_ropelite_search"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -256,6 +260,42 @@ def elitekv_attend_rows(layer: Layer, cache: CacheDesc, q_rope, q_abs, seq_lens,
                                      workspace.numel() * workspace.element_size(), _ptr(out), _stream()),
            "elitekv_attend_rows")
     return out
+
+
+def elitekv_ropelite_workspace_size(n_heads: int, n: int, d_h: int) -> int:
+    b = C.c_size_t()
+    _check(lib().elitekv_ropelite_workspace_size(n_heads, n, d_h, C.byref(b)), "elitekv_ropelite_workspace_size")
+    return b.value
+
+
+def _ropelite_ws(Q):
+    H, n, d_h = Q.shape
+    return torch.empty(elitekv_ropelite_workspace_size(H, n, d_h), dtype=torch.uint8, device=Q.device)
+
+
+def elitekv_ropelite_distances(Q, K, rope_base: float = 10000.0, elite_mask=None, workspace=None):
+    """Q, K bf16 [n_heads][n][d_h]; elite_mask optional int64 [n_heads] (bit i = chunk i chosen).
+    Returns fp32 [n_heads][d_h/2]."""
+    H, n, d_h = Q.shape
+    ws = _ropelite_ws(Q) if workspace is None else workspace
+    dist = torch.empty((H, d_h // 2), dtype=torch.float32, device=Q.device)
+    _check(lib().elitekv_ropelite_distances(_ptr(_dev(Q, torch.bfloat16)), _ptr(_dev(K, torch.bfloat16)), H, n, d_h,
+                                            rope_base, _ptr(_dev(elite_mask, torch.int64)) if elite_mask is not None else None,
+                                            ws.data_ptr(), ws.numel(), _ptr(dist), _stream()),
+           "elitekv_ropelite_distances")
+    return dist
+
+
+def elitekv_ropelite_search(Q, K, r: int, rope_base: float = 10000.0, trace: bool = False, workspace=None):
+    """r greedy rounds for every head.  Returns int32 [n_heads][r] (and fp32 [r][n_heads][d_h/2])."""
+    H, n, d_h = Q.shape
+    ws = _ropelite_ws(Q) if workspace is None else workspace
+    idx = torch.empty((H, r), dtype=torch.int32, device=Q.device)
+    tr = torch.empty((r, H, d_h // 2), dtype=torch.float32, device=Q.device) if trace else None
+    _check(lib().elitekv_ropelite_search(_ptr(_dev(Q, torch.bfloat16)), _ptr(_dev(K, torch.bfloat16)), H, n, d_h,
+                                         rope_base, r, ws.data_ptr(), ws.numel(), _ptr(idx), _ptr(tr), _stream()),
+           "elitekv_ropelite_search")
+    return (idx, tr) if trace else idx
 
 
 class DecodeStepRunner:

@@ -475,6 +475,50 @@ def attend_rows_bench(ek, layer, cache, w, lens, device, flush, cache_bytes, rep
     return out
 
 
+def ropelite_bench(ek, device, reps: int = 3):
+    """RoPElite search (Algorithm 1) on synthetic activations of one 7B-shaped layer: 32 heads,
+    d_h = 128, a calibration sequence of 2048 tokens, r = 8 rounds.  ALU-bound: per causal pair and
+    chunk the kernel issues 9 FP32 lane instructions (two 2-term products, the rotated-minus-plain
+    term, the masked residual sum, the absolute difference into the candidate's running sum);
+    peak = SMs x 128 FP32 lanes x the maximum SM clock."""
+    H, n, d_h, r = 32, 2048, 128, 8
+    g = torch.Generator(device=device).manual_seed(31337)
+    Q = torch.randn((H, n, d_h), generator=g, device=device).to(torch.bfloat16)
+    K = torch.randn((H, n, d_h), generator=g, device=device).to(torch.bfloat16)
+    ws = torch.empty(ek.elitekv_ropelite_workspace_size(H, n, d_h), dtype=torch.uint8, device=device)
+    ek.elitekv_ropelite_search(Q, K, r, workspace=ws)
+    evs = []
+    for _ in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        idx = ek.elitekv_ropelite_search(Q, K, r, workspace=ws)
+        b.record()
+        evs.append((a, b))
+    torch.cuda.synchronize()
+    ms = sum(a.elapsed_time(b) for a, b in evs) / reps
+    pairs = H * n * (n + 1) // 2
+    lane_instr = 9.0 * (d_h // 2) * pairs * r
+    props = torch.cuda.get_device_properties(device)
+    peak = props.multi_processor_count * 128 * 1.965e9
+    # the float64 oracle on a small sample of the same activations: one head, 256 tokens, one round
+    from oracle import ropelite_oracle as RO
+    q64, k64 = Q[0, :256].double().cpu().numpy(), K[0, :256].double().cpu().numpy()
+    t0 = time.perf_counter()
+    want = RO.distances(q64, k64, [], d_h)
+    t_cpu = time.perf_counter() - t0
+    got = ek.elitekv_ropelite_distances(Q[:1, :256].contiguous(), K[:1, :256].contiguous())[0].double().cpu().numpy()
+    return {"heads": H, "tokens": n, "d_h": d_h, "rounds": r, "ms": ms, "ms_per_round": ms / r,
+            "head_rounds_per_s": H * r / (ms * 1e-3),
+            "roofline": {"bound": "alu", "achieved": lane_instr / (ms * 1e-3) / 1e12, "peak": peak / 1e12,
+                         "unit": "T FP32 lane-instr/s", "frac": lane_instr / (ms * 1e-3) / peak,
+                         "peak_kind": "SMs x 128 lanes x 1965 MHz"},
+            "parity_sample": {"rel_err_max": float(np.max(np.abs(got - want) / want))},
+            "cpu_baseline": {"value": 1.0 / (t_cpu * (n * (n + 1) / 2) / (256 * 257 / 2)), "unit": "head-rounds/s",
+                             "kind": "oracle", "cores": oracle_threads(),
+                             "sample": "one head, 256 of 2048 tokens, one round; scaled by the number of causal pairs"},
+            "first_head_elite": idx[0].tolist()}
+
+
 def run_gpu(args, w: gen.Workload):
     from paper_2503_01586_b200 import binding as ek
     ek.lib()   # fail loudly if the CUDA library is missing
@@ -618,7 +662,7 @@ def run_gpu(args, w: gen.Workload):
             comparator = None
 
     # ---- the other benchmark configurations and the prefill append (one GPU, rank 0 only)
-    sweep, prefill, projection, rows = None, None, None, None
+    sweep, prefill, projection, rows, ropelite = None, None, None, None, None
     if rank == 0 and world == 1 and not args.no_sweep:
         rows = attend_rows_bench(ek, layer, cache, w, lens, device, flush, cache_bytes)
         del layer, cache, dev, ws, bufs, keep, eager_runner
@@ -626,6 +670,7 @@ def run_gpu(args, w: gen.Workload):
         t_sweep = time.perf_counter()
         prefill = append_prefill(ek, device, flush)
         projection = project_append_bench(ek, device, flush)
+        ropelite = ropelite_bench(ek, device)
         sweep = []
         for name in SWEEP:
             if name == w.name:
@@ -680,6 +725,7 @@ def run_gpu(args, w: gen.Workload):
     line["stages"]["append_prefill"] = prefill
     line["stages"]["project_append"] = projection
     line["stages"]["attend_rows"] = rows
+    line["stages"]["ropelite_search"] = ropelite
     line["sweep"] = sweep
     print(json.dumps(line))
     if dist is not None:

@@ -14,8 +14,8 @@
 // pairs therefore yields the distances of ALL candidates of a round:  dist[j] = sum |R - D_j|.
 // This is FP32 arithmetic on CUDA cores (there is no contraction deeper than 2 here).
 //
-// distance kernel: grid (row tiles of 4 query positions, heads), 128 threads.  Warp w owns query
-// row m0 + w, its lanes own keys; key tiles of 64 are staged in shared memory as fp32 pairs
+// distance kernel: grid (row tiles of 16 query positions, heads), 128 threads.  Warp w owns query
+// rows m0 + 4 w .. m0 + 4 w + 3, its lanes own keys; key tiles of 64 are staged in shared memory as fp32 pairs
 // [chunk][key] together with the slice of the (cos - 1, sin) table the tile's relative positions
 // need, [chunk][m - n].  A thread keeps the 64 D_i of its pair and 64 running sums in registers.
 // Block results go to a [head][row tile][chunk] array; the select kernel adds them in a fixed
@@ -25,7 +25,9 @@
 
 namespace {
 
-constexpr int kRlRows = 4;        // query rows per block (one per warp)
+constexpr int kRlRows = 16;       // query rows per block (four per warp)
+constexpr int kRlWarps = 4;
+constexpr int kRlRowsPerWarp = kRlRows / kRlWarps;
 constexpr int kRlKeys = 64;       // keys per stage
 constexpr int kRlThreads = 128;
 constexpr int kRlSpan = kRlKeys + kRlRows - 1;     // relative positions a stage can meet
@@ -52,13 +54,12 @@ ropelite_distance_kernel(const bf16* __restrict__ Q, const bf16* __restrict__ K,
   float2 (*s_k)[kRlKeys] = (float2 (*)[kRlKeys])smem_rl;                              // [HALF][keys]
   float2 (*s_t)[kRlSpanPad] = (float2 (*)[kRlSpanPad])(smem_rl + HALF * kRlKeys);     // [HALF][relative position]
   float2 (*s_q)[HALF] = (float2 (*)[HALF])(smem_rl + HALF * (kRlKeys + kRlSpanPad)); // [rows][HALF]
-  float (*s_red)[HALF] = (float (*)[HALF])(smem_rl + HALF * (kRlKeys + kRlSpanPad + kRlRows));
+  float (*s_red)[HALF] = (float (*)[HALF])(smem_rl + HALF * (kRlKeys + kRlSpanPad + kRlRows));       // [warps][HALF]
   const int n_tiles = gridDim.x;
   const int mt = n_tiles - 1 - (int)blockIdx.x;          // long rows first
   const int head = blockIdx.y;
   const int m0 = mt * kRlRows;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m = m0 + warp;
   const unsigned long long mask = masks ? masks[head] : 0ull;
   const bf16* Qh = Q + (size_t)head * n * d_h;
   const bf16* Kh = K + (size_t)head * n * d_h;
@@ -94,16 +95,18 @@ ropelite_distance_kernel(const bf16* __restrict__ Q, const bf16* __restrict__ K,
     }
     __syncthreads();
 #pragma unroll 1
-    for (int u = 0; u < kRlKeys / 32; ++u) {
-      const int nn = lane + 32 * u;
+    for (int e = 0; e < kRlRowsPerWarp * (kRlKeys / 32); ++e) {
+      const int rr = warp * kRlRowsPerWarp + e / (kRlKeys / 32);     // row inside the block
+      const int m = m0 + rr;
+      const int nn = lane + 32 * (e % (kRlKeys / 32));
       const int key = n0 + nn;
       if (!(key <= m && m < n)) continue;                  // causal pairs only
-      const int dd = warp + (kRlKeys - 1) - nn;            // (m - key) - d_min
+      const int dd = rr + (kRlKeys - 1) - nn;              // (m - key) - d_min
       float d[HALF];
       float R = 0.f;
 #pragma unroll
       for (int i = 0; i < HALF; ++i) {
-        const float2 q = s_q[warp][i], k = s_k[i][nn], t = s_t[i][dd];
+        const float2 q = s_q[rr][i], k = s_k[i][nn], t = s_t[i][dd];
         const float a = fmaf(q.x, k.x, q.y * k.y);
         const float b = fmaf(q.y, k.x, -(q.x * k.y));
         d[i] = fmaf(a, t.x, -(b * t.y));
@@ -123,7 +126,7 @@ ropelite_distance_kernel(const bf16* __restrict__ Q, const bf16* __restrict__ K,
   for (int j = threadIdx.x; j < HALF; j += kRlThreads) {
     float v = 0.f;
 #pragma unroll
-    for (int w = 0; w < kRlRows; ++w) v += s_red[w][j];
+    for (int w = 0; w < kRlWarps; ++w) v += s_red[w][j];
     partial[((size_t)head * n_tiles + mt) * HALF + j] = v;
   }
 }
@@ -180,7 +183,7 @@ int rl_launch_distance(const void* Q, const void* K, int heads, int n, int d_h, 
                        const unsigned long long* masks, float* partial, cudaStream_t st) {
   dim3 grid((unsigned)((n + kRlRows - 1) / kRlRows), (unsigned)heads);
   const int half = d_h / 2;
-  const int smem = half * (kRlKeys + kRlSpanPad + kRlRows) * (int)sizeof(float2) + kRlRows * half * (int)sizeof(float);
+  const int smem = half * (kRlKeys + kRlSpanPad + kRlRows) * (int)sizeof(float2) + kRlWarps * half * (int)sizeof(float);
   if (d_h == 128) {
     EKV_CUDA_OK(cudaFuncSetAttribute(ropelite_distance_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     ropelite_distance_kernel<64><<<grid, kRlThreads, smem, st>>>((const bf16*)Q, (const bf16*)K, n, tab, masks, partial);

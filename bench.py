@@ -519,6 +519,21 @@ def ropelite_bench(ek, device, reps: int = 3):
             "first_head_elite": idx[0].tolist()}
 
 
+def run_stage(args):
+    from paper_2503_01586_b200 import binding as ek
+    ek.lib()
+    torch.cuda.set_device(0)
+    device = torch.device("cuda", 0)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=device)
+    if args.stage == "append_prefill":
+        rec = append_prefill(ek, device, flush, reps=2)
+    elif args.stage == "project_append":
+        rec = project_append_bench(ek, device, flush, reps=2)
+    else:
+        rec = ropelite_bench(ek, device, reps=1)
+    print(json.dumps({"stage": args.stage, "record": rec}))
+
+
 def run_gpu(args, w: gen.Workload):
     from paper_2503_01586_b200 import binding as ek
     ek.lib()   # fail loudly if the CUDA library is missing
@@ -798,8 +813,13 @@ def main():
     ap.add_argument("--dry-run-ranks", action="store_true",
                     help="launcher check without a GPU: every rank joins a gloo group, takes part in the "
                          "max-over-ranks reduction of a dummy timing and rank 0 prints a JSON line")
+    ap.add_argument("--stage", default=None, choices=["append_prefill", "project_append", "ropelite_search"],
+                    help="time only this side measurement and print its record (for profiling one kernel)")
     args = ap.parse_args()
     w = gen.CONFIGS[args.workload]
+    if args.stage:
+        run_stage(args)
+        return
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         launch_replicas(args)
         return

@@ -68,13 +68,17 @@ combine_fast_kernel(const float* part_acc, const float* part_ml,   // written by
     cp_async16(&s_w[k][v * 8], Wuv + (size_t)(k0 + k) * n_phys * kFD + (size_t)(h % n_phys) * kFD + v * 8);
   }
   cp_async_commit();
-  ekv_pdl_wait();         // the weights above are constant; everything below reads the split-K kernel's output
-
   const int n_groups = (B + kFB - 1) / kFB;
+  // The plan (seq_first) was written before the split-K kernel started computing (that kernel
+  // waited for it before it let this one be launched), so the first group's item ranges are
+  // fetched while the split-K kernel is still running.
+  if (tid <= min(kFB, B)) s_first[tid] = __ldcg(seq_first + tid);
+  ekv_pdl_wait();         // everything below reads the split-K kernel's output
+
   for (int g = 0; g < n_groups; ++g) {
     const int b0 = g * kFB, nb = min(kFB, B - b0);
     __syncthreads();
-    if (tid <= nb) s_first[tid] = __ldcg(seq_first + b0 + tid);
+    if (g > 0 && tid <= nb) s_first[tid] = __ldcg(seq_first + b0 + tid);
     __syncthreads();
     // (m, l) of the group's items for this head: one trip to global memory, then shared
     const int gi0 = s_first[0], gin = s_first[nb] - gi0;

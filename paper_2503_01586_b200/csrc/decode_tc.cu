@@ -22,10 +22,15 @@
 // With separated latents (S-LRD, Section 3.2: a latent row is [c_k | c_v]) pass A streams only
 // the key latent's chunks and pass B only the value latent's, so nothing is read twice.
 //
+// Layers whose fp32 output is too wide for TMEM even with 32 heads (d_c = 3072) split the
+// OUTPUT columns between two blocks instead of the heads: both blocks compute the scores of all
+// 32 heads (pass A over the whole latent), each accumulates its half of the latent columns in
+// pass B, so a block streams a tile one and a half times instead of twice.
+//
 // A block is a persistent worker: it walks the items of the balanced plan that fall into its
-// share of the batch's tiles and writes one partial result (m, l, acc) per item.  Layers whose
-// fp32 output does not fit TMEM's 512 columns for 32 heads (d_c > 1920) run with 16 heads per
-// block, layers with more than 32 heads as several head groups; the head groups of an item are
+// share of the batch's tiles and writes one partial result (m, l, acc) per item.  Layers with
+// more than 32 heads run as several head groups (and with 16 heads per block where even half the
+// output is too wide for 32); the head groups of an item are
 // adjacent blocks so that they share L2.
 //
 // Roles (288 threads):
@@ -73,6 +78,7 @@ struct TcArgs {
   int kw, voff, vw;         // latent columns of the scores [0, kw) and of the outputs [voff, voff + vw)
   int n_groups;             // blocks per worker: query rows x head groups of N heads; blockIdx.x = worker * n_groups + group
   int rows, gpr, nv;        // query rows per sequence, head groups per row, rows * n_h
+  int vparts;               // blocks that share a head group by splitting the OUTPUT columns between them
   const int32_t* seq_lens;  // rows > 1: row i of sequence b sees seq_lens[b] - (rows - 1 - i) tokens
   float scale_log2e;
 };
@@ -108,16 +114,18 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
                  const TcArgs a) {
   extern __shared__ unsigned char smem_raw[];
   const int worker = blockIdx.x / a.n_groups;         // persistent worker: walks its plan items
-  const int grp = blockIdx.x % a.n_groups;
+  const int grp = (blockIdx.x % a.n_groups) / a.vparts;
+  const int vpart = (blockIdx.x % a.n_groups) % a.vparts;   // which share of the output columns this block accumulates
   const int qrow = grp / a.gpr;                       // query row of this block (0 when decoding)
   const int h0 = (grp % a.gpr) * N;                   // first head of this block's group
   const int vh0 = qrow * a.n_h + h0;                  // the same in the [rows][n_h] layout of queries and results
   const int nh_here = min(N, a.n_h - h0);
   const int d_c = a.d_c;
   const int NKC = a.kw >> 6;     // 64-wide latent chunks of pass A
-  const int NB = a.vw >> 7;      // 128-row output blocks = slot pairs of pass B
+  const int vw_blk = a.vw / a.vparts;                 // output columns of this block
+  const int NB = vw_blk >> 7;    // 128-row output blocks = slot pairs of pass B
   const int NUSE = NKC + 2 * NB; // ring uses per tile
-  const int vc0 = a.voff >> 6;   // first 64-wide chunk of the columns pass B reads
+  const int vc0 = (a.voff + vpart * vw_blk) >> 6;     // first 64-wide chunk of the columns pass B reads
   const bool reread = a.voff == 0;   // joint latent: pass B reads what pass A read
   constexpr int NRB = N * R2 / 64;   // rope boxes per tile
   constexpr int HPB = 64 / R2;       // heads per rope box
@@ -518,7 +526,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
       named_bar_sync(1, kSoftmaxThreads);
       if (lane < N) s_wmax[quarter * N + lane] = wl;
       named_bar_sync(1, kSoftmaxThreads);
-      if (quarter == 0 && lane < nh_here) {
+      if (quarter == 0 && lane < nh_here && vpart == 0) {     // the blocks of a head group hold the same statistics
         const float lsum = s_wmax[lane] + s_wmax[N + lane] + s_wmax[2 * N + lane] + s_wmax[3 * N + lane];
         a.part_ml[((size_t)item * a.nv + vh0 + lane) * 2 + 0] = m_ref;
         a.part_ml[((size_t)item * a.nv + vh0 + lane) * 2 + 1] = lsum;
@@ -548,7 +556,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
         fence_proxy_async();
         named_bar_sync(1, kSoftmaxThreads);
         if (threadIdx.x == 64) {
-          tma_store_4d(&map_part, blk * 128, h0, qrow, item, smem_u32(tile_s));
+          tma_store_4d(&map_part, vpart * vw_blk + blk * 128, h0, qrow, item, smem_u32(tile_s));
           bulk_commit_group();
         }
       }
@@ -578,12 +586,21 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap map_lat, const __grid_const
 
 }  // namespace
 
-// Heads per block: 32 when 32 fp32 output columns per 128 latent coordinates plus the score
-// columns fit TMEM's 512 columns (d_c <= 1920), else 16.  A layer with more heads than that runs
-// as head groups (the last one partly filled: 40 heads = 32 + 8); each group streams the token
-// tile itself, and the groups of an item are adjacent blocks so that the later readers hit L2.
-static int tc_pick_n(const elitekv_layer* L) {
+// Heads per block: 32 when 32 fp32 output columns per 128 latent coordinates of the block's
+// output share plus the score columns fit TMEM's 512 columns, else 16.  A layer with more heads
+// than that runs as head groups (the last one partly filled: 40 heads = 32 + 8); each group
+// streams the token tile itself, and the blocks of an item are adjacent so that the later readers
+// hit L2.
+// Output-column shares per head group: 1, or 2 when only half of the output fits TMEM beside
+// the scores of 32 heads.
+static int tc_pick_parts(const elitekv_layer* L) {
   const int nb = L->vw / 128;
+  if ((nb + 1) * 32 <= 512) return 1;
+  if (L->n_h <= 32 && nb % 2 == 0 && (nb / 2 + 1) * 32 <= 512) return 2;
+  return 1;
+}
+static int tc_pick_n(const elitekv_layer* L) {
+  const int nb = L->vw / 128 / tc_pick_parts(L);
   if ((nb + 1) * 32 <= 512) return 32;
   if ((nb + 1) * 16 <= 512) return 16;
   return 0;
@@ -604,7 +621,7 @@ int ekv_tc_supported(const elitekv_layer* L, const elitekv_cache* cache) {
   return 1;
 }
 
-static int tc_groups(const elitekv_layer* L) {
+static int tc_groups(const elitekv_layer* L) {      // head groups per query row
   const int n = tc_pick_n(L);
   return n ? (L->n_h + n - 1) / n : 1;
 }
@@ -612,7 +629,7 @@ static int tc_groups(const elitekv_layer* L) {
 // One persistent worker (a block per query row and head group) per SM share; items = workers +
 // sequences at most.
 int ekv_tc_workers(const elitekv_layer* L, int rows) {
-  const int per = tc_groups(L) * (rows > 0 ? rows : 1);
+  const int per = tc_groups(L) * tc_pick_parts(L) * (rows > 0 ? rows : 1);
   return L->sm_count / per > 0 ? L->sm_count / per : 1;
 }
 int ekv_tc_max_items(const elitekv_layer* L, int B, int rows) { return ekv_tc_workers(L, rows) + B; }
@@ -654,7 +671,8 @@ int ekv_launch_decode_tc(const elitekv_layer* L, const elitekv_cache* cache, con
   a.vw = L->vw;
   a.rows = rows_q;
   a.gpr = tc_groups(L);
-  a.n_groups = a.gpr * rows_q;
+  a.vparts = tc_pick_parts(L);
+  a.n_groups = a.gpr * rows_q * a.vparts;
   a.nv = rows_q * L->n_h;
   a.seq_lens = ws.seq_lens;
   a.scale_log2e = L->scale * 1.4426950408889634f;

@@ -46,6 +46,8 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
   const int qpitch = kpad + 8;                       // row pitch of the query tile (bank spread)
   bf16* s_w = (bf16*)smem_b;                         // [kpad][128 + 8] weight slab
   bf16* s_q = s_w + (size_t)kpad * kAbsorbPitch;    // [16][qpitch] un-rotated query dims
+  bf16* s_raw = s_q + (size_t)kAbsorbBatch * qpitch;    // [16][d_h] whole query rows as they come (16-byte aligned: both sizes before it are multiples of 8 elements)
+  int* s_dims = (int*)(s_raw + (size_t)kAbsorbBatch * d_h);   // [dn] query dim of every K index
   __shared__ __align__(8) uint64_t w_bar;
   __shared__ int s_abort;
   const bool rope_block = blockIdx.y == gridDim.y - 1;      // last grid row: query RoPE only
@@ -100,12 +102,29 @@ absorb_kernel(const bf16* __restrict__ q, const int32_t* __restrict__ q_pos, int
   for (int b0 = 0; b0 < B; b0 += kAbsorbBatch) {
     const int nb = min(kAbsorbBatch, B - b0);
     __syncthreads();
-    // un-rotated query dims of 16 sequences, bf16 as they come; K padding and missing rows are zeros
+    // un-rotated query dims of 16 sequences, bf16 as they come; K padding and missing rows are
+    // zeros.  The dim table and the query rows are fetched side by side (whole rows, 16-byte
+    // loads) and the gather runs out of shared memory: one trip to memory instead of two
+    // dependent ones.
+    if (b0 == 0)
+      for (int i = threadIdx.x; i < dn; i += blockDim.x) s_dims[i] = __ldg(dims + 2 * r + i);
+    if ((d_h & 7) == 0) {
+      for (int e = threadIdx.x; e < kAbsorbBatch * (d_h / 8); e += blockDim.x) {
+        const int bb = e / (d_h / 8), v = e % (d_h / 8);
+        uint4 raw = make_uint4(0, 0, 0, 0);
+        if (bb < nb) raw = __ldg((const uint4*)(q + ((size_t)(b0 + bb) * n_h + h) * d_h) + v);
+        *(uint4*)(s_raw + (size_t)bb * d_h + v * 8) = raw;
+      }
+    } else {      // head dims that are not whole 16-byte units: element by element
+      for (int e = threadIdx.x; e < kAbsorbBatch * d_h; e += blockDim.x) {
+        const int bb = e / d_h, v = e % d_h;
+        s_raw[e] = bb < nb ? q[((size_t)(b0 + bb) * n_h + h) * d_h + v] : __float2bfloat16_rn(0.f);
+      }
+    }
+    __syncthreads();
     for (int e = threadIdx.x; e < kAbsorbBatch * kpad; e += blockDim.x) {
       const int bb = e / kpad, i = e % kpad;
-      bf16 v = __float2bfloat16_rn(0.f);
-      if (bb < nb && i < dn) v = q[((size_t)(b0 + bb) * n_h + h) * d_h + dims[2 * r + i]];
-      s_q[bb * qpitch + i] = v;
+      s_q[bb * qpitch + i] = i < dn ? s_raw[(size_t)bb * d_h + s_dims[i]] : __float2bfloat16_rn(0.f);
     }
     __syncthreads();
     if (!w_ready) {
@@ -158,7 +177,8 @@ int ekv_launch_absorb(const elitekv_layer* L, const void* q, const int32_t* q_po
   // the absorbed query spans the latent columns the scores read (all of them, or the key latent)
   dim3 grid(L->n_h, (L->kw + kAbsorbCoords - 1) / kAbsorbCoords + 1);   // + one row of rope blocks
   const int kpad = (L->dn + 15) & ~15;
-  const size_t smem = sizeof(bf16) * ((size_t)kpad * kAbsorbPitch + (size_t)kAbsorbBatch * (kpad + 8)) + 16;
+  const size_t smem = sizeof(bf16) * ((size_t)kpad * kAbsorbPitch + (size_t)kAbsorbBatch * (kpad + 8) +
+                                      (size_t)kAbsorbBatch * L->d_h) + sizeof(int) * (size_t)L->dn + 16;
   if ((int)smem > L->smem_optin || L->kw % 8 != 0) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
   EKV_CUDA_OK(cudaFuncSetAttribute(absorb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   absorb_kernel<<<grid, kAbsorbThreads, smem, st>>>(

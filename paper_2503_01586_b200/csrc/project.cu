@@ -9,7 +9,8 @@
 // (cos, sin) of pos * theta_{idx[h][j]}, everything is rounded once to bf16 and written straight
 // to the token's cache row (contiguous or paged).  k_e and c never touch memory.
 //
-// One block computes a [128 tokens x 128 output columns] tile: warp 0 streams the operand tiles
+// One block computes a [128 tokens x 128 output columns] tile (prefill-sized calls: 256 x 256,
+// see further down): warp 0 streams the operand tiles
 // ([128 x 64] of x and of the transposed weight, 128-byte swizzle) through a 4-stage ring, warp 1
 // issues tcgen05.mma (M = 128, N = 128, K = 16, bf16 in, fp32 in TMEM), warps 2-5 run the epilogue.
 // A tile lies either in the rope part or in the latent part (both are multiples of 128 wide).
@@ -240,6 +241,133 @@ project_append_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
   }
 }
 
+// ------------------------------------------------------------------ prefill form: 256 x 256 tiles
+// A 128 x 128 tile asks L2 for 32 KB of operands per 256 tensor-core clocks; at prefill size all
+// SMs together ask for more than L2 delivers, and the tensor pipe idles more than half of the
+// time.  A block of the prefill form computes 256 tokens x 256 columns: the two halves of the
+// token rows are two accumulators (TMEM columns 0-255 and 256-511) that share every weight tile,
+// so a stage of 64 KB (256 rows of x and 256 rows of the weights, 64 of d each) feeds eight
+// M128 N256 K16 MMAs = 1024 clocks: half the operand bytes per flop.
+constexpr int kBM = 256, kBN = 256;
+constexpr int kBStages = 3;
+constexpr int kBStageBytes = (kBM + kBN) * kPK * 2;   // 64 KB
+constexpr int kBThreads = 224;    // warp 0 loads x, warp 6 the weights (one issuing warp draws ~50 GB/s, two
+                                  // about twice that), warp 1 issues the MMAs, warps 2-5 run the epilogue
+
+struct __align__(8) BigBarriers {
+  uint64_t full[kBStages], empty[kBStages], done;
+};
+
+__global__ void __launch_bounds__(kBThreads, 1)
+project_append_big_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                          const ProjArgs a) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* base = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  BigBarriers* bars = (BigBarriers*)(base + kBStages * kBStageBytes);
+  uint32_t* s_tmem = (uint32_t*)(bars + 1);
+  volatile int* s_abort = (volatile int*)(s_tmem + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n0 = blockIdx.x * kBN;
+  const long long t0 = (long long)blockIdx.y * kBM;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kBStages; ++i) {
+      mbar_init(smem_u32(&bars->full[i]), 2);      // one arrival per loading warp
+      mbar_init(smem_u32(&bars->empty[i]), 1);
+    }
+    mbar_init(smem_u32(&bars->done), 1);
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+  }
+  constexpr uint32_t tmem_cols = 512;      // the whole tensor memory: one block per SM (192 KB of shared memory)
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+
+  if (warp == 0 || warp == 6) {
+    // ---- warp 0: one 256-row box of x per stage (rows past the end: zeros); warp 6: one of the weights
+    const bool wload = warp == 6;
+    bool ok = true;
+    for (int k = 0; k < a.nk && ok; ++k) {
+      const int s = k % kBStages;
+      ok = warp_wait(smem_u32(&bars->empty[s]), ((k / kBStages) & 1) ^ 1, s_abort, wload ? 4 : 1);
+      if (!ok) break;
+      if (elect_one()) {
+        const uint32_t fb = smem_u32(&bars->full[s]);
+        mbar_expect_tx(fb, (uint32_t)(kBStageBytes / 2));
+        if (wload) tma_load_2d(smem_u32(base + s * kBStageBytes + kBM * kPK * 2), &map_w, k * kPK, n0, fb);
+        else tma_load_2d(smem_u32(base + s * kBStageBytes), &map_x, k * kPK, (int)t0, fb);
+      }
+      __syncwarp();
+    }
+  } else if (warp == 1) {
+    constexpr uint32_t idesc = make_idesc(128, kBN, 0, 0);
+    constexpr uint32_t hi_sw = desc_hi(1024, 2);
+    const uint32_t base16 = (smem_u32(base) >> 4) & 0x3FFFu;
+    bool ok = true;
+    for (int k = 0; k < a.nk && ok; ++k) {
+      const int s = k % kBStages;
+      ok = warp_wait(smem_u32(&bars->full[s]), (k / kBStages) & 1, s_abort, 2);
+      if (!ok) break;
+      const uint32_t la0 = (base16 + (uint32_t)s * (kBStageBytes >> 4)) | (1u << 16);   // token rows 0-127
+      const uint32_t la1 = la0 + ((128 * kPK * 2) >> 4);                                // token rows 128-255
+      const uint32_t lb = la0 + ((kBM * kPK * 2) >> 4);
+      if (elect_one()) {
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {          // +32 bytes along d per step
+          tc_mma_w(tmem_base, la0 + 2 * ks, hi_sw, lb + 2 * ks, hi_sw, idesc, (k | ks) != 0);
+          tc_mma_w(tmem_base + kBN, la1 + 2 * ks, hi_sw, lb + 2 * ks, hi_sw, idesc, (k | ks) != 0);
+        }
+        tc_commit(smem_u32(&bars->empty[s]));
+      }
+      __syncwarp();
+    }
+    if (ok && elect_one()) tc_commit(smem_u32(&bars->done));
+    __syncwarp();
+  } else {
+    // ---- epilogue: a thread owns token rows trow and trow + 128 of the tile
+    const int quarter = warp & 3;
+    const int trow = quarter * 32 + lane;
+    long long row[2];
+    int p[2] = {0, 0};
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf) {
+      const long long t = t0 + hf * 128 + trow;
+      row[hf] = t < a.T ? token_row(a, t, &p[hf]) : -1;
+    }
+    const bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->done), 0, s_abort, 3));
+    tc_fence_after();
+    if (ok) {
+#pragma unroll 1
+      for (int hf = 0; hf < 2; ++hf) {
+        for (int cc = 0; cc < kBN / 32; ++cc) {
+          float v[32];
+          tc_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(hf * kBN + cc * 32), v);
+          tc_wait_ld();
+          if (row[hf] < 0) continue;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) finish_columns(a, v + 8 * q, row[hf], p[hf], n0 + cc * 32 + 8 * q);
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*s_abort) drain_after_abort();
+  if (threadIdx.x == 0 && *s_abort) ekv_record(a.status, ELITEKV_ERR_TIMEOUT, (int)blockIdx.x | (*s_abort << 16), (int)blockIdx.y);
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+  }
+}
+
 }  // namespace
 
 int ekv_launch_project_append(const elitekv_layer* L, const elitekv_cache* cache, const CacheView& cv,
@@ -249,6 +377,26 @@ int ekv_launch_project_append(const elitekv_layer* L, const elitekv_cache* cache
   const int n_out = rope_w + L->d_c;
   if (L->d % kPK != 0 || rope_w % kPN != 0 || L->d_c % kPN != 0) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
   if (T >= (1ll << 31)) return ELITEKV_ERR_UNSUPPORTED_SHAPE;
+  // prefill-sized calls whose output width is whole 256-column tiles: the 256 x 256 form
+  if (T >= 1024 && n_out % kBN == 0) {
+    const int smem_big = kBStages * kBStageBytes + (int)sizeof(BigBarriers) + 64 + 1024;
+    if (smem_big <= L->smem_optin) {
+      CUtensorMap b_x, b_w;
+      int rcb = make_map(&b_x, x, (unsigned long long)T, (unsigned long long)L->d, kBM);
+      if (rcb == ELITEKV_OK) rcb = make_map(&b_w, L->d_WcatT, (unsigned long long)n_out, (unsigned long long)L->d, kBN);
+      if (rcb != ELITEKV_OK) return rcb;
+      ProjArgs b;
+      b.seq_id = seq_id; b.pos = pos; b.T = T;
+      b.rope = (bf16*)cache->rope; b.latent = (bf16*)cache->latent; b.cv = cv;
+      b.idx = L->d_idx; b.cs = L->d_cs; b.rope_w = rope_w; b.d_c = L->d_c;
+      b.half = L->d_h / 2; b.max_pos = L->max_pos; b.nk = L->d / kPK; b.status = L->d_status;
+      EKV_CUDA_OK(cudaFuncSetAttribute(project_append_big_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_big));
+      dim3 grid((unsigned)(n_out / kBN), (unsigned)((T + kBM - 1) / kBM));
+      project_append_big_kernel<<<grid, kBThreads, smem_big, st>>>(b_x, b_w, b);
+      EKV_CUDA_OK(cudaGetLastError());
+      return ELITEKV_OK;
+    }
+  }
   // at most one token tile and enough depth for every block of a cluster: the split-depth form
   const bool split = T <= kPM && L->d / kPK >= kSplit;
   const int smem = kPStages * kPStageBytes + (split ? kRecvBytes : 0) + (int)sizeof(ProjBarriers) + 64 + 1024;

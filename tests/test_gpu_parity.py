@@ -214,6 +214,20 @@ def test_project_append_split_depth_uneven_shares(ek):
     _projection_case(ek, gen.shrink(gen.SWEEP_875, B=1, ctx=5), 576, [5], False, 99)
 
 
+@pytest.mark.parametrize("paged", [False, True])
+def test_project_append_prefill_sized_call(ek, paged):
+    """1000+ tokens with an output width of whole 256-column tiles take the 256 x 256 form (two
+    accumulators sharing every weight tile).  7B shape: 1400 tokens = 5 full token tiles and a
+    ragged sixth, shuffled order."""
+    _projection_case(ek, gen.shrink(gen.LLAMA7B_75, B=3, ctx=1000), 4096, [1000, 337, 63], paged, 101 + paged)
+
+
+def test_project_append_prefill_form_rope_boundary_inside_a_tile(ek):
+    """13B shape: 640 rope columns + 1920 latent columns = ten 256-column tiles, the third of
+    which holds rope columns and latent columns side by side."""
+    _projection_case(ek, gen.shrink(gen.LLAMA13B_75, B=2, ctx=900), 5120, [900, 300], False, 103)
+
+
 def test_project_append_needs_projection_weights_and_a_covered_shape(ek):
     w = replace(SMALL, seed=95)
     st = H.setup(w, lens=[5, 5, 5])

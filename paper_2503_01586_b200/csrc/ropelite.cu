@@ -51,10 +51,11 @@ ropelite_distance_kernel(const bf16* __restrict__ Q, const bf16* __restrict__ K,
                          float* __restrict__ partial /* [heads][row tiles][HALF] */) {
   constexpr int d_h = 2 * HALF;
   extern __shared__ __align__(16) float2 smem_rl[];
-  float2 (*s_k)[kRlKeys] = (float2 (*)[kRlKeys])smem_rl;                              // [HALF][keys]
-  float2 (*s_t)[kRlSpanPad] = (float2 (*)[kRlSpanPad])(smem_rl + HALF * kRlKeys);     // [HALF][relative position]
-  float2 (*s_q)[HALF] = (float2 (*)[HALF])(smem_rl + HALF * (kRlKeys + kRlSpanPad)); // [rows][HALF]
-  float (*s_red)[HALF] = (float (*)[HALF])(smem_rl + HALF * (kRlKeys + kRlSpanPad + kRlRows));       // [warps][HALF]
+  // keys stay packed as they come (a bf16 pair per chunk: one 4-byte load per pair and chunk, widened in registers)
+  float2 (*s_t)[kRlSpanPad] = (float2 (*)[kRlSpanPad])smem_rl;                        // [HALF][relative position]
+  float2 (*s_q)[HALF] = (float2 (*)[HALF])(smem_rl + HALF * kRlSpanPad);             // [rows][HALF]
+  float (*s_red)[HALF] = (float (*)[HALF])(smem_rl + HALF * (kRlSpanPad + kRlRows)); // [warps][HALF]
+  uint32_t (*s_k)[kRlKeys] = (uint32_t (*)[kRlKeys])(&s_red[kRlWarps][0]);           // [HALF][keys]
   const int n_tiles = gridDim.x;
   const int mt = n_tiles - 1 - (int)blockIdx.x;          // long rows first
   const int head = blockIdx.y;
@@ -82,9 +83,8 @@ ropelite_distance_kernel(const bf16* __restrict__ Q, const bf16* __restrict__ K,
       const int nn = e % kRlKeys, g4 = e / kRlKeys;         // 4 chunks = 8 elements = 16 bytes
       uint4 raw = make_uint4(0, 0, 0, 0);
       if (n0 + nn < n) raw = *(const uint4*)(Kh + (size_t)(n0 + nn) * d_h + g4 * 8);
-      const bf162* p = (const bf162*)&raw;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) s_k[g4 * 4 + c][nn] = __bfloat1622float2(p[c]);
+      s_k[g4 * 4 + 0][nn] = raw.x; s_k[g4 * 4 + 1][nn] = raw.y;
+      s_k[g4 * 4 + 2][nn] = raw.z; s_k[g4 * 4 + 3][nn] = raw.w;
     }
     // table slice: relative positions d_min .. d_min + span - 1 (negative ones belong to masked pairs)
     const int d_min = m0 - n0 - (kRlKeys - 1);
@@ -106,7 +106,9 @@ ropelite_distance_kernel(const bf16* __restrict__ Q, const bf16* __restrict__ K,
       float R = 0.f;
 #pragma unroll
       for (int i = 0; i < HALF; ++i) {
-        const float2 q = s_q[rr][i], k = s_k[i][nn], t = s_t[i][dd];
+        const float2 q = s_q[rr][i], t = s_t[i][dd];
+        const uint32_t kp = s_k[i][nn];
+        const float2 k = make_float2(__uint_as_float(kp << 16), __uint_as_float(kp & 0xffff0000u));   // bf16 pair -> fp32
         const float a = fmaf(q.x, k.x, q.y * k.y);
         const float b = fmaf(q.y, k.x, -(q.x * k.y));
         d[i] = fmaf(a, t.x, -(b * t.y));
@@ -183,7 +185,8 @@ int rl_launch_distance(const void* Q, const void* K, int heads, int n, int d_h, 
                        const unsigned long long* masks, float* partial, cudaStream_t st) {
   dim3 grid((unsigned)((n + kRlRows - 1) / kRlRows), (unsigned)heads);
   const int half = d_h / 2;
-  const int smem = half * (kRlKeys + kRlSpanPad + kRlRows) * (int)sizeof(float2) + kRlWarps * half * (int)sizeof(float);
+  const int smem = half * (kRlSpanPad + kRlRows) * (int)sizeof(float2) + kRlWarps * half * (int)sizeof(float) +
+                   half * kRlKeys * (int)sizeof(uint32_t);
   if (d_h == 128) {
     EKV_CUDA_OK(cudaFuncSetAttribute(ropelite_distance_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     ropelite_distance_kernel<64><<<grid, kRlThreads, smem, st>>>((const bf16*)Q, (const bf16*)K, n, tab, masks, partial);

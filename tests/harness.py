@@ -58,6 +58,7 @@ def setup(w: gen.Workload, *, lens: Optional[Sequence[int]] = None, decode_kerne
     overwrite rows of st.k_e / st.c before they are appended."""
     idx = gen.elite_index_sets(w)
     W_uk, W_uv = gen.up_projections(w, device)
+    d_ck = d_ck or w.d_ck
     if d_ck:
         # S-LRD: B^k_S reads the first d_ck latent columns, B^v_S the remaining ones
         W_uk, W_uv = W_uk[:d_ck].contiguous(), W_uv[d_ck:].contiguous()

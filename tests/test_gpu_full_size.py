@@ -103,3 +103,39 @@ def test_config5_prefill_append_4096_tokens_bit_exact(ek):
                                           table32=table32.cpu().numpy())
     assert np.array_equal(H.bits(st.latent_plane), lat_exp)
     assert np.array_equal(H.bits(st.rope_plane), rope_exp)
+
+
+def test_separated_latents_b32_ctx8192(ek):
+    """The sweep's S-LRD configuration (key latent 512, value latent 1024) at full size."""
+    _run(ek, gen.SWEEP_75_SLRD, 8)
+
+
+def test_query_rows_on_the_benchmark_workload(ek):
+    """Four causal query rows per sequence over the benchmark workload's cache (the shape
+    bench.py times for elitekv_attend_rows): sampled (sequence, head) units, all four rows each,
+    against the oracle's causal definition at full context."""
+    from oracle import elitekv_oracle as O
+    w, m = gen.LLAMA7B_75, 4
+    st = H.setup(w)
+    g = torch.Generator(device="cpu").manual_seed(77)
+    q = torch.randn((w.B, m, w.n_h, w.d_h), generator=g).to(torch.bfloat16).cuda()
+    q_pos = (st.lens_dev.view(-1, 1) - m + torch.arange(m, device="cuda", dtype=torch.int32).view(1, m)).to(torch.int32)
+    q_rope, q_abs = ek.elitekv_absorb_query(st.layer, q.view(w.B * m, w.n_h, w.d_h), q_pos.reshape(-1).contiguous())
+    ws = torch.empty(ek.elitekv_attend_rows_workspace_size(st.layer, w.B, m), dtype=torch.uint8, device="cuda")
+    out = ek.elitekv_attend_rows(st.layer, st.cache, q_rope, q_abs, st.lens_dev, m, ws)
+    torch.cuda.synchronize()
+    assert ek.elitekv_check_status(st.layer) == 0
+    assert torch.isfinite(out.float()).all()
+    idx = st.idx.numpy().astype(np.int64)
+    W_uk, W_uv = H.f64(st.W_uk), H.f64(st.W_uv)
+    for b, h in H.sample_units(st, 6, seed=21):
+        lo, hi = int(st.starts[b]), int(st.starts[b + 1])
+        n = hi - lo
+        key_pos = np.arange(n)
+        k_rope = O.rotate_elite_keys(H.f64(st.k_e[lo:hi]), key_pos, idx, w.d_h, w.rope_base)
+        want = O.attend_causal(H.f64(q[b]), n - m + np.arange(m), k_rope, key_pos, H.f64(st.c[lo:hi]), W_uk, W_uv,
+                               idx, w.d_h, base=w.rope_base, heads=[h])[:, 0]
+        rel, mx = H.errors(H.f64(out[b, :, h]), want)
+        assert rel <= H.REL_L2_TOL and mx <= H.MAX_ABS_TOL, (b, h, rel, mx)
+    del st, out
+    _free()
